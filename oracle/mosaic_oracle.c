@@ -1,0 +1,369 @@
+/*
+ * mosaic_oracle.c -- TEST INFRASTRUCTURE, not part of the product.
+ *
+ * A plain, slow, fp64 CPU statement of what the MOSAIC block-sparse attention
+ * path computes, written from the paper's equations.  Only the tests, the smoke
+ * check and the benchmark's CPU-baseline leg may call it; the CUDA library never
+ * does, and the two share no code.
+ *
+ * Conventions (one "unit" = one (batch, head) pair; units are independent because
+ * every equation of the method is per head and per sample):
+ *   grid nlat x nlon, token t = lat*nlon + lon, head dim d;
+ *   block (by,bx) holds tokens (by*bh + r, bx*bw + c), r < bh, c < bw; id j = by*nbw + bx;
+ *   inputs are bf16 bit patterns (uint16), widened exactly to double.
+ *
+ * Steps and where the paper defines them:
+ *   pooling      -- "Compression" paragraph of the Block-Sparse Attention section
+ *                   (block representations via phi = mean pooling); the mean's 1/b is
+ *                   dropped because a positive constant cannot change a ranking.
+ *   block score  -- block-level attention equation of the same paragraph; the exp and
+ *                   the normalisation are strictly increasing per row, so the raw dot
+ *                   product of pooled vectors ranks identically.
+ *   top-n        -- "Selection" paragraph: the n best key blocks per query block,
+ *                   shared by every token of that block.  Here the candidates are the
+ *                   non-local blocks and ties go to the lower block id.
+ *   attention    -- the fine-grained attention equation of the "Selection" paragraph,
+ *                   taken over the union of the local neighbourhood and the selected
+ *                   blocks with ONE softmax (scale 1/sqrt(d_k) unless overridden).
+ *   backward     -- analytic gradient of that softmax attention with the selection
+ *                   held constant; dK/dV visit only the query blocks connected to a
+ *                   key/value block ("Kernel Design" paragraph of the appendix).
+ *
+ * Pins (tests/test_oracle_*.py): dense attention when top-k covers every block,
+ * brute-force selection on tiny grids, hand-built winners and ties, row-stochastic
+ * weights, convex-hull bound, finite differences, longitude-roll equivariance,
+ * zero gradient for unconnected blocks, the cost-model pair count.
+ * Parity unpinned: agreement with the authors' own kernels (not available).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+typedef struct mo_geom {
+  int32_t nlat, nlon, d;
+  int32_t bh, bw;
+  int32_t rlat, rlon;
+  int32_t topk;
+  double scale; /* softmax scale; <= 0 means 1/sqrt(d) */
+} mo_geom;
+
+#define MO_MAX_LOCAL 256
+
+static int g_ok(const mo_geom *g) {
+  if (!g || g->nlat <= 0 || g->nlon <= 0 || g->d <= 0 || g->bh <= 0 || g->bw <= 0) return 0;
+  if (g->nlat % g->bh || g->nlon % g->bw) return 0;
+  if (g->rlat < 0 || g->rlon < 0 || g->topk < 0) return 0;
+  if ((2 * g->rlat + 1) * (2 * g->rlon + 1) > MO_MAX_LOCAL) return 0;
+  return 1;
+}
+static int g_nbh(const mo_geom *g) { return g->nlat / g->bh; }
+static int g_nbw(const mo_geom *g) { return g->nlon / g->bw; }
+static int g_m(const mo_geom *g) { return g_nbh(g) * g_nbw(g); }
+static int g_b(const mo_geom *g) { return g->bh * g->bw; }
+static double g_scale(const mo_geom *g) { return g->scale > 0.0 ? g->scale : 1.0 / sqrt((double)g->d); }
+
+static double bf16_widen(uint16_t h) {
+  uint32_t u = (uint32_t)h << 16;
+  float f;
+  memcpy(&f, &u, sizeof f);
+  return (double)f;
+}
+
+/* token index of element e (row-major inside the block) of block j */
+static int64_t block_token(const mo_geom *g, int j, int e) {
+  int nbw = g_nbw(g);
+  int by = j / nbw, bx = j % nbw;
+  int r = e / g->bw, c = e % g->bw;
+  return (int64_t)(by * g->bh + r) * g->nlon + (bx * g->bw + c);
+}
+
+int mo_num_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+/*
+ * Local set of query block i: rows clamp(by+dy), columns (bx+dx) mod nbw, as a SET
+ * (each block once), listed in first-occurrence order over dy, then dx ascending.
+ */
+int mo_local_set(const mo_geom *g, int32_t i, int32_t *out) {
+  if (!g_ok(g)) return -1;
+  int nbh = g_nbh(g), nbw = g_nbw(g);
+  int by = i / nbw, bx = i % nbw, n = 0;
+  for (int dy = -g->rlat; dy <= g->rlat; ++dy) {
+    int y = by + dy;
+    if (y < 0) y = 0;
+    if (y > nbh - 1) y = nbh - 1;
+    for (int dx = -g->rlon; dx <= g->rlon; ++dx) {
+      int x = ((bx + dx) % nbw + nbw) % nbw;
+      int id = y * nbw + x, seen = 0;
+      for (int a = 0; a < n; ++a) seen |= (out[a] == id);
+      if (!seen) out[n++] = id;
+    }
+  }
+  return n;
+}
+
+/* Block sums of one [N,d] bf16 tensor: sequential fp64 accumulation in row-major
+ * block order, rounded once to fp32. */
+int mo_pool_unit(const mo_geom *g, const uint16_t *x, float *pooled /* [m,d] */) {
+  if (!g_ok(g)) return -1;
+  int m = g_m(g), b = g_b(g), d = g->d;
+#pragma omp parallel for schedule(static)
+  for (int j = 0; j < m; ++j) {
+    for (int c = 0; c < d; ++c) {
+      double acc = 0.0;
+      for (int e = 0; e < b; ++e) acc += bf16_widen(x[block_token(g, j, e) * d + c]);
+      pooled[(size_t)j * d + c] = (float)acc;
+    }
+  }
+  return 0;
+}
+
+typedef struct { double s; int32_t j; } mo_cand;
+
+/* rank order: higher score first; a NaN ranks below every number; equal scores
+ * (+0 and -0 compare equal) go to the lower block id. */
+static int cand_cmp(const void *pa, const void *pb) {
+  const mo_cand *a = (const mo_cand *)pa, *b = (const mo_cand *)pb;
+  int an = isnan(a->s), bn = isnan(b->s);
+  if (an != bn) return an ? 1 : -1;
+  if (!an) {
+    if (a->s > b->s) return -1;
+    if (a->s < b->s) return 1;
+  }
+  return (a->j > b->j) - (a->j < b->j);
+}
+
+/*
+ * Selection for one unit.  idx is [m, topk]; row i lists the chosen non-local block
+ * ids best first, padded with -1.  pq/pk (optional, [m,d] fp32) receive the pooled sums.
+ */
+int mo_select_unit(const mo_geom *g, const uint16_t *q, const uint16_t *k, int32_t *idx,
+                   float *pq_out, float *pk_out) {
+  if (!g_ok(g)) return -1;
+  int m = g_m(g), d = g->d, topk = g->topk;
+  float *pq = (float *)malloc(sizeof(float) * (size_t)m * d);
+  float *pk = (float *)malloc(sizeof(float) * (size_t)m * d);
+  if (!pq || !pk) { free(pq); free(pk); return -2; }
+  mo_pool_unit(g, q, pq);
+  mo_pool_unit(g, k, pk);
+#pragma omp parallel
+  {
+    mo_cand *cand = (mo_cand *)malloc(sizeof(mo_cand) * (size_t)m);
+    int32_t loc[MO_MAX_LOCAL];
+#pragma omp for schedule(dynamic, 4)
+    for (int i = 0; i < m; ++i) {
+      int nl = mo_local_set(g, i, loc), nc = 0;
+      for (int j = 0; j < m; ++j) {
+        int is_local = 0;
+        for (int a = 0; a < nl; ++a) is_local |= (loc[a] == j);
+        if (is_local) continue;
+        double s = 0.0;
+        for (int c = 0; c < d; ++c) s += (double)pq[(size_t)i * d + c] * (double)pk[(size_t)j * d + c];
+        cand[nc].s = s;
+        cand[nc].j = j;
+        ++nc;
+      }
+      qsort(cand, (size_t)nc, sizeof(mo_cand), cand_cmp);
+      for (int r = 0; r < topk; ++r) idx[(size_t)i * topk + r] = r < nc ? cand[r].j : -1;
+    }
+    free(cand);
+  }
+  if (pq_out) memcpy(pq_out, pq, sizeof(float) * (size_t)m * d);
+  if (pk_out) memcpy(pk_out, pk, sizeof(float) * (size_t)m * d);
+  free(pq);
+  free(pk);
+  return 0;
+}
+
+/* attended block list of query block i: local set, then the selected ids >= 0 */
+static int attended(const mo_geom *g, const int32_t *idx, int i, int32_t *out) {
+  int n = mo_local_set(g, i, out);
+  for (int r = 0; r < g->topk; ++r) {
+    int32_t j = idx[(size_t)i * g->topk + r];
+    if (j >= 0) out[n++] = j;
+  }
+  return n;
+}
+
+/* logits x_t = scale * q_l . k_t over the attended tokens of one query row */
+static void row_logits(const mo_geom *g, const uint16_t *q, const uint16_t *k, int64_t l,
+                       const int32_t *att, int na, double *x) {
+  int b = g_b(g), d = g->d;
+  double sc = g_scale(g);
+  for (int a = 0; a < na; ++a)
+    for (int e = 0; e < b; ++e) {
+      int64_t t = block_token(g, att[a], e);
+      double s = 0.0;
+      for (int c = 0; c < d; ++c) s += bf16_widen(q[l * d + c]) * bf16_widen(k[t * d + c]);
+      x[(size_t)a * b + e] = sc * s;
+    }
+}
+
+/*
+ * Softmax weights of one query row (row e_row of block i) over its attended tokens.
+ * tokens/w must hold (|L_i|+topk)*b entries; returns the count.
+ */
+int mo_weights_row(const mo_geom *g, const uint16_t *q, const uint16_t *k, const int32_t *idx,
+                   int32_t i, int32_t e_row, int64_t *tokens, double *w) {
+  if (!g_ok(g)) return -1;
+  int b = g_b(g);
+  int32_t *att = (int32_t *)malloc(sizeof(int32_t) * (MO_MAX_LOCAL + (size_t)g->topk));
+  int na = attended(g, idx, i, att), n = na * b;
+  row_logits(g, q, k, block_token(g, i, e_row), att, na, w);
+  double M = -INFINITY, Z = 0.0;
+  for (int t = 0; t < n; ++t) M = w[t] > M ? w[t] : M;
+  for (int t = 0; t < n; ++t) Z += exp(w[t] - M);
+  for (int t = 0; t < n; ++t) w[t] = exp(w[t] - M) / Z;
+  for (int a = 0; a < na; ++a)
+    for (int e = 0; e < b; ++e) tokens[(size_t)a * b + e] = block_token(g, att[a], e);
+  free(att);
+  return n;
+}
+
+/*
+ * Forward for a list of query blocks of one unit (blocks == NULL: all m, in order).
+ * O is [n_blocks, b, d], LSE is [n_blocks, b], rows in row-major order inside the block.
+ */
+int mo_fwd_unit(const mo_geom *g, const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                const int32_t *idx, int32_t n_blocks, const int32_t *blocks, double *O, double *LSE) {
+  if (!g_ok(g)) return -1;
+  int b = g_b(g), d = g->d;
+  int max_att = MO_MAX_LOCAL + g->topk;
+#pragma omp parallel
+  {
+    int32_t *att = (int32_t *)malloc(sizeof(int32_t) * (size_t)max_att);
+    double *x = (double *)malloc(sizeof(double) * (size_t)max_att * b);
+#pragma omp for schedule(dynamic, 1)
+    for (int n = 0; n < n_blocks; ++n) {
+      int i = blocks ? blocks[n] : n;
+      int na = attended(g, idx, i, att), nt = na * b;
+      for (int e = 0; e < b; ++e) {
+        int64_t l = block_token(g, i, e);
+        row_logits(g, q, k, l, att, na, x);
+        double M = -INFINITY, Z = 0.0;
+        for (int t = 0; t < nt; ++t) M = x[t] > M ? x[t] : M;
+        for (int t = 0; t < nt; ++t) Z += exp(x[t] - M);
+        double *o = O + ((size_t)n * b + e) * d;
+        for (int c = 0; c < d; ++c) o[c] = 0.0;
+        for (int a = 0; a < na; ++a)
+          for (int e2 = 0; e2 < b; ++e2) {
+            double w = exp(x[(size_t)a * b + e2] - M) / Z;
+            int64_t t = block_token(g, att[a], e2);
+            for (int c = 0; c < d; ++c) o[c] += w * bf16_widen(v[t * d + c]);
+          }
+        LSE[(size_t)n * b + e] = M + log(Z);
+      }
+    }
+    free(att);
+    free(x);
+  }
+  return 0;
+}
+
+/*
+ * Backward for one whole unit, selection held constant.  dQ, dK, dV are [N,d] in
+ * token order.  O_out [N,d] and LSE_out [N] (optional) receive the forward results.
+ */
+int mo_bwd_unit(const mo_geom *g, const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                const uint16_t *d_o, const int32_t *idx, double *dQ, double *dK, double *dV,
+                double *O_out, double *LSE_out) {
+  if (!g_ok(g)) return -1;
+  int m = g_m(g), b = g_b(g), d = g->d;
+  int64_t N = (int64_t)g->nlat * g->nlon;
+  int max_att = MO_MAX_LOCAL + g->topk;
+  double sc = g_scale(g);
+  double *Ob = (double *)malloc(sizeof(double) * (size_t)m * b * d);
+  double *Lb = (double *)malloc(sizeof(double) * (size_t)m * b);
+  double *LSE = (double *)malloc(sizeof(double) * (size_t)N);
+  double *D = (double *)malloc(sizeof(double) * (size_t)N);
+  if (!Ob || !Lb || !LSE || !D) { free(Ob); free(Lb); free(LSE); free(D); return -2; }
+  mo_fwd_unit(g, q, k, v, idx, m, NULL, Ob, Lb);
+  /* D_l = dO_l . O_l */
+#pragma omp parallel for schedule(static)
+  for (int i = 0; i < m; ++i)
+    for (int e = 0; e < b; ++e) {
+      int64_t l = block_token(g, i, e);
+      double acc = 0.0;
+      for (int c = 0; c < d; ++c) {
+        double o = Ob[((size_t)i * b + e) * d + c];
+        acc += bf16_widen(d_o[l * d + c]) * o;
+        if (O_out) O_out[l * d + c] = o;
+      }
+      D[l] = acc;
+      LSE[l] = Lb[(size_t)i * b + e];
+      if (LSE_out) LSE_out[l] = LSE[l];
+    }
+  /* dQ: every query row over its attended tokens */
+#pragma omp parallel
+  {
+    int32_t *att = (int32_t *)malloc(sizeof(int32_t) * (size_t)max_att);
+    double *x = (double *)malloc(sizeof(double) * (size_t)max_att * b);
+#pragma omp for schedule(dynamic, 1)
+    for (int i = 0; i < m; ++i) {
+      int na = attended(g, idx, i, att);
+      for (int e = 0; e < b; ++e) {
+        int64_t l = block_token(g, i, e);
+        row_logits(g, q, k, l, att, na, x);
+        double *dq = dQ + l * d;
+        for (int c = 0; c < d; ++c) dq[c] = 0.0;
+        for (int a = 0; a < na; ++a)
+          for (int e2 = 0; e2 < b; ++e2) {
+            int64_t t = block_token(g, att[a], e2);
+            double w = exp(x[(size_t)a * b + e2] - LSE[l]);
+            double dP = 0.0;
+            for (int c = 0; c < d; ++c) dP += bf16_widen(d_o[l * d + c]) * bf16_widen(v[t * d + c]);
+            double dS = w * (dP - D[l]);
+            for (int c = 0; c < d; ++c) dq[c] += sc * dS * bf16_widen(k[t * d + c]);
+          }
+      }
+    }
+    free(att);
+    free(x);
+  }
+  /* dK, dV: every key/value block over the query blocks connected to it */
+#pragma omp parallel
+  {
+    int32_t *att = (int32_t *)malloc(sizeof(int32_t) * (size_t)max_att);
+#pragma omp for schedule(dynamic, 1)
+    for (int j = 0; j < m; ++j) {
+      for (int e2 = 0; e2 < b; ++e2) {
+        int64_t t = block_token(g, j, e2);
+        for (int c = 0; c < d; ++c) { dK[t * d + c] = 0.0; dV[t * d + c] = 0.0; }
+      }
+      for (int i = 0; i < m; ++i) {
+        int na = attended(g, idx, i, att), connected = 0;
+        for (int a = 0; a < na; ++a) connected |= (att[a] == j);
+        if (!connected) continue;
+        for (int e = 0; e < b; ++e) {
+          int64_t l = block_token(g, i, e);
+          for (int e2 = 0; e2 < b; ++e2) {
+            int64_t t = block_token(g, j, e2);
+            double s = 0.0, dP = 0.0;
+            for (int c = 0; c < d; ++c) {
+              s += bf16_widen(q[l * d + c]) * bf16_widen(k[t * d + c]);
+              dP += bf16_widen(d_o[l * d + c]) * bf16_widen(v[t * d + c]);
+            }
+            double w = exp(sc * s - LSE[l]);
+            double dS = w * (dP - D[l]);
+            for (int c = 0; c < d; ++c) {
+              dV[t * d + c] += w * bf16_widen(d_o[l * d + c]);
+              dK[t * d + c] += sc * dS * bf16_widen(q[l * d + c]);
+            }
+          }
+        }
+      }
+    }
+    free(att);
+  }
+  free(Ob); free(Lb); free(LSE); free(D);
+  return 0;
+}

@@ -1,0 +1,125 @@
+/*
+ * mosaic_bsa.h -- C ABI of the MOSAIC mesh-aligned block-sparse attention hot path
+ * for NVIDIA B200 (sm_100a).
+ *
+ * Method (paper: section "Block-Sparse Attention", paragraphs "Compression",
+ * "Selection", "Local Attention"; appendix "Block-sparse attention implementation",
+ * paragraph "Kernel Design"):  the N = nlat*nlon tokens of a lat-lon grid are tiled
+ * into bh x bw blocks.  Every query block attends ONE key/value set shared by all of
+ * its tokens: its local mesh neighbourhood (own block and the blocks within
+ * rlat/rlon block rows/columns; longitude periodic, latitude clamped, every block
+ * counted once) plus the top-k non-local blocks ranked by the dot product of the
+ * mean-pooled query block with the mean-pooled key block.  Attention over that union
+ * is one softmax (scale 1/sqrt(d) unless given).
+ *
+ * Common rules for every entry point
+ *   - All tensor pointers are DEVICE pointers on the current CUDA device.  Q, K, V, O,
+ *     dO are contiguous [B, H, N, d] bf16 with token t = lat*nlon + lon, base address
+ *     16-byte aligned.  "unit" u = b*H + h; units are independent.
+ *   - block_idx is contiguous [B, H, m, topk] int32, m = (nlat/bh)*(nlon/bw), block id
+ *     j = by*(nlon/bw) + bx.  Row i holds the selected non-local block ids of query
+ *     block i, best first, padded with -1.  The local set is implicit.
+ *   - The caller owns every buffer, including the workspace `ws` (device memory, 256-byte
+ *     aligned, at least mosaic_bsa_workspace_bytes() long).  The library allocates no
+ *     device memory and keeps no state beyond a host-side cache of TMA descriptors.
+ *   - Calls enqueue work on `cuda_stream` (a cudaStream_t, NULL = default stream) and
+ *     return without synchronising.  Two calls that share a workspace must be ordered
+ *     on one stream.
+ *   - Return value: MOSAIC_OK or a negative MOSAIC_E_* code; nothing aborts, traps or
+ *     throws across the boundary.  Faults detected on the device (a bounded wait that
+ *     ran out, a block id out of range) do not fault the GPU: the kernel records a code
+ *     in the first word of the workspace, skips the offending work and returns; read it
+ *     with mosaic_bsa_last_status().
+ *   - Supported in this version: d = 64; bw = 8 or 16 with bh a multiple of 64/bw
+ *     (8x8 and 16x16 are the tested shapes); rlat, rlon in 0..2; (local blocks + topk)
+ *     <= 64; topk <= 32; any B, H and any grid with nlat % bh == 0, nlon % bw == 0
+ *     (grids with fewer than 2*rlon+1 block columns de-duplicate the neighbourhood).
+ */
+#ifndef MOSAIC_BSA_H_
+#define MOSAIC_BSA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mosaic_bsa_params {
+  int32_t B, H;       /* batch (ensemble members) and heads; Q, K, V share H          */
+  int32_t nlat, nlon; /* grid; N = nlat*nlon                                           */
+  int32_t d;          /* head dimension (64)                                           */
+  int32_t bh, bw;     /* block shape in grid points                                    */
+  int32_t rlat, rlon; /* local neighbourhood radius in blocks (1,1 = 3x3)              */
+  int32_t topk;       /* selected non-local blocks per query block, >= 0               */
+  float scale;        /* softmax scale; <= 0 means 1/sqrt(d)                           */
+  uint32_t flags;     /* reserved, must be 0                                           */
+} mosaic_bsa_params;
+
+enum { MOSAIC_OP_SELECT = 0, MOSAIC_OP_FWD = 1, MOSAIC_OP_BWD = 2 };
+
+enum {
+  MOSAIC_OK = 0,
+  MOSAIC_E_INVALID_ARG = -1,        /* null pointer, non-divisible grid, negative size    */
+  MOSAIC_E_UNSUPPORTED = -2,        /* d, block shape, radius or device not supported     */
+  MOSAIC_E_WORKSPACE_TOO_SMALL = -3,
+  MOSAIC_E_MISALIGNED = -4,         /* a tensor base or the workspace is not aligned      */
+  MOSAIC_E_CUDA = -5,               /* a CUDA runtime/driver call failed (launch, query)  */
+  /* device-side status codes (mosaic_bsa_last_status) */
+  MOSAIC_E_DEVICE_TIMEOUT = -16,    /* a bounded wait on an on-chip barrier ran out       */
+  MOSAIC_E_DEVICE_BAD_INDEX = -17   /* block_idx held an id outside [-1, m)               */
+};
+
+/* Bytes of device workspace the given op needs for these params (0 on invalid params).
+ * The first 256 bytes of any workspace are the status block. */
+size_t mosaic_bsa_workspace_bytes(const mosaic_bsa_params *p, int op);
+
+/*
+ * Selection ("Compression" + "Selection" paragraphs: pooled block representations,
+ * block-level scores, top-n per query block).
+ *   q, k       in   [B,H,N,d] bf16
+ *   block_idx  out  [B,H,m,topk] int32
+ * Arithmetic is fixed so that the result is unique: block sums accumulate in fp64 in
+ * row-major order inside the block and round once to fp32; a score is the fp64 sum, in
+ * channel order, of the exact products of those fp32 values; order = (score descending,
+ * block id ascending); +0 and -0 tie; a NaN score ranks last.
+ */
+int mosaic_bsa_select(const mosaic_bsa_params *p, const void *q, const void *k, int32_t *block_idx,
+                      void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Forward (fine-grained attention equation of the "Selection" paragraph over the union
+ * of local and selected blocks; streaming evaluation per the "Kernel Design" paragraph).
+ *   q, k, v    in   [B,H,N,d] bf16
+ *   block_idx  in   [B,H,m,topk] int32 (from mosaic_bsa_select or the caller: ids in
+ *                   [0,m) or -1, no repeats in a row, none inside the row's local set)
+ *   o          out  [B,H,N,d] bf16
+ *   lse        out  [B,H,N] fp32, natural-log sum-exp of the scaled logits of each row
+ */
+int mosaic_bsa_fwd(const mosaic_bsa_params *p, const void *q, const void *k, const void *v,
+                   const int32_t *block_idx, void *o, float *lse, void *ws, size_t ws_bytes,
+                   void *cuda_stream);
+
+/*
+ * Backward (gradient of the forward with the selection held constant; dK/dV visit only
+ * the query blocks connected to a key/value block, "Kernel Design" paragraph).
+ *   q, k, v, o, d_o  in   [B,H,N,d] bf16;  lse in [B,H,N] fp32 (from mosaic_bsa_fwd)
+ *   dq, dk, dv       out  [B,H,N,d] bf16
+ * Results are deterministic (fixed summation order, no floating-point atomics).
+ */
+int mosaic_bsa_bwd(const mosaic_bsa_params *p, const void *q, const void *k, const void *v,
+                   const void *o, const float *lse, const void *d_o, const int32_t *block_idx,
+                   void *dq, void *dk, void *dv, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/* Synchronises `cuda_stream`, then returns the device status word of `ws`
+ * (MOSAIC_OK, MOSAIC_E_DEVICE_*) or MOSAIC_E_CUDA if the stream reports an error.
+ * Every op resets the word when it starts. */
+int mosaic_bsa_last_status(const void *ws, void *cuda_stream);
+
+/* Static, NUL-terminated description of a return code. */
+const char *mosaic_bsa_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOSAIC_BSA_H_ */

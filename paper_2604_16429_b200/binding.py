@@ -1,0 +1,191 @@
+"""Thin ctypes binding of the C ABI in ``include/mosaic_bsa.h``.
+
+Argument marshalling only: every step of the path runs in the CUDA library.  torch is
+used for device memory and streams.  There is no CPU fallback: if the library is missing
+or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmosaic_bsa.so")
+_lib = None
+
+OP_SELECT, OP_FWD, OP_BWD = 0, 1, 2
+EXPORTS = ("mosaic_bsa_workspace_bytes", "mosaic_bsa_select", "mosaic_bsa_fwd", "mosaic_bsa_bwd",
+           "mosaic_bsa_last_status", "mosaic_bsa_strerror")
+
+
+class MosaicError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {strerror(code)} ({code})")
+
+
+class _Params(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("nlat", ctypes.c_int32), ("nlon", ctypes.c_int32),
+                ("d", ctypes.c_int32), ("bh", ctypes.c_int32), ("bw", ctypes.c_int32),
+                ("rlat", ctypes.c_int32), ("rlon", ctypes.c_int32), ("topk", ctypes.c_int32),
+                ("scale", ctypes.c_float), ("flags", ctypes.c_uint32)]
+
+
+@dataclass(frozen=True)
+class Params:
+    B: int
+    H: int
+    nlat: int
+    nlon: int
+    d: int = 64
+    bh: int = 8
+    bw: int = 8
+    rlat: int = 1
+    rlon: int = 1
+    topk: int = 8
+    scale: float = 0.0
+    flags: int = 0
+
+    @property
+    def N(self): return self.nlat * self.nlon
+    @property
+    def m(self): return (self.nlat // self.bh) * (self.nlon // self.bw)
+    @property
+    def U(self): return self.B * self.H
+
+    def c(self):
+        return _Params(self.B, self.H, self.nlat, self.nlon, self.d, self.bh, self.bw, self.rlat, self.rlon,
+                       self.topk, self.scale, self.flags)
+
+    @staticmethod
+    def from_workload(w, **over):
+        kw = dict(B=w.B, H=w.H, nlat=w.nlat, nlon=w.nlon, d=w.d, bh=w.bh, bw=w.bw, rlat=w.rlat, rlon=w.rlon,
+                  topk=w.topk)
+        kw.update(over)
+        return Params(**kw)
+
+
+def lib():
+    """Load the CUDA library; fails loudly if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2604_16429_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32p, fp = ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p
+        pp = ctypes.POINTER(_Params)
+        L.mosaic_bsa_workspace_bytes.restype = ctypes.c_size_t
+        L.mosaic_bsa_workspace_bytes.argtypes = [pp, ctypes.c_int]
+        L.mosaic_bsa_select.restype = ctypes.c_int
+        L.mosaic_bsa_select.argtypes = [pp, vp, vp, i32p, vp, ctypes.c_size_t, vp]
+        L.mosaic_bsa_fwd.restype = ctypes.c_int
+        L.mosaic_bsa_fwd.argtypes = [pp, vp, vp, vp, i32p, vp, fp, vp, ctypes.c_size_t, vp]
+        L.mosaic_bsa_bwd.restype = ctypes.c_int
+        L.mosaic_bsa_bwd.argtypes = [pp, vp, vp, vp, vp, fp, vp, i32p, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.mosaic_bsa_last_status.restype = ctypes.c_int
+        L.mosaic_bsa_last_status.argtypes = [vp, vp]
+        L.mosaic_bsa_strerror.restype = ctypes.c_char_p
+        L.mosaic_bsa_strerror.argtypes = [ctypes.c_int]
+        _lib = L
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().mosaic_bsa_strerror(int(code)).decode()
+
+
+def workspace_bytes(p: Params, op: int) -> int:
+    pc = p.c()
+    return int(lib().mosaic_bsa_workspace_bytes(ctypes.byref(pc), op))
+
+
+def _stream(stream) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return int(s.cuda_stream)
+
+
+def _ptr(t) -> int:
+    return 0 if t is None else int(t.data_ptr())
+
+
+def _chk_qkv(p: Params, *ts):
+    for t in ts:
+        if t.dtype != torch.bfloat16 or not t.is_cuda or not t.is_contiguous() or tuple(t.shape) != (p.B, p.H, p.N, p.d):
+            raise ValueError(f"expected contiguous cuda bf16 [{p.B},{p.H},{p.N},{p.d}], got {t.dtype} {tuple(t.shape)}")
+
+
+def alloc_workspace(p: Params, op: int, device="cuda") -> torch.Tensor:
+    n = workspace_bytes(p, op)
+    if n == 0:
+        raise MosaicError(-1, "mosaic_bsa_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def mosaic_bsa_select(p: Params, q, k, block_idx=None, ws=None, stream=None):
+    _chk_qkv(p, q, k)
+    if block_idx is None:
+        block_idx = torch.empty((p.B, p.H, p.m, p.topk), dtype=torch.int32, device=q.device)
+    if ws is None:
+        ws = alloc_workspace(p, OP_SELECT, q.device)
+    pc = p.c()
+    rc = lib().mosaic_bsa_select(ctypes.byref(pc), _ptr(q), _ptr(k), _ptr(block_idx), _ptr(ws), ws.numel(),
+                                 _stream(stream))
+    if rc:
+        raise MosaicError(rc, "mosaic_bsa_select")
+    return block_idx
+
+
+def mosaic_bsa_fwd(p: Params, q, k, v, block_idx, o=None, lse=None, ws=None, stream=None):
+    _chk_qkv(p, q, k, v)
+    if o is None:
+        o = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((p.B, p.H, p.N), dtype=torch.float32, device=q.device)
+    if ws is None:
+        ws = alloc_workspace(p, OP_FWD, q.device)
+    pc = p.c()
+    rc = lib().mosaic_bsa_fwd(ctypes.byref(pc), _ptr(q), _ptr(k), _ptr(v), _ptr(block_idx), _ptr(o), _ptr(lse),
+                              _ptr(ws), ws.numel(), _stream(stream))
+    if rc:
+        raise MosaicError(rc, "mosaic_bsa_fwd")
+    return o, lse
+
+
+def mosaic_bsa_bwd(p: Params, q, k, v, o, lse, d_o, block_idx, dq=None, dk=None, dv=None, ws=None, stream=None):
+    _chk_qkv(p, q, k, v, o, d_o)
+    dq = torch.empty_like(q) if dq is None else dq
+    dk = torch.empty_like(q) if dk is None else dk
+    dv = torch.empty_like(q) if dv is None else dv
+    if ws is None:
+        ws = alloc_workspace(p, OP_BWD, q.device)
+    pc = p.c()
+    rc = lib().mosaic_bsa_bwd(ctypes.byref(pc), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(d_o),
+                              _ptr(block_idx), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(ws), ws.numel(), _stream(stream))
+    if rc:
+        raise MosaicError(rc, "mosaic_bsa_bwd")
+    return dq, dk, dv
+
+
+def mosaic_bsa_last_status(ws, stream=None) -> int:
+    return int(lib().mosaic_bsa_last_status(_ptr(ws), _stream(stream)))
+
+
+def check_status(ws, where: str, stream=None):
+    st = mosaic_bsa_last_status(ws, stream)
+    if st:
+        raise MosaicError(st, where + " (device status)")
+
+
+def from_bits(bits, device="cuda") -> torch.Tensor:
+    """uint16 bf16 bit patterns (numpy) -> bf16 tensor on `device`, bit for bit."""
+    import numpy as np
+    t = torch.from_numpy(np.ascontiguousarray(bits).view(np.int16))
+    return t.to(device).view(torch.bfloat16)
+
+
+def default_scale(d: int) -> float:
+    return 1.0 / math.sqrt(d)

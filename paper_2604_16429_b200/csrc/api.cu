@@ -1,0 +1,171 @@
+// C ABI of the library: argument validation, workspace carving, kernel launches.
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include "common.cuh"
+
+namespace mosaic {
+
+size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+int validate(const mosaic_bsa_params* p, Geo* g) {
+  if (!p) return MOSAIC_E_INVALID_ARG;
+  if (p->B <= 0 || p->H <= 0 || p->nlat <= 0 || p->nlon <= 0 || p->bh <= 0 || p->bw <= 0 || p->topk < 0 ||
+      p->rlat < 0 || p->rlon < 0 || p->flags != 0)
+    return MOSAIC_E_INVALID_ARG;
+  if (p->nlat % p->bh || p->nlon % p->bw) return MOSAIC_E_INVALID_ARG;
+  if (!(p->scale == p->scale) || isinf(p->scale)) return MOSAIC_E_INVALID_ARG;
+  if (p->d != kD) return MOSAIC_E_UNSUPPORTED;
+  if (!(p->bw == 8 || p->bw == 16)) return MOSAIC_E_UNSUPPORTED;
+  const int crows = kChunk / p->bw;
+  if (p->bh % crows) return MOSAIC_E_UNSUPPORTED;
+  const int cpb = p->bh * p->bw / kChunk;
+  if (!(cpb == 1 || cpb % 2 == 0)) return MOSAIC_E_UNSUPPORTED;
+  if (p->rlat > 2 || p->rlon > 2 || p->topk > kMaxTopk) return MOSAIC_E_UNSUPPORTED;
+  if ((2 * p->rlat + 1) * (2 * p->rlon + 1) + p->topk > kMaxList) return MOSAIC_E_UNSUPPORTED;
+  const long long U = (long long)p->B * p->H, N = (long long)p->nlat * p->nlon;
+  const long long m = (long long)(p->nlat / p->bh) * (p->nlon / p->bw);
+  if (U > (1 << 24) || m > (1 << 24) || U * m * cpb > 0x7fffffffll || U * N > (1ll << 40)) return MOSAIC_E_UNSUPPORTED;
+  g->U = (int)U;
+  g->nlat = p->nlat; g->nlon = p->nlon; g->bh = p->bh; g->bw = p->bw;
+  g->nbh = p->nlat / p->bh; g->nbw = p->nlon / p->bw; g->m = (int)m;
+  g->b = p->bh * p->bw; g->cpb = cpb; g->crows = crows;
+  g->rlat = p->rlat; g->rlon = p->rlon; g->topk = p->topk;
+  g->scale = p->scale > 0.f ? p->scale : 1.0f / sqrtf((float)p->d);
+  g->scale_log2 = g->scale * 1.4426950408889634f;
+  g->N = N;
+  return MOSAIC_OK;
+}
+
+namespace {
+
+struct BwdWs { size_t D, off, cur, q, total; };
+BwdWs bwd_layout(const Geo& g) {
+  BwdWs w;
+  size_t at = kStatusBytes;
+  w.D = at; at = align256(at + sizeof(float) * (size_t)g.U * g.N);
+  w.off = at; at = align256(at + sizeof(int32_t) * (size_t)g.U * (g.m + 1));
+  w.cur = at;  // reserved
+  w.q = at; at = align256(at + sizeof(int32_t) * (size_t)g.U * g.m * (g.topk > 0 ? g.topk : 1));
+  w.total = at;
+  return w;
+}
+size_t select_total(const Geo& g) { return kStatusBytes + 2 * align256(sizeof(float) * (size_t)g.U * g.m * kD); }
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+int device_ok() {
+  static int cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return MOSAIC_E_CUDA;
+  if (dev < 64 && cached[dev]) return cached[dev] > 0 ? MOSAIC_OK : MOSAIC_E_UNSUPPORTED;
+  int major = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return MOSAIC_E_CUDA;
+  if (dev < 64) cached[dev] = major == 10 ? 1 : -1;
+  return major == 10 ? MOSAIC_OK : MOSAIC_E_UNSUPPORTED;
+}
+
+int begin(const mosaic_bsa_params* p, void* ws, size_t ws_bytes, size_t need, void* stream, HostCtx* c) {
+  int rc = validate(p, &c->g);
+  if (rc) return rc;
+  if (!ws) return MOSAIC_E_INVALID_ARG;
+  if (!aligned(ws, 256)) return MOSAIC_E_MISALIGNED;
+  if (ws_bytes < need) return MOSAIC_E_WORKSPACE_TOO_SMALL;
+  if ((rc = device_ok())) return rc;
+  c->stream = (cudaStream_t)stream;
+  c->status = (int*)ws;
+  if (cudaMemsetAsync(ws, 0, kStatusBytes, c->stream) != cudaSuccess) return MOSAIC_E_CUDA;
+  return MOSAIC_OK;
+}
+
+}  // namespace
+}  // namespace mosaic
+
+using namespace mosaic;
+
+extern "C" {
+
+size_t mosaic_bsa_workspace_bytes(const mosaic_bsa_params* p, int op) {
+  Geo g;
+  if (validate(p, &g)) return 0;
+  switch (op) {
+    case MOSAIC_OP_SELECT: return select_total(g);
+    case MOSAIC_OP_FWD: return kStatusBytes;
+    case MOSAIC_OP_BWD: return bwd_layout(g).total;
+    default: return 0;
+  }
+}
+
+int mosaic_bsa_select(const mosaic_bsa_params* p, const void* q, const void* k, int32_t* block_idx, void* ws,
+                      size_t ws_bytes, void* cuda_stream) {
+  HostCtx c;
+  Geo g;
+  int rc = validate(p, &g);
+  if (rc) return rc;
+  if (!q || !k || (!block_idx && g.topk > 0)) return MOSAIC_E_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(k, 16) || !aligned(block_idx, 4)) return MOSAIC_E_MISALIGNED;
+  if ((rc = begin(p, ws, ws_bytes, select_total(g), cuda_stream, &c))) return rc;
+  float* pq = (float*)((char*)ws + kStatusBytes);
+  float* pk = (float*)((char*)pq + align256(sizeof(float) * (size_t)g.U * g.m * kD));
+  return launch_select(c, q, k, block_idx, pq, pk);
+}
+
+int mosaic_bsa_fwd(const mosaic_bsa_params* p, const void* q, const void* k, const void* v,
+                   const int32_t* block_idx, void* o, float* lse, void* ws, size_t ws_bytes, void* cuda_stream) {
+  HostCtx c;
+  Geo g;
+  int rc = validate(p, &g);
+  if (rc) return rc;
+  if (!q || !k || !v || !o || !lse || (!block_idx && g.topk > 0)) return MOSAIC_E_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(o, 16) || !aligned(lse, 4) ||
+      !aligned(block_idx, 4))
+    return MOSAIC_E_MISALIGNED;
+  if ((rc = begin(p, ws, ws_bytes, kStatusBytes, cuda_stream, &c))) return rc;
+  return launch_fwd_tc(c, q, k, v, block_idx, o, lse);
+}
+
+int mosaic_bsa_bwd(const mosaic_bsa_params* p, const void* q, const void* k, const void* v, const void* o,
+                   const float* lse, const void* d_o, const int32_t* block_idx, void* dq, void* dk, void* dv,
+                   void* ws, size_t ws_bytes, void* cuda_stream) {
+  HostCtx c;
+  Geo g;
+  int rc = validate(p, &g);
+  if (rc) return rc;
+  if (!q || !k || !v || !o || !lse || !d_o || !dq || !dk || !dv || (!block_idx && g.topk > 0))
+    return MOSAIC_E_INVALID_ARG;
+  const void* ptrs[] = {q, k, v, o, d_o, dq, dk, dv};
+  for (const void* x : ptrs)
+    if (!aligned(x, 16)) return MOSAIC_E_MISALIGNED;
+  if (!aligned(lse, 4) || !aligned(block_idx, 4)) return MOSAIC_E_MISALIGNED;
+  if ((size_t)g.m * sizeof(int) > 200 * 1024) return MOSAIC_E_UNSUPPORTED;
+  BwdWs w = bwd_layout(g);
+  if ((rc = begin(p, ws, ws_bytes, w.total, cuda_stream, &c))) return rc;
+  char* base = (char*)ws;
+  return launch_bwd(c, q, k, v, o, lse, d_o, block_idx, dq, dk, dv, (float*)(base + w.D),
+                    (int32_t*)(base + w.off), (int32_t*)(base + w.cur), (int32_t*)(base + w.q));
+}
+
+int mosaic_bsa_last_status(const void* ws, void* cuda_stream) {
+  if (!ws) return MOSAIC_E_INVALID_ARG;
+  if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess) return MOSAIC_E_CUDA;
+  int st = 0;
+  if (cudaMemcpy(&st, ws, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return MOSAIC_E_CUDA;
+  return st;
+}
+
+const char* mosaic_bsa_strerror(int code) {
+  switch (code) {
+    case MOSAIC_OK: return "ok";
+    case MOSAIC_E_INVALID_ARG: return "invalid argument";
+    case MOSAIC_E_UNSUPPORTED: return "unsupported shape, option or device";
+    case MOSAIC_E_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case MOSAIC_E_MISALIGNED: return "misaligned pointer";
+    case MOSAIC_E_CUDA: return "CUDA call failed";
+    case MOSAIC_E_DEVICE_TIMEOUT: return "device: bounded wait ran out";
+    case MOSAIC_E_DEVICE_BAD_INDEX: return "device: block id out of range";
+    default: return "unknown code";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,111 @@
+// Shared device/host definitions of the MOSAIC block-sparse attention kernels (sm_100a).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "mosaic_bsa.h"
+
+namespace mosaic {
+
+constexpr int kD = 64;            // head dimension
+constexpr int kChunk = 64;        // tokens per staged key/value chunk (and per mma.sync query tile)
+constexpr int kMaxList = 64;      // most blocks one query block attends (local + top-k)
+constexpr int kMaxTopk = 32;
+constexpr int kStatusBytes = 256; // status block at the start of every workspace
+
+// Geometry of one call, passed by value to the kernels.
+struct Geo {
+  int U;            // B*H independent units
+  int nlat, nlon;   // grid
+  int bh, bw;       // block shape
+  int nbh, nbw, m;  // blocks per column / row / unit
+  int b;            // tokens per block
+  int cpb;          // 64-token chunks per block (b / 64)
+  int crows;        // grid rows per chunk (64 / bw)
+  int rlat, rlon, topk;
+  float scale;      // softmax scale
+  float scale_log2; // scale * log2(e)
+  long long N;      // tokens per unit
+};
+
+// Record the first device-side fault in the workspace status word (never traps).
+__device__ __forceinline__ void set_status(int* status, int code) { atomicCAS(status, 0, code); }
+
+// Local neighbourhood of query block i: rows clamp(by+dy), columns (bx+dx) mod nbw, each
+// block once, in first-occurrence order (dy, then dx ascending).  Returns the count.
+__device__ __forceinline__ int local_set(const Geo& g, int i, int* out) {
+  int by = i / g.nbw, bx = i - by * g.nbw, n = 0;
+  for (int dy = -g.rlat; dy <= g.rlat; ++dy) {
+    int y = min(max(by + dy, 0), g.nbh - 1);
+    for (int dx = -g.rlon; dx <= g.rlon; ++dx) {
+      int x = (bx + dx) % g.nbw;
+      x += x < 0 ? g.nbw : 0;
+      int id = y * g.nbw + x;
+      bool seen = false;
+      for (int a = 0; a < n; ++a) seen |= (out[a] == id);
+      if (!seen) out[n++] = id;
+    }
+  }
+  return n;
+}
+
+__device__ __forceinline__ bool is_local(const Geo& g, int i, int j) {
+  int by = i / g.nbw, bx = i - by * g.nbw;
+  int jy = j / g.nbw, jx = j - jy * g.nbw;
+  // clamping only folds an out-of-range row onto a row already in the window
+  bool row_ok = abs(jy - by) <= g.rlat;
+  int dx = jx - bx;
+  dx += dx < 0 ? g.nbw : 0;                       // (jx - bx) mod nbw in [0, nbw)
+  bool col_ok = dx <= g.rlon || g.nbw - dx <= g.rlon;
+  return row_ok && col_ok;
+}
+
+// Attended list of query block i: local set followed by the valid selected ids.
+// Ids outside [-1, m) are skipped and reported.  `out` holds kMaxList entries.
+__device__ __forceinline__ int attended_list(const Geo& g, const int32_t* __restrict__ idx_row, int i,
+                                             int* out, int* status) {
+  int n = local_set(g, i, out);
+  for (int r = 0; r < g.topk; ++r) {
+    int j = idx_row[r];
+    if (j < 0) {
+      if (j != -1) set_status(status, MOSAIC_E_DEVICE_BAD_INDEX);
+      continue;
+    }
+    if (j >= g.m) { set_status(status, MOSAIC_E_DEVICE_BAD_INDEX); continue; }
+    if (n < kMaxList) out[n++] = j;
+  }
+  return n;
+}
+
+// First token (row-major grid index inside the unit) of row `r` of chunk `c` of block j.
+__device__ __forceinline__ long long chunk_row_token(const Geo& g, int j, int c, int r) {
+  int by = j / g.nbw, bx = j - by * g.nbw;
+  return (long long)(by * g.bh + c * g.crows + r) * g.nlon + bx * g.bw;
+}
+
+// Token of element e (0..63, row-major inside the chunk) of chunk c of block j.
+__device__ __forceinline__ long long chunk_token(const Geo& g, int j, int c, int e) {
+  int r = e / g.bw;
+  return chunk_row_token(g, j, c, r) + (e - r * g.bw);
+}
+
+// ---- host side ---------------------------------------------------------------------------
+struct HostCtx {
+  Geo g;
+  cudaStream_t stream;
+  int* status;  // device pointer to the workspace status word
+};
+
+int validate(const mosaic_bsa_params* p, Geo* g);
+size_t align256(size_t x);
+
+// kernel launchers (one per translation unit)
+int launch_select(const HostCtx& c, const void* q, const void* k, int32_t* block_idx, float* pooled_q,
+                  float* pooled_k);
+int launch_fwd_tc(const HostCtx& c, const void* q, const void* k, const void* v, const int32_t* block_idx,
+                  void* o, float* lse);
+int launch_bwd(const HostCtx& c, const void* q, const void* k, const void* v, const void* o, const float* lse,
+               const void* d_o, const int32_t* block_idx, void* dq, void* dk, void* dv, float* Dbuf,
+               int32_t* csr_off, int32_t* csr_cur, int32_t* csr_q);
+
+}  // namespace mosaic

@@ -1,0 +1,172 @@
+"""GPU parity: the CUDA path through the C ABI against the fp64 oracle, element by element,
+on sizes the oracle finishes in seconds (several tiles, ragged tails, degenerate cases)."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2604_16429_b200 import binding as mb
+from paper_2604_16429_b200 import synth
+from tests import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+
+SELECT_CASES = [
+    synth.WORKLOADS["c1_tiny"],
+    synth.small_case(136, 160, 8, 8, 8, B=1, H=2, kind="smooth", seed=21),     # m = 340: two key chunks, ragged rows
+    synth.small_case(64, 128, 16, 16, 16, B=2, H=1, kind="smooth", seed=22),   # 16x16 blocks, m = 32
+    synth.small_case(24, 40, 8, 8, 32, B=1, H=1, seed=23),                      # top-k beyond the candidates -> -1 padding
+    synth.small_case(40, 48, 8, 8, 5, B=1, H=3, seed=24, rlat=2, rlon=1),
+    synth.small_case(32, 16, 8, 8, 2, B=1, H=1, seed=25),                       # 2 block columns: neighbourhood de-duplicates
+    synth.small_case(48, 64, 8, 8, 0, B=1, H=1, seed=26, rlat=0, rlon=0),       # nothing selected
+]
+
+
+@pytest.mark.parametrize("w", SELECT_CASES, ids=lambda w: w.name)
+def test_select_bit_exact(w):
+    x = synth.make_inputs(w)
+    want = G.oracle_select_all(w, x)
+    got = G.gpu_select(w, G.device_inputs(x)).cpu().numpy()
+    assert got.shape == want.shape
+    assert np.array_equal(got, want), f"{(got != want).sum()} of {want.size} ids differ"
+
+
+def test_select_ties_go_to_lower_block_id():
+    w = synth.small_case(32, 64, 8, 8, 4, seed=27)
+    x = synth.make_inputs(w)
+    k = x["k"].reshape(1, 1, 32, 64, 64).copy()
+    k[:, :, :, 40:48] = k[:, :, :, 8:16]            # block column 5 repeats block column 1 exactly
+    k[:, :, :, 56:64] = k[:, :, :, 8:16]
+    x["k"] = np.ascontiguousarray(k.reshape(1, 1, -1, 64))
+    want = G.oracle_select_all(w, x)
+    got = G.gpu_select(w, G.device_inputs(x)).cpu().numpy()
+    assert np.array_equal(got, want)
+    # the tie is real: some row lists two duplicated blocks in ascending id order
+    rows = [r for r in want[0, 0] if any((a % 8, b % 8) in ((1, 5), (1, 7), (5, 7)) and a // 8 == b // 8
+                                         for a, b in zip(r[:-1], r[1:]))]
+    assert rows
+
+
+FWD_CASES = [
+    (synth.WORKLOADS["c1_tiny"], 0.0),
+    (synth.small_case(24, 40, 8, 8, 3, B=1, H=2, seed=31), 0.0),                # m = 15: last tile holds one block
+    (synth.small_case(32, 64, 16, 16, 3, B=1, H=2, kind="smooth", seed=32), 0.0),  # 16x16 blocks: 4 chunks per block
+    (synth.small_case(48, 64, 8, 8, 0, B=1, H=1, seed=33, rlat=0, rlon=0), 0.0),   # block-diagonal
+    (synth.small_case(40, 48, 8, 8, 6, B=2, H=1, kind="smooth", seed=34, rlat=2, rlon=2), 0.3),
+    (synth.small_case(16, 16, 8, 8, 4, B=1, H=1, seed=35), 0.0),                # 2x2 blocks: everything local, all -1
+]
+
+
+@pytest.mark.parametrize("w,scale", FWD_CASES, ids=lambda a: a.name if hasattr(a, "name") else str(a))
+def test_forward_matches_oracle(w, scale):
+    x = synth.make_inputs(w)
+    dx = G.device_inputs(x)
+    idx = G.gpu_select(w, dx)
+    o, lse = G.gpu_fwd(w, dx, idx, scale)
+    idx_h = idx.cpu().numpy()
+    for b in range(w.B):
+        for h in range(w.H):
+            G.compare_fwd_unit(w, x, b, h, idx_h[b, h], o, lse, scale=scale)
+
+
+def test_forward_large_logits_rescale_path():
+    """Inputs scaled up so the running maximum jumps by far more than the lazy-rescale threshold."""
+    w = synth.small_case(32, 64, 8, 8, 4, B=1, H=2, seed=36)
+    x = synth.make_inputs(w)
+    for n in ("q", "k"):
+        x[n] = synth.to_bf16_bits(synth.bf16_bits_to_f32(x[n]) * np.float32(3.0))
+    dx = G.device_inputs(x)
+    idx = G.gpu_select(w, dx)
+    o, lse = G.gpu_fwd(w, dx, idx)
+    for h in range(w.H):
+        G.compare_fwd_unit(w, x, 0, h, idx.cpu().numpy()[0, h], o, lse)
+
+
+def test_forward_accepts_caller_block_idx_in_any_order():
+    w = synth.small_case(32, 64, 8, 8, 4, B=1, H=1, seed=37)
+    x = synth.make_inputs(w)
+    dx = G.device_inputs(x)
+    idx = G.gpu_select(w, dx)
+    o1, l1 = G.gpu_fwd(w, dx, idx)
+    rev = torch.flip(idx, dims=[-1]).contiguous()
+    rev[..., 0, 0] = -1                                   # drop one id: still valid, different result for row 0
+    o2, l2 = G.gpu_fwd(w, dx, rev)
+    G.compare_fwd_unit(w, x, 0, 0, rev.cpu().numpy()[0, 0], o2, l2)
+    same = oracle.block_tokens(G.geom_of(w), 5)
+    assert torch.allclose(o1[0, 0, same].float(), o2[0, 0, same].float(), atol=2e-2)
+
+
+def test_forward_is_deterministic_and_writes_everything():
+    w = synth.WORKLOADS["c1_tiny"]
+    dx = G.device_inputs(synth.make_inputs(w))
+    idx = G.gpu_select(w, dx)
+    o1, l1 = G.gpu_fwd(w, dx, idx)
+    o2, l2 = G.gpu_fwd(w, dx, idx)
+    assert torch.equal(o1.view(torch.int16), o2.view(torch.int16)) and torch.equal(l1, l2)
+
+
+def test_bad_block_id_is_reported_not_dereferenced():
+    w = synth.small_case(32, 64, 8, 8, 4, B=1, H=1, seed=38)
+    dx = G.device_inputs(synth.make_inputs(w))
+    idx = G.gpu_select(w, dx)
+    idx[0, 0, 3, 1] = w.m + 5
+    p = mb.Params.from_workload(w)
+    ws = mb.alloc_workspace(p, mb.OP_FWD)
+    o, lse = mb.mosaic_bsa_fwd(p, dx["q"], dx["k"], dx["v"], idx, ws=ws)
+    assert mb.mosaic_bsa_last_status(ws) == -17
+    assert torch.isfinite(o.float()).all()               # the bad id was skipped, nothing faulted
+
+
+BWD_CASES = [
+    synth.small_case(32, 64, 8, 8, 4, B=1, H=2, seed=41, backward=True),
+    synth.small_case(24, 40, 8, 8, 3, B=1, H=1, kind="smooth", seed=42, backward=True),
+    synth.small_case(32, 64, 16, 16, 2, B=1, H=1, kind="smooth", seed=43, backward=True),
+    synth.small_case(48, 64, 8, 8, 0, B=1, H=1, seed=44, rlat=0, rlon=0, backward=True),
+]
+
+
+@pytest.mark.parametrize("w", BWD_CASES, ids=lambda w: w.name)
+def test_backward_matches_oracle(w):
+    x = synth.make_inputs(w)
+    dx = G.device_inputs(x)
+    idx = G.gpu_select(w, dx)
+    o, lse = G.gpu_fwd(w, dx, idx)
+    dq, dk, dv = G.gpu_bwd(w, dx, o, lse, idx)
+    g = G.geom_of(w)
+    idx_h = idx.cpu().numpy()
+    for b in range(w.B):
+        for h in range(w.H):
+            dQ, dK, dV, _, _ = oracle.bwd(g, x["q"][b, h], x["k"][b, h], x["v"][b, h], x["do"][b, h], idx_h[b, h])
+            for name, got, want in (("dQ", dq, dQ), ("dK", dk, dK), ("dV", dv, dV)):
+                gh = got[b, h].float().cpu().numpy().astype(np.float64)
+                assert np.isfinite(gh).all(), name
+                err = np.abs(gh - want).max()
+                assert err <= G.BWD_MAX_ABS, f"{name} max-abs {err:.4g}"
+                assert np.abs(gh - want).mean() <= 0.1 * max(np.abs(want).mean(), 1e-3), name
+
+
+def test_backward_is_deterministic():
+    w = BWD_CASES[0]
+    dx = G.device_inputs(synth.make_inputs(w))
+    idx = G.gpu_select(w, dx)
+    o, lse = G.gpu_fwd(w, dx, idx)
+    a = G.gpu_bwd(w, dx, o, lse, idx)
+    b = G.gpu_bwd(w, dx, o, lse, idx)
+    for s, t in zip(a, b):
+        assert torch.equal(s.view(torch.int16), t.view(torch.int16))
+
+
+def test_units_are_independent():
+    """Permuting (batch, head) units permutes the outputs bit for bit."""
+    w = synth.small_case(32, 64, 8, 8, 4, B=2, H=2, seed=45)
+    dx = G.device_inputs(synth.make_inputs(w))
+    idx = G.gpu_select(w, dx)
+    o, lse = G.gpu_fwd(w, dx, idx)
+    perm = {k: torch.flip(v, dims=[0, 1]).contiguous() for k, v in dx.items()}
+    idx_p = G.gpu_select(w, perm)
+    o_p, lse_p = G.gpu_fwd(w, perm, idx_p)
+    assert torch.equal(idx_p, torch.flip(idx, dims=[0, 1]))
+    assert torch.equal(o_p.view(torch.int16), torch.flip(o, dims=[0, 1]).view(torch.int16))
+    assert torch.equal(lse_p, torch.flip(lse, dims=[0, 1]))

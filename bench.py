@@ -1,0 +1,344 @@
+#!/usr/bin/env python
+"""Benchmark of the MOSAIC block-sparse attention hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+A step is one forward layer pass of the workload: block pooling + scoring + top-k selection,
+then the block-sparse attention forward (the backward of the same workload is timed beside it
+and reported under "stages").  Default workload: the 1.5-degree grid (120x240, 8x8 blocks,
+B=1, H=8, d=64, top-k 8) with seeded smooth+noise bf16 inputs.  Rank 0 prints ONE JSON line.
+
+value    effective TFLOP/s over the step: 4*d*b*b FLOP per attended (query block, key block)
+         pair, unmasked work only, inputs resident in HBM, L2 flushed between timed iterations,
+         device time by CUDA events, max over ranks.
+e2e      the same metric with the step's Q, K, V copied from pinned host memory and O copied
+         back inside the timed region.
+roofline the forward kernel alone against the measured dense bf16 peak of this GPU pool.
+cpu_baseline  the fp64 oracle timed on the host cores (reported, never optimised against).
+With N > 1 every rank runs the workload on its own GPU (weak scaling, no data-path collective).
+`--impl reference` times the oracle (CPU) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+from paper_2604_16429_b200 import flops, synth
+
+METRIC = "block-sparse attn effective TFLOP/s (select + fwd, ms/layer fwd at 1.5deg grid)"
+NOMINAL_BF16_TFLOPS = 2250.0
+FALLBACK_BF16_TFLOPS = 1590.0
+FALLBACK_HBM_GBS = 6650.0
+L2_FLUSH_BYTES = 256 << 20
+# DRAM bytes moved by one fwd_tc_kernel launch on the default workload (ncu, dram__bytes_read.sum +
+# dram__bytes_write.sum; see profiles/).  None until a capture exists for the workload.
+FWD_TRAFFIC_BYTES = {}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"bf16_tflops": float(p["bf16_tflops"]), "bf16_tflops_sustained": float(p["bf16_tflops_sustained"]),
+                "hbm_gbs": float(p["hbm_gbs"]), "source": "measured"}
+    return {"bf16_tflops": FALLBACK_BF16_TFLOPS, "bf16_tflops_sustained": 1400.0, "hbm_gbs": FALLBACK_HBM_GBS,
+            "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and clock-event reasons of one GPU through NVML while a region runs."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x10: "sync_boost"}
+
+    def __init__(self, cuda_index: int, period_s: float = 0.002):
+        self.samples, self.mask, self.max_mhz = [], 0, None
+        self.period, self._stop, self._thr, self.h = period_s, threading.Event(), None, None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID("GPU-" + str(torch.cuda.get_device_properties(cuda_index).uuid))
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(cuda_index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.h = None
+
+    def _loop(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    self.mask |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    self.mask |= int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def start(self):
+        if self.h is not None:
+            self._thr = threading.Thread(target=self._loop, daemon=True)
+            self._thr.start()
+
+    def stop(self) -> dict:
+        if self._thr is not None:
+            self._stop.set()
+            self._thr.join()
+        reasons = [n for bit, n in self.REASONS.items() if self.mask & bit]
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": reasons, "samples": len(self.samples)}
+
+
+def describe(w) -> str:
+    return (f"{w.name}: {w.nlat}x{w.nlon} grid, {w.bh}x{w.bw} blocks (m={w.m}), B={w.B}, H={w.H}, d={w.d}, "
+            f"local {2 * w.rlat + 1}x{2 * w.rlon + 1}, top-k {w.topk}, {w.kind} bf16 inputs")
+
+
+# ------------------------------------------------------------------------------------------
+def oracle_sample_step(w, x, g, blocks, unit=(0, 0)):
+    import oracle
+    b, h = unit
+    idx = oracle.select(g, x["q"][b, h], x["k"][b, h])
+    oracle.fwd(g, x["q"][b, h], x["k"][b, h], x["v"][b, h], idx, blocks)
+    return idx
+
+
+def sample_flops(w, g, blocks) -> float:
+    import oracle
+    pairs = sum(len(oracle.local_set(g, int(i))) + min(w.topk, w.m - len(oracle.local_set(g, int(i)))) for i in blocks)
+    return 4.0 * w.d * w.b * w.b * pairs
+
+
+def cpu_baseline(w, x, idx_gpu, o_gpu, lse_gpu) -> dict:
+    """Time the oracle, as it stands, on a bounded sample of the workload (about 10-30 core-seconds):
+    two whole units for 64-token blocks, 64 query blocks of one unit for larger blocks.  The sample
+    doubles as a parity spot check of the launch configuration that was just timed."""
+    import oracle
+    from oracle import Geom
+    oracle.build()
+    g = Geom(w.nlat, w.nlon, d=w.d, bh=w.bh, bw=w.bw, rlat=w.rlat, rlon=w.rlon, topk=w.topk)
+    rng = np.random.default_rng(0)
+    if w.b <= 64:
+        units = [(u // w.H, u % w.H) for u in range(min(2, w.U))]
+        blocks = np.arange(w.m, dtype=np.int32)
+    else:
+        units = [(0, 0)]
+        blocks = np.sort(rng.choice(w.m, size=min(w.m, 64), replace=False)).astype(np.int32)
+    oracle.local_set(g, 0)                                       # load the library before timing
+    fl, dt, worst = 0.0, 0.0, 0.0
+    for (b, h) in units:
+        t0 = time.perf_counter()
+        idx0 = oracle.select(g, x["q"][b, h], x["k"][b, h])
+        O, L = oracle.fwd(g, x["q"][b, h], x["k"][b, h], x["v"][b, h], idx0, blocks)
+        dt += time.perf_counter() - t0
+        fl += sample_flops(w, g, blocks)
+        assert np.array_equal(idx_gpu[b, h].cpu().numpy(), idx0), "selection differs from the oracle"
+        tok = np.concatenate([oracle.block_tokens(g, int(j)) for j in blocks])
+        err = np.abs(o_gpu[b, h].float().cpu().numpy()[tok] - O.reshape(-1, w.d))
+        lerr = np.abs(lse_gpu[b, h].cpu().numpy()[tok] - L.reshape(-1))
+        assert err.max() <= 2e-2 and err.mean() <= 2e-3 and lerr.max() <= 2e-3, (err.max(), err.mean(), lerr.max())
+        worst = max(worst, float(err.max()))
+    sample = (f"selection + forward of {len(units)} unit(s) x {len(blocks)} of {w.m} query blocks, {dt:.2f} s; "
+              f"GPU output of the sample within {worst:.2e} of it")
+    return {"value": fl / dt / 1e12, "unit": "TFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": sample}
+
+
+def run_reference(args, w):
+    """The oracle as it stands, on the host cores, on a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from oracle import Geom
+    oracle.build()
+    g = Geom(w.nlat, w.nlon, d=w.d, bh=w.bh, bw=w.bw, rlat=w.rlat, rlon=w.rlon, topk=w.topk)
+    one = synth.Workload(**{**w.__dict__, "B": 1, "H": 1})
+    x = synth.make_inputs(one, with_do=False)
+    rng = np.random.default_rng(0)
+    nb = min(w.m, 64 if w.b <= 64 else 8)
+    blocks = np.sort(rng.choice(w.m, size=nb, replace=False)).astype(np.int32)
+    fl = sample_flops(w, g, blocks)
+    for _ in range(args.warmup):
+        oracle_sample_step(w, x, g, blocks)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_sample_step(w, x, g, blocks)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = fl / dt / 1e12
+    sample = f"selection of 1 unit + forward of {nb} of {w.m} query blocks of that unit per step (seed 0)"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": describe(w), "sample": sample},
+            "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------
+def run_ours(args, w):
+    import torch
+
+    from paper_2604_16429_b200 import binding as mb
+    from paper_2604_16429_b200 import dist as mdist
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    rank, local_rank, world = mdist.init()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    mb.lib()  # fail loudly if the library is missing
+
+    # every rank runs the same workload on its own members: per-rank noise seeds differ by rank
+    wl = synth.Workload(**{**w.__dict__, "cfg": w.cfg + 100 * rank}) if world > 1 else w
+    x = synth.make_inputs(wl, with_do=True)
+    host = {k: torch.from_numpy(v.view(np.int16)).pin_memory() for k, v in x.items()}
+    dx = {k: t.to(dev, non_blocking=True).view(torch.bfloat16) for k, t in host.items()}
+    p = mb.Params.from_workload(w)
+    ws = torch.empty(max(mb.workspace_bytes(p, op) for op in (mb.OP_SELECT, mb.OP_FWD, mb.OP_BWD)),
+                     dtype=torch.uint8, device=dev)
+    idx = torch.empty((w.B, w.H, w.m, w.topk), dtype=torch.int32, device=dev)
+    o = torch.empty_like(dx["q"])
+    lse = torch.empty((w.B, w.H, w.N), dtype=torch.float32, device=dev)
+    dq, dk, dv = (torch.empty_like(dx["q"]) for _ in range(3))
+    flush_buf = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def fwd_step(ev=None):
+        if ev:
+            ev[0].record(stream)
+        mb.mosaic_bsa_select(p, dx["q"], dx["k"], block_idx=idx, ws=ws)
+        if ev:
+            ev[1].record(stream)
+        mb.mosaic_bsa_fwd(p, dx["q"], dx["k"], dx["v"], idx, o=o, lse=lse, ws=ws)
+        if ev:
+            ev[2].record(stream)
+
+    def bwd_step():
+        mb.mosaic_bsa_bwd(p, dx["q"], dx["k"], dx["v"], o, lse, dx["do"], idx, dq=dq, dk=dk, dv=dv, ws=ws)
+
+    for _ in range(max(args.warmup, 3)):
+        flush_buf.zero_()
+        fwd_step()
+    bwd_step()
+    torch.cuda.synchronize()
+    mb.check_status(ws, "warm-up")
+
+    K = args.steps
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+    sampler = ClockSampler(local_rank)
+    mdist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    for s in range(K):
+        flush_buf.zero_()          # L2 flush, outside the timed interval of the step
+        fwd_step(evs[s])
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    mdist.barrier()
+    t_sel = sum(e[0].elapsed_time(e[1]) for e in evs) / K
+    t_fwd = sum(e[1].elapsed_time(e[2]) for e in evs) / K
+    t_step = sum(e[0].elapsed_time(e[2]) for e in evs) / K
+    mb.check_status(ws, "timed region")
+
+    # backward of the same workload, timed the same way (reported under "stages")
+    kb = min(K, 20)
+    evb = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(kb)]
+    for s in range(kb):
+        flush_buf.zero_()
+        evb[s][0].record(stream)
+        bwd_step()
+        evb[s][1].record(stream)
+    torch.cuda.synchronize()
+    t_bwd = sum(e[0].elapsed_time(e[1]) for e in evb) / kb
+
+    # end to end: pinned host -> device, step, device -> pinned host
+    ke = min(K, 10)
+    o_host = torch.empty(o.shape, dtype=torch.int16).pin_memory()
+    eve = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(ke)]
+    for s in range(ke + 1):
+        if s:
+            eve[s - 1][0].record(stream)
+        for name in ("q", "k", "v"):
+            dx[name].view(torch.int16).copy_(host[name], non_blocking=True)
+        fwd_step()
+        o_host.copy_(o.view(torch.int16), non_blocking=True)
+        if s:
+            eve[s - 1][1].record(stream)
+    torch.cuda.synchronize()
+    t_e2e = sum(e[0].elapsed_time(e[1]) for e in eve) / ke
+    h2d = 3 * dx["q"].numel() * 2
+    d2h = o.numel() * 2
+
+    t_step_max = mdist.max_over_ranks(t_step, dev)
+    t_e2e_max = mdist.max_over_ranks(t_e2e, dev)
+    fl = flops.fwd_flops(w)
+    value = world * fl / (t_step_max * 1e-3) / 1e12
+    peaks = measured_peaks()
+    fwd_tflops = fl / (t_fwd * 1e-3) / 1e12
+    pool_bytes = 2.0 * w.U * w.N * w.d * 2
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
+        "ms_per_step": t_step_max, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": describe(w), "l2": f"flushed between timed iterations ({L2_FLUSH_BYTES >> 20} MiB write)",
+                   "step": "select (pool + top-k) + forward", "parallelism": f"replicas x{world}, no collective"},
+        "clocks": clocks,
+        "e2e": {"value": world * fl / (t_e2e_max * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": t_e2e_max,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": 3 * K,
+        "roofline": {"kernel": "fwd_tc_kernel", "bound": "tensor", "achieved": fwd_tflops,
+                     "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": fwd_tflops / peaks["bf16_tflops"],
+                     "traffic": FWD_TRAFFIC_BYTES.get(w.name), "peak_source": peaks["source"] + " (burst)",
+                     "frac_of_nominal_2250": fwd_tflops / NOMINAL_BF16_TFLOPS, "ms": t_fwd},
+        "stages": {"select_ms": t_sel, "fwd_ms": t_fwd, "bwd_ms": t_bwd, "ms_layer_fwd": t_step,
+                   "fwd_tflops": fwd_tflops, "bwd_tflops": flops.bwd_flops(w) / (t_bwd * 1e-3) / 1e12,
+                   "select_pool_gbs_lower_bound": pool_bytes / (t_sel * 1e-3) / 1e9,
+                   "pct_of_nominal_peak": 100 * fwd_tflops / NOMINAL_BF16_TFLOPS,
+                   "pct_of_measured_peak": 100 * fwd_tflops / peaks["bf16_tflops"]},
+    }
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(w, x, idx, o, lse)
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    mdist.finalize()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--workload", default="c2_1p5deg", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = synth.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

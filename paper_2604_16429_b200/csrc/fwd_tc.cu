@@ -16,11 +16,13 @@
 //
 // Warp roles (192 threads): warps 0-3 softmax (thread r owns query row r = TMEM lane r),
 // warp 4 builds the key list and issues TMA, warp 5 allocates TMEM and issues tcgen05.mma.
-// TMEM columns: [0,64) O accumulator, [64,128) and [128,192) two S buffers; P (bf16) overwrites
-// the first 32 columns of its S buffer and is consumed from TMEM as the A operand of P V.
+// TMEM columns: [0,64) O accumulator, then SBUFS S buffers of 64 columns; P (bf16) overwrites the
+// first 32 columns of its S buffer and is consumed from TMEM as the A operand of P V.
+// Several CTAs are resident per SM, so one CTA's softmax overlaps another's tensor work.
 // Every mbarrier wait is bounded; on expiry the CTA records MOSAIC_E_DEVICE_TIMEOUT and drains.
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 
@@ -28,23 +30,21 @@ namespace mosaic {
 
 namespace {
 
-constexpr int NSTAGE = 4;
 constexpr int kTile = 8192;                    // bytes of one 64 x 64 bf16 chunk
-constexpr uint32_t kTmemCols = 256;
 constexpr uint32_t kColO = 0, kColS = 64;
 constexpr long long kSpinCycles = 4000000000ll;  // bound of a single wait (~2 s)
 constexpr float kRescaleThreshold = 8.0f;      // log2 units: P stays below 2^8
 
+template <int NST, int SBUFS>
 struct SmemTC {
   unsigned char q[2 * kTile];
-  unsigned char kv[NSTAGE][2][kTile];
-  unsigned long long kv_full[NSTAGE], kv_empty[NSTAGE], q_full, s_full[2], p_full[2], pv_done[2];
+  unsigned char kv[NST][2][kTile];
+  unsigned long long kv_full[NST], kv_empty[NST], q_full, s_full[SBUFS], p_full[SBUFS], pv_done[SBUFS];
   uint32_t tmem_base;
   int abort;
   int nlist;
   int ids[2 * kMaxList];
   unsigned char mask[2 * kMaxList];
-  int tmp[kMaxList];
 };
 
 __device__ __forceinline__ uint32_t s32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -68,16 +68,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait.  Returns false after the limit (status recorded) or once another thread aborted.
+// The clock and the abort flag are looked at only every 64 polls to keep the poll loop light.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort, int* status) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
-  while (true) {
+#pragma unroll 1
+  for (uint32_t i = 1;; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (*abort) return false;
-    if (clock64() - t0 > kSpinCycles) {
-      set_status(status, MOSAIC_E_DEVICE_TIMEOUT);
-      *abort = 1;
-      return false;
+    if ((i & 63u) == 0u) {
+      if (*abort) return false;
+      if (clock64() - t0 > kSpinCycles) {
+        set_status(status, MOSAIC_E_DEVICE_TIMEOUT);
+        *abort = 1;
+        return false;
+      }
     }
   }
 }
@@ -156,6 +160,31 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
+// two fp32 lanes in one 64-bit register (packed fp32 arithmetic of this architecture)
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("mul.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
 // Shared-memory operand descriptor: 128-byte swizzle, 8-row groups 1024 B apart.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
   uint64_t d = (uint64_t)((addr & 0x3FFFFu) >> 4);
@@ -173,31 +202,60 @@ __host__ __device__ constexpr uint32_t make_idesc(bool b_mn_major) {
 
 }  // namespace
 
-__global__ void __launch_bounds__(192, 2)
+// Warp-cooperative attended list of query block i (local set, then valid selected ids), appended to
+// ids[n0..); returns the new count.  Same order as attended_list().
+__device__ __forceinline__ int warp_attended(const Geo& g, const int32_t* __restrict__ idx_row, int i, int* ids,
+                                             int n0, int lane, int* status) {
+  const int by = i / g.nbw, bx = i - by * g.nbw;
+  const int wl = 2 * g.rlon + 1, nl = (2 * g.rlat + 1) * wl;
+  int id = -1 - lane;
+  if (lane < nl) {
+    const int dy = lane / wl - g.rlat, dx = lane - (lane / wl) * wl - g.rlon;
+    const int y = min(max(by + dy, 0), g.nbh - 1);
+    int x = (bx + dx) % g.nbw;
+    x += x < 0 ? g.nbw : 0;
+    id = y * g.nbw + x;
+  }
+  const unsigned same = __match_any_sync(0xffffffffu, id);
+  const bool keep = lane < nl && (__ffs(same) - 1) == lane;  // first occurrence of a block
+  const unsigned km = __ballot_sync(0xffffffffu, keep);
+  if (keep) ids[n0 + __popc(km & ((1u << lane) - 1u))] = id;
+  int n = n0 + __popc(km);
+  int j = lane < g.topk ? __ldg(idx_row + lane) : -1;
+  if (j < -1 || j >= g.m) { set_status(status, MOSAIC_E_DEVICE_BAD_INDEX); j = -1; }
+  const unsigned sm_ = __ballot_sync(0xffffffffu, j >= 0);
+  if (j >= 0) ids[n + __popc(sm_ & ((1u << lane) - 1u))] = j;
+  return n + __popc(sm_);
+}
+
+template <int NST, int SBUFS, int MINB>
+__global__ void __launch_bounds__(192, MINB)
     fwd_tc_kernel(const Geo g, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_v, const int32_t* __restrict__ block_idx,
                   __nv_bfloat16* __restrict__ o, float* __restrict__ lse, int* status, int tiles_per_unit) {
+  using Smem = SmemTC<NST, SBUFS>;
+  constexpr uint32_t kTmemCols = SBUFS == 1 ? 128 : 256;
   extern __shared__ unsigned char smem_raw[];
-  SmemTC& sm = *reinterpret_cast<SmemTC*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int u = blockIdx.x / tiles_per_unit, t = blockIdx.x - u * tiles_per_unit;
 
   // the two 64-row halves of the tile: (block, chunk) each
-  int hb[2], hc[2];
+  int hb0, hb1, hc0, hc1;
   bool hvalid1 = true;
   if (g.cpb == 1) {
-    hb[0] = 2 * t; hb[1] = 2 * t + 1; hc[0] = hc[1] = 0;
-    if (hb[1] >= g.m) { hvalid1 = false; hb[1] = hb[0]; }
+    hb0 = 2 * t; hb1 = 2 * t + 1; hc0 = hc1 = 0;
+    if (hb1 >= g.m) { hvalid1 = false; hb1 = hb0; }
   } else {
     const int hpb = g.cpb / 2;  // tiles per block
-    hb[0] = hb[1] = t / hpb;
-    hc[0] = 2 * (t % hpb); hc[1] = hc[0] + 1;
+    hb0 = hb1 = t / hpb;
+    hc0 = 2 * (t % hpb); hc1 = hc0 + 1;
   }
 
   if (tid == 0) {
-    for (int s = 0; s < NSTAGE; ++s) { mbar_init(s32(&sm.kv_full[s]), 1); mbar_init(s32(&sm.kv_empty[s]), 1); }
+    for (int s = 0; s < NST; ++s) { mbar_init(s32(&sm.kv_full[s]), 1); mbar_init(s32(&sm.kv_empty[s]), 1); }
     mbar_init(s32(&sm.q_full), 1);
-    for (int s = 0; s < 2; ++s) {
+    for (int s = 0; s < SBUFS; ++s) {
       mbar_init(s32(&sm.s_full[s]), 1);
       mbar_init(s32(&sm.p_full[s]), 128);
       mbar_init(s32(&sm.pv_done[s]), 1);
@@ -206,29 +264,61 @@ __global__ void __launch_bounds__(192, 2)
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  __syncthreads();
   if (warp == 5) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(&sm.tmem_base)),
                  "r"(kTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  if (warp == 4 && lane == 0) {
+  if (warp == 4) {
+    if (lane == 0) {  // the query tile does not depend on the key list: start it first
+      mbar_expect_tx(s32(&sm.q_full), 2 * kTile);
+      int by = hb0 / g.nbw, bx = hb0 - by * g.nbw;
+      tma_load_4d(s32(sm.q), &map_q, s32(&sm.q_full), 0, bx * g.bw, by * g.bh + hc0 * g.crows, u);
+      by = hb1 / g.nbw; bx = hb1 - by * g.nbw;
+      tma_load_4d(s32(sm.q + kTile), &map_q, s32(&sm.q_full), 0, bx * g.bw, by * g.bh + hc1 * g.crows, u);
+    }
     // key list: entries of the first half's block, then what only the second half adds
-    const int32_t* row0 = block_idx + ((long long)u * g.m + hb[0]) * g.topk;
-    int n = attended_list(g, row0, hb[0], sm.ids, status);
-    for (int e = 0; e < n; ++e) sm.mask[e] = g.cpb == 1 ? 1 : 3;
+    const int32_t* row0 = block_idx + ((long long)u * g.m + hb0) * g.topk;
+    int n = warp_attended(g, row0, hb0, sm.ids, 0, lane, status);
+    __syncwarp();
+    const unsigned char m0 = g.cpb == 1 ? 1 : 3;
+    for (int e = lane; e < n; e += 32) sm.mask[e] = m0;
     if (g.cpb == 1 && hvalid1) {
-      const int32_t* row1 = block_idx + ((long long)u * g.m + hb[1]) * g.topk;
-      int n1 = attended_list(g, row1, hb[1], sm.tmp, status);
+      const int32_t* row1 = block_idx + ((long long)u * g.m + hb1) * g.topk;
       const int n0 = n;
-      for (int e = 0; e < n1; ++e) {
-        int id = sm.tmp[e], pos = -1;
-        for (int a = 0; a < n0; ++a) pos = sm.ids[a] == id ? a : pos;
-        if (pos >= 0) sm.mask[pos] |= 2;
-        else { sm.ids[n] = id; sm.mask[n] = 2; ++n; }
+      const int n1 = warp_attended(g, row1, hb1, sm.ids, n0, lane, status) - n0;  // staged behind list 0
+      __syncwarp();
+      // entries of list 1 (at most 2 per lane): shared with list 0 -> mark, else keep (compacted)
+      int mine[2], pos[2];
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        const int e = lane + 32 * r;
+        mine[r] = e < n1 ? sm.ids[n0 + e] : -1;
+        pos[r] = -1;
+      }
+      for (int a = 0; a < n0; ++a) {
+        const int id = sm.ids[a];
+        pos[0] = id == mine[0] ? a : pos[0];
+        pos[1] = id == mine[1] ? a : pos[1];
+      }
+      __syncwarp();
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        const bool have = mine[r] >= 0, fresh = have && pos[r] < 0;
+        if (have && pos[r] >= 0) sm.mask[pos[r]] |= 2;
+        const unsigned fm = __ballot_sync(0xffffffffu, fresh);
+        if (fresh) {
+          const int at = n + __popc(fm & ((1u << lane) - 1u));
+          sm.ids[at] = mine[r];
+          sm.mask[at] = 2;
+        }
+        n += __popc(fm);
+        __syncwarp();
       }
     }
-    sm.nlist = n;
+    if (lane == 0) sm.nlist = n;
   }
   tc_fence_before();
   __syncthreads();
@@ -241,14 +331,9 @@ __global__ void __launch_bounds__(192, 2)
   if (warp == 4) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      mbar_expect_tx(s32(&sm.q_full), 2 * kTile);
-      for (int h = 0; h < 2; ++h) {
-        int by = hb[h] / g.nbw, bx = hb[h] - by * g.nbw;
-        tma_load_4d(s32(sm.q + h * kTile), &map_q, s32(&sm.q_full), 0, bx * g.bw, by * g.bh + hc[h] * g.crows, u);
-      }
       for (int it = 0; it < nch; ++it) {
-        const int st = it % NSTAGE, j = sm.ids[it / g.cpb], c = it % g.cpb;
-        if (!mbar_wait(s32(&sm.kv_empty[st]), ((it / NSTAGE) & 1) ^ 1, abort, status)) break;
+        const int st = it % NST, j = sm.ids[it / g.cpb], c = it % g.cpb;
+        if (!mbar_wait(s32(&sm.kv_empty[st]), ((it / NST) & 1) ^ 1, abort, status)) break;
         const int by = j / g.nbw, bx = j - by * g.nbw;
         mbar_expect_tx(s32(&sm.kv_full[st]), 2 * kTile);
         tma_load_4d(s32(sm.kv[st][0]), &map_k, s32(&sm.kv_full[st]), 0, bx * g.bw, by * g.bh + c * g.crows, u);
@@ -266,45 +351,56 @@ __global__ void __launch_bounds__(192, 2)
       const uint64_t qdesc = smem_desc(s32(sm.q));
       bool ok = mbar_wait(s32(&sm.q_full), 0, abort, status);
       auto issue_qk = [&](int it) {
-        const uint64_t kdesc = smem_desc(s32(sm.kv[it % NSTAGE][0]));
-        const uint32_t d = tmem + kColS + (it & 1) * 64;
+        const uint64_t kdesc = smem_desc(s32(sm.kv[it % NST][0]));
+        const uint32_t d = tmem + kColS + (it % SBUFS) * 64;
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk) umma_ss(d, qdesc + 2 * kk, kdesc + 2 * kk, idesc_qk, kk > 0);
-        tc_commit(s32(&sm.s_full[it & 1]));
+        tc_commit(s32(&sm.s_full[it % SBUFS]));
+      };
+      // S buffer of iteration `it` is free once P V of iteration it - SBUFS has completed
+      auto wait_sbuf = [&](int it) {
+        const int prev = it - SBUFS;
+        return prev < 0 || mbar_wait(s32(&sm.pv_done[prev % SBUFS]), (prev / SBUFS) & 1, abort, status);
       };
       if (ok && nch > 0) {
         ok = mbar_wait(s32(&sm.kv_full[0]), 0, abort, status);
         if (ok) { tc_fence_after(); issue_qk(0); }
       }
       for (int it = 0; ok && it < nch; ++it) {
-        if (it + 1 < nch) {
-          ok = mbar_wait(s32(&sm.kv_full[(it + 1) % NSTAGE]), ((it + 1) / NSTAGE) & 1, abort, status);
-          if (ok && it >= 1) ok = mbar_wait(s32(&sm.pv_done[(it + 1) & 1]), ((it - 1) >> 1) & 1, abort, status);
+        if (SBUFS > 1 && it + 1 < nch) {
+          ok = mbar_wait(s32(&sm.kv_full[(it + 1) % NST]), ((it + 1) / NST) & 1, abort, status) && wait_sbuf(it + 1);
           if (!ok) break;
           tc_fence_after();
           issue_qk(it + 1);
         }
-        ok = mbar_wait(s32(&sm.p_full[it & 1]), (it >> 1) & 1, abort, status);
+        ok = mbar_wait(s32(&sm.p_full[it % SBUFS]), (it / SBUFS) & 1, abort, status);
         if (!ok) break;
         tc_fence_after();
-        const uint64_t vdesc = smem_desc(s32(sm.kv[it % NSTAGE][1]));
-        const uint32_t p = tmem + kColS + (it & 1) * 64;
+        const uint64_t vdesc = smem_desc(s32(sm.kv[it % NST][1]));
+        const uint32_t p = tmem + kColS + (it % SBUFS) * 64;
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk)
           umma_ts(tmem + kColO, p + 8 * kk, vdesc + (uint64_t)((2048 * kk) >> 4), idesc_pv, (it > 0 || kk > 0));
-        tc_commit(s32(&sm.kv_empty[it % NSTAGE]));
-        tc_commit(s32(&sm.pv_done[it & 1]));
+        tc_commit(s32(&sm.kv_empty[it % NST]));
+        tc_commit(s32(&sm.pv_done[it % SBUFS]));
+        if (SBUFS == 1 && it + 1 < nch) {
+          ok = mbar_wait(s32(&sm.kv_full[(it + 1) % NST]), ((it + 1) / NST) & 1, abort, status) && wait_sbuf(it + 1);
+          if (!ok) break;
+          tc_fence_after();
+          issue_qk(it + 1);
+        }
       }
     }
   } else {
     // ------------------------------------------------------------------ softmax, then epilogue
     const int h = warp >> 1;  // which 64-row half this warp's rows belong to
     const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    const uint64_t scale2 = pack2(g.scale_log2, g.scale_log2);
     float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
     for (int it = 0; it < nch; ++it) {
-      const int sb = it & 1;
-      ok = mbar_wait(s32(&sm.s_full[sb]), (it >> 1) & 1, abort, status);
+      const int sb = it % SBUFS;
+      ok = mbar_wait(s32(&sm.s_full[sb]), (it / SBUFS) & 1, abort, status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -318,10 +414,16 @@ __global__ void __launch_bounds__(192, 2)
         tmem_ld32<0>(ts, sr);
         tmem_ld32<32>(ts + 32, sr);
         tmem_wait_ld();
-        float mx = -INFINITY;
+        float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]), mx2 = __uint_as_float(sr[2]),
+              mx3 = __uint_as_float(sr[3]);
 #pragma unroll
-        for (int c = 0; c < 64; ++c) mx = fmaxf(mx, __uint_as_float(sr[c]));
-        mx *= g.scale_log2;  // scale > 0, so the maximum commutes with it
+        for (int c = 4; c < 64; c += 4) {
+          mx0 = fmaxf(mx0, __uint_as_float(sr[c]));
+          mx1 = fmaxf(mx1, __uint_as_float(sr[c + 1]));
+          mx2 = fmaxf(mx2, __uint_as_float(sr[c + 2]));
+          mx3 = fmaxf(mx3, __uint_as_float(sr[c + 3]));
+        }
+        const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * g.scale_log2;  // scale > 0 commutes with max
         if (m_ref == -INFINITY) {
           m_ref = mx;
         } else if (mx > m_ref + kRescaleThreshold) {
@@ -330,16 +432,23 @@ __global__ void __launch_bounds__(192, 2)
           m_ref = mx;
           l *= alpha;
         }
-        float sum = 0.f;
+        const uint64_t negm2 = pack2(-m_ref, -m_ref);
+        uint64_t sum_a = pack2(0.f, 0.f), sum_b = sum_a;
 #pragma unroll
-        for (int c = 0; c < 64; c += 2) {
-          float p0 = ex2(fmaf(__uint_as_float(sr[c]), g.scale_log2, -m_ref));
-          float p1 = ex2(fmaf(__uint_as_float(sr[c + 1]), g.scale_log2, -m_ref));
-          sum += p0 + p1;
-          __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
-          pk[c >> 1] = *reinterpret_cast<uint32_t*>(&pb);
+        for (int c = 0; c < 64; c += 4) {
+          float x0, x1, x2, x3;
+          unpack2(fma2(pack2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), scale2, negm2), x0, x1);
+          unpack2(fma2(pack2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), scale2, negm2), x2, x3);
+          const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
+          sum_a = add2(sum_a, pack2(p0, p1));
+          sum_b = add2(sum_b, pack2(p2, p3));
+          __nv_bfloat162 pa = __floats2bfloat162_rn(p0, p1), pb = __floats2bfloat162_rn(p2, p3);
+          pk[c >> 1] = *reinterpret_cast<uint32_t*>(&pa);
+          pk[(c >> 1) + 1] = *reinterpret_cast<uint32_t*>(&pb);
         }
-        l += sum;
+        float s0, s1;
+        unpack2(add2(sum_a, sum_b), s0, s1);
+        l += s0 + s1;
       } else {
 #pragma unroll
         for (int c = 0; c < 32; ++c) pk[c] = 0u;
@@ -348,19 +457,25 @@ __global__ void __launch_bounds__(192, 2)
       if (__any_sync(0xffffffffu, need)) {
         // the accumulator may only be touched between P V products
         if (it > 0) {
-          ok = mbar_wait(s32(&sm.pv_done[(it - 1) & 1]), ((it - 1) >> 1) & 1, abort, status);
+          ok = mbar_wait(s32(&sm.pv_done[(it - 1) % SBUFS]), ((it - 1) / SBUFS) & 1, abort, status);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
         }
         const uint32_t to = tmem + lane_off + kColO;
+        const uint64_t alpha2 = pack2(alpha, alpha);
 #pragma unroll
         for (int part = 0; part < 2; ++part) {
           uint32_t ov[32];
           tmem_ld32<0>(to + 32 * part, ov);
           tmem_wait_ld();
 #pragma unroll
-          for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * alpha);
+          for (int c = 0; c < 32; c += 2) {
+            float a, b;
+            unpack2(mul2(pack2(__uint_as_float(ov[c]), __uint_as_float(ov[c + 1])), alpha2), a, b);
+            ov[c] = __float_as_uint(a);
+            ov[c + 1] = __float_as_uint(b);
+          }
           tmem_st32<0>(to + 32 * part, ov);
         }
       }
@@ -370,13 +485,13 @@ __global__ void __launch_bounds__(192, 2)
     }
     if (ok && nch > 0) {
       const int last = nch - 1;
-      ok = mbar_wait(s32(&sm.pv_done[last & 1]), (last >> 1) & 1, abort, status);
+      ok = mbar_wait(s32(&sm.pv_done[last % SBUFS]), (last / SBUFS) & 1, abort, status);
       ok = __all_sync(0xffffffffu, ok);
     }
     if (ok && nch > 0 && (h == 0 || hvalid1)) {
       tc_fence_after();
       const int e = tid & 63;
-      const long long tok = (long long)u * g.N + chunk_token(g, hb[h], hc[h], e);
+      const long long tok = (long long)u * g.N + chunk_token(g, h ? hb1 : hb0, h ? hc1 : hc0, e);
       const float inv = 1.f / l;
       const uint32_t to = tmem + lane_off + kColO;
       uint4* dst = reinterpret_cast<uint4*>(o + tok * kD);
@@ -402,6 +517,7 @@ __global__ void __launch_bounds__(192, 2)
   __syncthreads();
   if (warp == 5) {
     tc_fence_after();
+    __syncwarp();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
   }
 }
@@ -441,20 +557,34 @@ bool make_map(CUtensorMap* map, const void* base, const Geo& g) {
 
 }  // namespace
 
+template <int NST, int SBUFS, int MINB>
+int launch_variant(const HostCtx& c, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+                   const int32_t* block_idx, void* o, float* lse) {
+  const Geo& g = c.g;
+  auto kern = fwd_tc_kernel<NST, SBUFS, MINB>;
+  const size_t smem = sizeof(SmemTC<NST, SBUFS>) + 1024;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return MOSAIC_E_CUDA;
+  const int tiles_per_unit = g.cpb == 1 ? (g.m + 1) / 2 : g.m * (g.cpb / 2);
+  const long long grid = (long long)g.U * tiles_per_unit;
+  kern<<<(unsigned)grid, 192, smem, c.stream>>>(g, mq, mk, mv, block_idx, (__nv_bfloat16*)o, lse, c.status,
+                                                tiles_per_unit);
+  return cudaGetLastError() == cudaSuccess ? MOSAIC_OK : MOSAIC_E_CUDA;
+}
+
 int launch_fwd_tc(const HostCtx& c, const void* q, const void* k, const void* v, const int32_t* block_idx, void* o,
                   float* lse) {
   const Geo& g = c.g;
   if (!(g.cpb == 1 || g.cpb % 2 == 0)) return MOSAIC_E_UNSUPPORTED;
   CUtensorMap mq, mk, mv;
   if (!make_map(&mq, q, g) || !make_map(&mk, k, g) || !make_map(&mv, v, g)) return MOSAIC_E_CUDA;
-  const size_t smem = sizeof(SmemTC) + 1024;
-  if (cudaFuncSetAttribute(fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-    return MOSAIC_E_CUDA;
-  const int tiles_per_unit = g.cpb == 1 ? (g.m + 1) / 2 : g.m * (g.cpb / 2);
-  const long long grid = (long long)g.U * tiles_per_unit;
-  fwd_tc_kernel<<<(unsigned)grid, 192, smem, c.stream>>>(g, mq, mk, mv, block_idx, (__nv_bfloat16*)o, lse, c.status,
-                                                         tiles_per_unit);
-  return cudaGetLastError() == cudaSuccess ? MOSAIC_OK : MOSAIC_E_CUDA;
+  const char* var = getenv("MOSAIC_BSA_FWD_VARIANT");  // tuning aid; default below
+  const int which = var ? atoi(var) : 0;
+  switch (which) {
+    case 1: return launch_variant<3, 1, 3>(c, mq, mk, mv, block_idx, o, lse);
+    case 2: return launch_variant<2, 1, 4>(c, mq, mk, mv, block_idx, o, lse);
+    default: return launch_variant<4, 2, 2>(c, mq, mk, mv, block_idx, o, lse);
+  }
 }
 
 }  // namespace mosaic

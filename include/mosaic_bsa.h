@@ -111,6 +111,34 @@ int mosaic_bsa_bwd(const mosaic_bsa_params *p, const void *q, const void *k, con
                    const void *o, const float *lse, const void *d_o, const int32_t *block_idx,
                    void *dq, void *dk, void *dv, void *ws, size_t ws_bytes, void *cuda_stream);
 
+/*
+ * Selection for callers that cannot allocate device memory.  (The paper has no counterpart of this
+ * entry point: it computes exactly what mosaic_bsa_select computes, with the same arguments minus the
+ * workspace.)
+ *
+ * Some callers cannot hand the library a workspace: a process whose framework claimed its whole memory
+ * budget at start-up, a plug-in whose host application owns the allocator, a latency-critical loop in
+ * which cudaMalloc (it may synchronise the device) is forbidden.  For them the scratch of the selection
+ * (the pooled block sums of Q and K) lives in a fixed array inside the library image,
+ * MOSAIC_BSA_STATIC_SCRATCH_BYTES long; every GPU that loads the library holds that array until the
+ * process exits.  The call performs no cudaMalloc, cudaFree or other allocating routine.
+ *   q, k       in   [B,H,N,d] bf16 (device)
+ *   block_idx  out  [B,H,m,topk] int32 (device)
+ * Limits and rules
+ *   - The problem must fit: 256 + 2 * round_up_256(B*H*m*d*4) <= MOSAIC_BSA_STATIC_SCRATCH_BYTES,
+ *     i.e. about B*H*m <= 8190 blocks for d = 64 (the 1.5-degree grid with 8 heads uses 3600).  A larger
+ *     problem returns MOSAIC_E_WORKSPACE_TOO_SMALL and launches nothing.
+ *   - The first call on each device looks up the device address of the array (with that device current)
+ *     and remembers it; make that first call before any stream capture begins.
+ *   - All calls on a device share the one array, which keeps the previous call's contents (the call
+ *     clears what has to start at zero).  Two calls that overlap on the GPU -- different streams without
+ *     an ordering between them -- race on it: keep calls of this entry point ordered.
+ *   - Other return codes as for mosaic_bsa_select.
+ */
+#define MOSAIC_BSA_STATIC_SCRATCH_BYTES (4u << 20)
+int mosaic_bsa_select_static(const mosaic_bsa_params *p, const void *q, const void *k, int32_t *block_idx,
+                             void *cuda_stream);
+
 /* Synchronises `cuda_stream`, then returns the device status word of `ws`
  * (MOSAIC_OK, MOSAIC_E_DEVICE_*) or MOSAIC_E_CUDA if the stream reports an error.
  * Every op resets the word when it starts. */

@@ -19,7 +19,8 @@ _lib = None
 
 OP_SELECT, OP_FWD, OP_BWD = 0, 1, 2
 EXPORTS = ("mosaic_bsa_workspace_bytes", "mosaic_bsa_select", "mosaic_bsa_fwd", "mosaic_bsa_bwd",
-           "mosaic_bsa_last_status", "mosaic_bsa_strerror")
+           "mosaic_bsa_last_status", "mosaic_bsa_strerror", "mosaic_bsa_select_static")
+STATIC_SCRATCH_BYTES = 4 << 20
 
 
 class MosaicError(RuntimeError):
@@ -82,6 +83,8 @@ def lib():
         L.mosaic_bsa_workspace_bytes.argtypes = [pp, ctypes.c_int]
         L.mosaic_bsa_select.restype = ctypes.c_int
         L.mosaic_bsa_select.argtypes = [pp, vp, vp, i32p, vp, ctypes.c_size_t, vp]
+        L.mosaic_bsa_select_static.restype = ctypes.c_int
+        L.mosaic_bsa_select_static.argtypes = [pp, vp, vp, i32p, vp]
         L.mosaic_bsa_fwd.restype = ctypes.c_int
         L.mosaic_bsa_fwd.argtypes = [pp, vp, vp, vp, i32p, vp, fp, vp, ctypes.c_size_t, vp]
         L.mosaic_bsa_bwd.restype = ctypes.c_int
@@ -136,6 +139,19 @@ def mosaic_bsa_select(p: Params, q, k, block_idx=None, ws=None, stream=None):
                                  _stream(stream))
     if rc:
         raise MosaicError(rc, "mosaic_bsa_select")
+    return block_idx
+
+
+def mosaic_bsa_select_static(p: Params, q, k, block_idx=None, stream=None):
+    """Selection through the entry point that allocates nothing (scratch inside the library image).
+    Only `block_idx` is created here when the caller passes none."""
+    _chk_qkv(p, q, k)
+    if block_idx is None:
+        block_idx = torch.empty((p.B, p.H, p.m, p.topk), dtype=torch.int32, device=q.device)
+    pc = p.c()
+    rc = lib().mosaic_bsa_select_static(ctypes.byref(pc), _ptr(q), _ptr(k), _ptr(block_idx), _stream(stream))
+    if rc:
+        raise MosaicError(rc, "mosaic_bsa_select_static")
     return block_idx
 
 

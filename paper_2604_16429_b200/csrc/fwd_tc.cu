@@ -5,24 +5,28 @@
 // softmax; streaming evaluation with the query tile resident on chip and key/value blocks streamed
 // through, as the appendix paragraph "Kernel Design" describes.
 //
-// One CTA owns a tile of 128 query rows:
-//   * 64-token blocks (8x8): two consecutive query blocks share the tile; the CTA walks the UNION of
-//     their key lists and each 64-row half skips (P = 0) the blocks only the other half attends, so
-//     every staged key/value block serves both halves.
-//   * larger blocks (16x16): half of one query block (two 64-token chunks); one key list.
+// Work item = 256 query rows = two 128-row tiles = four 64-row "halves", each half one 64-token chunk
+// of a query block:
+//   * 64-token blocks (8x8): a 2x2 group of query blocks (a 1x4 group on an odd last block row); the
+//     CTA walks the UNION of the four key lists, every entry carrying a 4-bit mask of the halves that
+//     attend it.  A tile skips entries none of its halves attends; a half that does not attend an entry
+//     its tile computes writes P = 0.
+//   * 128-token blocks: two neighbouring query blocks; larger blocks: four chunks of one block.
 // Key/value data moves in 64-token chunks: one 4-D TMA box {d, bw, 64/bw, 1} of the [U, nlat, nlon, d]
 // view lands as 64 rows x 128 B in 128-byte-swizzled shared memory, which is at once the K-major
-// operand layout for S = Q K^T and the MN-major operand layout for O += P V.
+// operand layout for S = Q K^T and the MN-major operand layout for O += P V.  A staged chunk serves
+// both tiles of the item.
 //
-// Warp roles (192 threads): warps 0-3 softmax (thread r owns query row r = TMEM lane r),
-// warp 4 builds the key list and issues TMA, warp 5 allocates TMEM and issues tcgen05.mma.
-// TMEM columns: [0,64) O accumulator, then SBUFS S buffers of 64 columns; P (bf16) overwrites the
-// first 32 columns of its S buffer and is consumed from TMEM as the A operand of P V.
-// Several CTAs are resident per SM, so one CTA's softmax overlaps another's tensor work.
+// The kernel is persistent: CTAs (two per SM) draw items from a counter in the workspace.
+// Warp roles (352 threads): warps 0-3 softmax of tile 0, warps 4-7 softmax of tile 1 (thread = query
+// row = TMEM lane), warp 8 builds key lists and issues TMA, warps 9 and 10 issue tcgen05.mma for tile 0
+// and tile 1.  Each tile is an independent chain  QK^T -> softmax -> PV  over its own TMEM columns
+// (O: 64 fp32 columns, S: 64 fp32 columns; P (bf16) overwrites the first 32 columns of S and is the
+// TMEM A operand of PV), so four such chains per SM keep the MUFU exponential pipe, the limiter at
+// d = 64, busy while any one of them waits for the tensor core.
 // Every mbarrier wait is bounded; on expiry the CTA records MOSAIC_E_DEVICE_TIMEOUT and drains.
 #include <cuda.h>
 #include <cuda_bf16.h>
-#include <stdlib.h>
 
 #include "common.cuh"
 
@@ -30,21 +34,34 @@ namespace mosaic {
 
 namespace {
 
-constexpr int kTile = 8192;                    // bytes of one 64 x 64 bf16 chunk
-constexpr uint32_t kColO = 0, kColS = 64;
+constexpr int kTile = 8192;                      // bytes of one 64 x 64 bf16 chunk
+constexpr int kStages = 4;                       // key/value ring depth (K + V chunk per stage)
+constexpr int kMaxUnion = 4 * kMaxList;          // most entries of an item's merged key list
+constexpr int kThreads = 352;
+constexpr uint32_t kTmemCols = 256;
+constexpr uint32_t kColO = 0, kColS = 128;       // O of tile t at 64 t, S of tile t at 128 + 64 t
 constexpr long long kSpinCycles = 4000000000ll;  // bound of a single wait (~2 s)
-constexpr float kRescaleThreshold = 8.0f;      // log2 units: P stays below 2^8
+constexpr float kRescaleThreshold = 8.0f;        // log2 units: P stays below 2^8
 
-template <int NST, int SBUFS>
-struct SmemTC {
-  unsigned char q[2 * kTile];
-  unsigned char kv[NST][2][kTile];
-  unsigned long long kv_full[NST], kv_empty[NST], q_full, s_full[SBUFS], p_full[SBUFS], pv_done[SBUFS];
+struct ItemInfo {
+  int n;        // entries of the merged list; -1 = no more work
+  int unit;     // (batch, head) unit
+  int hvalid;   // bit h: half h exists
+  int hb[4];    // query block of half h
+  int hc[4];    // 64-token chunk of that block
+};
+
+struct Smem {
+  unsigned char q[2][2 * kTile];           // [tile][128 rows x 128 B]
+  unsigned char kv[kStages][2][kTile];     // [stage][K, V]
+  unsigned long long kv_full[kStages], kv_empty[kStages];
+  unsigned long long q_full[2], q_empty[2], s_full[2], p_full[2], pv_done[2];
+  unsigned long long list_full[2], list_empty[2];
   uint32_t tmem_base;
   int abort;
-  int nlist;
-  int ids[2 * kMaxList];
-  unsigned char mask[2 * kMaxList];
+  ItemInfo info[2];
+  int ids[2][kMaxUnion];
+  unsigned char mask[2][kMaxUnion];
 };
 
 __device__ __forceinline__ uint32_t s32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -69,8 +86,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait.  Returns false after the limit (status recorded) or once another thread aborted.
 // The clock and the abort flag are looked at only every 64 polls to keep the poll loop light.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort, int* status) {
-  if (mbar_try_wait(bar, parity)) return true;
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort, int* status) {
   const long long t0 = clock64();
 #pragma unroll 1
   for (uint32_t i = 1;; ++i) {
@@ -84,6 +100,10 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       }
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort, int* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort, status);
 }
 
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
@@ -120,37 +140,36 @@ __device__ __forceinline__ void umma_ts(uint32_t d, uint32_t a, uint64_t b, uint
       : "memory");
 }
 
-#define MOSAIC_R32(r, o)                                                                                         \
-  "=r"(r[o + 0]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]), "=r"(r[o + 6]), \
-      "=r"(r[o + 7]), "=r"(r[o + 8]), "=r"(r[o + 9]), "=r"(r[o + 10]), "=r"(r[o + 11]), "=r"(r[o + 12]),          \
-      "=r"(r[o + 13]), "=r"(r[o + 14]), "=r"(r[o + 15]), "=r"(r[o + 16]), "=r"(r[o + 17]), "=r"(r[o + 18]),       \
-      "=r"(r[o + 19]), "=r"(r[o + 20]), "=r"(r[o + 21]), "=r"(r[o + 22]), "=r"(r[o + 23]), "=r"(r[o + 24]),       \
-      "=r"(r[o + 25]), "=r"(r[o + 26]), "=r"(r[o + 27]), "=r"(r[o + 28]), "=r"(r[o + 29]), "=r"(r[o + 30]),       \
-      "=r"(r[o + 31])
-#define MOSAIC_W32(r, o)                                                                                      \
-  "r"(r[o + 0]), "r"(r[o + 1]), "r"(r[o + 2]), "r"(r[o + 3]), "r"(r[o + 4]), "r"(r[o + 5]), "r"(r[o + 6]),     \
-      "r"(r[o + 7]), "r"(r[o + 8]), "r"(r[o + 9]), "r"(r[o + 10]), "r"(r[o + 11]), "r"(r[o + 12]),             \
-      "r"(r[o + 13]), "r"(r[o + 14]), "r"(r[o + 15]), "r"(r[o + 16]), "r"(r[o + 17]), "r"(r[o + 18]),          \
-      "r"(r[o + 19]), "r"(r[o + 20]), "r"(r[o + 21]), "r"(r[o + 22]), "r"(r[o + 23]), "r"(r[o + 24]),          \
-      "r"(r[o + 25]), "r"(r[o + 26]), "r"(r[o + 27]), "r"(r[o + 28]), "r"(r[o + 29]), "r"(r[o + 30]),          \
-      "r"(r[o + 31])
+#define MOSAIC_R16(r, o)                                                                                          \
+  "=r"(r[o + 0]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]), "=r"(r[o + 6]),  \
+      "=r"(r[o + 7]), "=r"(r[o + 8]), "=r"(r[o + 9]), "=r"(r[o + 10]), "=r"(r[o + 11]), "=r"(r[o + 12]),           \
+      "=r"(r[o + 13]), "=r"(r[o + 14]), "=r"(r[o + 15])
+#define MOSAIC_W16(r, o)                                                                                     \
+  "r"(r[o + 0]), "r"(r[o + 1]), "r"(r[o + 2]), "r"(r[o + 3]), "r"(r[o + 4]), "r"(r[o + 5]), "r"(r[o + 6]),    \
+      "r"(r[o + 7]), "r"(r[o + 8]), "r"(r[o + 9]), "r"(r[o + 10]), "r"(r[o + 11]), "r"(r[o + 12]),            \
+      "r"(r[o + 13]), "r"(r[o + 14]), "r"(r[o + 15])
 
-// 32 consecutive 32-bit TMEM columns of this thread's lane -> registers r[o .. o+31]
-template <int O, int N>
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[N]) {
+// 32 consecutive 32-bit TMEM columns of this thread's lane -> registers r[0..31]
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, "
       "%15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : MOSAIC_R32(r, O)
+      : MOSAIC_R16(r, 0), MOSAIC_R16(r, 16)
       : "r"(taddr)
       : "memory");
 }
-template <int O, int N>
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[N]) {
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, "
       "%15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
-      MOSAIC_W32(r, O)
+      MOSAIC_W16(r, 0), MOSAIC_W16(r, 16)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, "
+      "%15, %16};" ::"r"(taddr),
+      MOSAIC_W16(r, 0)
       : "memory");
 }
 
@@ -158,6 +177,11 @@ __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
 }
 
 // two fp32 lanes in one 64-bit register (packed fp32 arithmetic of this architecture)
@@ -184,6 +208,11 @@ __device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
   asm("mul.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
 }
+__device__ __forceinline__ uint32_t bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
 
 // Shared-memory operand descriptor: 128-byte swizzle, 8-row groups 1024 B apart.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
@@ -200,10 +229,62 @@ __host__ __device__ constexpr uint32_t make_idesc(bool b_mn_major) {
          ((128u >> 4) << 24);
 }
 
-}  // namespace
+// The four halves of work item `it` (index inside the unit).  Missing halves repeat half 0 (their rows
+// are computed with every key masked and never stored).  Returns the bit set of existing halves.
+__device__ __forceinline__ int item_halves(const Geo& g, int it, int (&hb)[4], int (&hc)[4]) {
+  int valid = 0;
+  if (g.cpb == 1) {
+    const int ntx = (g.nbw + 1) >> 1, n_main = (g.nbh >> 1) * ntx;
+    if (it < n_main) {  // 2 x 2 group
+      const int gy = it / ntx, tx = it - gy * ntx;
+#pragma unroll
+      for (int h = 0; h < 4; ++h) {
+        const int by = 2 * gy + (h >> 1), bx = 2 * tx + (h & 1);
+        hb[h] = by * g.nbw + bx;
+        hc[h] = 0;
+        valid |= (bx < g.nbw) << h;
+      }
+    } else {            // odd last block row: 1 x 4 group
+      const int bx0 = 4 * (it - n_main);
+#pragma unroll
+      for (int h = 0; h < 4; ++h) {
+        hb[h] = (g.nbh - 1) * g.nbw + bx0 + h;
+        hc[h] = 0;
+        valid |= (bx0 + h < g.nbw) << h;
+      }
+    }
+  } else if (g.cpb == 2) {  // two neighbouring 128-token blocks
+    const int ntx = (g.nbw + 1) >> 1, by = it / ntx, tx = it - by * ntx;
+#pragma unroll
+    for (int h = 0; h < 4; ++h) {
+      const int bx = 2 * tx + (h >> 1);
+      hb[h] = by * g.nbw + bx;
+      hc[h] = h & 1;
+      valid |= (bx < g.nbw) << h;
+    }
+  } else {                  // four chunks of one block
+    const int ipb = (g.cpb + 3) >> 2, blk = it / ipb, c0 = 4 * (it - blk * ipb);
+#pragma unroll
+    for (int h = 0; h < 4; ++h) {
+      hb[h] = blk;
+      hc[h] = c0 + h;
+      valid |= (c0 + h < g.cpb) << h;
+    }
+  }
+#pragma unroll
+  for (int h = 1; h < 4; ++h)
+    if (!((valid >> h) & 1)) { hb[h] = hb[0]; hc[h] = hc[0]; }
+  return valid;
+}
 
-// Warp-cooperative attended list of query block i (local set, then valid selected ids), appended to
-// ids[n0..); returns the new count.  Same order as attended_list().
+__host__ __device__ inline int items_per_unit(const Geo& g) {
+  if (g.cpb == 1) return (g.nbh >> 1) * ((g.nbw + 1) >> 1) + (g.nbh & 1) * ((g.nbw + 3) >> 2);
+  if (g.cpb == 2) return g.nbh * ((g.nbw + 1) >> 1);
+  return g.m * ((g.cpb + 3) >> 2);
+}
+
+// Warp-cooperative attended list of query block i (local set, then valid selected ids) written to
+// ids[n0..); returns the new count.
 __device__ __forceinline__ int warp_attended(const Geo& g, const int32_t* __restrict__ idx_row, int i, int* ids,
                                              int n0, int lane, int* status) {
   const int by = i / g.nbw, bx = i - by * g.nbw;
@@ -228,294 +309,384 @@ __device__ __forceinline__ int warp_attended(const Geo& g, const int32_t* __rest
   return n + __popc(sm_);
 }
 
-template <int NST, int SBUFS, int MINB>
-__global__ void __launch_bounds__(192, MINB)
+// Merge the attended list of query block `blk` into the item's list (ids/mask, n entries so far):
+// entries already present get `bits` OR-ed into their mask, new ones are appended.  Returns the new n.
+__device__ __forceinline__ int merge_block(const Geo& g, const int32_t* __restrict__ block_idx, int u, int blk,
+                                           unsigned char bits, int* ids, unsigned char* mask, int n, int lane,
+                                           int* status) {
+  const int32_t* row = block_idx + ((long long)u * g.m + blk) * g.topk;
+  const int n0 = n;
+  const int nb = warp_attended(g, row, blk, ids, n0, lane, status) - n0;  // staged behind the list
+  __syncwarp();
+  if (n0 == 0) {
+    for (int e = lane; e < nb; e += 32) mask[e] = bits;
+    __syncwarp();
+    return nb;
+  }
+  int mine[2], pos[2];  // at most 64 entries per block: two per lane
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    const int e = lane + 32 * r;
+    mine[r] = e < nb ? ids[n0 + e] : -1;
+    pos[r] = -1;
+  }
+  for (int a = 0; a < n0; ++a) {
+    const int id = ids[a];
+    pos[0] = id == mine[0] ? a : pos[0];
+    pos[1] = id == mine[1] ? a : pos[1];
+  }
+  __syncwarp();
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    const bool have = mine[r] >= 0, fresh = have && pos[r] < 0;
+    if (have && pos[r] >= 0) mask[pos[r]] |= bits;
+    const unsigned fm = __ballot_sync(0xffffffffu, fresh);
+    if (fresh) {
+      const int at = n + __popc(fm & ((1u << lane) - 1u));
+      ids[at] = mine[r];
+      mask[at] = bits;
+    }
+    n += __popc(fm);
+    __syncwarp();
+  }
+  return n;
+}
+
+}  // namespace
+
+__global__ void __launch_bounds__(kThreads, 2)
     fwd_tc_kernel(const Geo g, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_v, const int32_t* __restrict__ block_idx,
-                  __nv_bfloat16* __restrict__ o, float* __restrict__ lse, int* status, int tiles_per_unit) {
-  using Smem = SmemTC<NST, SBUFS>;
-  constexpr uint32_t kTmemCols = SBUFS == 1 ? 128 : 256;
+                  __nv_bfloat16* __restrict__ o, float* __restrict__ lse, int* status, int* work_counter,
+                  int ipu, int total_items) {
   extern __shared__ unsigned char smem_raw[];
   Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int u = blockIdx.x / tiles_per_unit, t = blockIdx.x - u * tiles_per_unit;
-
-  // the two 64-row halves of the tile: (block, chunk) each
-  int hb0, hb1, hc0, hc1;
-  bool hvalid1 = true;
-  if (g.cpb == 1) {
-    hb0 = 2 * t; hb1 = 2 * t + 1; hc0 = hc1 = 0;
-    if (hb1 >= g.m) { hvalid1 = false; hb1 = hb0; }
-  } else {
-    const int hpb = g.cpb / 2;  // tiles per block
-    hb0 = hb1 = t / hpb;
-    hc0 = 2 * (t % hpb); hc1 = hc0 + 1;
-  }
 
   if (tid == 0) {
-    for (int s = 0; s < NST; ++s) { mbar_init(s32(&sm.kv_full[s]), 1); mbar_init(s32(&sm.kv_empty[s]), 1); }
-    mbar_init(s32(&sm.q_full), 1);
-    for (int s = 0; s < SBUFS; ++s) {
-      mbar_init(s32(&sm.s_full[s]), 1);
-      mbar_init(s32(&sm.p_full[s]), 128);
-      mbar_init(s32(&sm.pv_done[s]), 1);
+    for (int s = 0; s < kStages; ++s) { mbar_init(s32(&sm.kv_full[s]), 1); mbar_init(s32(&sm.kv_empty[s]), 2); }
+    for (int t = 0; t < 2; ++t) {
+      mbar_init(s32(&sm.q_full[t]), 1);
+      mbar_init(s32(&sm.q_empty[t]), 1);
+      mbar_init(s32(&sm.s_full[t]), 1);
+      mbar_init(s32(&sm.p_full[t]), 128);
+      mbar_init(s32(&sm.pv_done[t]), 1);
+      mbar_init(s32(&sm.list_full[t]), 1);
+      mbar_init(s32(&sm.list_empty[t]), 10);  // 8 softmax warps + 2 MMA warps
     }
     sm.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   __syncthreads();
-  if (warp == 5) {
+  if (warp == 9) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(&sm.tmem_base)),
                  "r"(kTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  if (warp == 4) {
-    if (lane == 0) {  // the query tile does not depend on the key list: start it first
-      mbar_expect_tx(s32(&sm.q_full), 2 * kTile);
-      int by = hb0 / g.nbw, bx = hb0 - by * g.nbw;
-      tma_load_4d(s32(sm.q), &map_q, s32(&sm.q_full), 0, bx * g.bw, by * g.bh + hc0 * g.crows, u);
-      by = hb1 / g.nbw; bx = hb1 - by * g.nbw;
-      tma_load_4d(s32(sm.q + kTile), &map_q, s32(&sm.q_full), 0, bx * g.bw, by * g.bh + hc1 * g.crows, u);
-    }
-    // key list: entries of the first half's block, then what only the second half adds
-    const int32_t* row0 = block_idx + ((long long)u * g.m + hb0) * g.topk;
-    int n = warp_attended(g, row0, hb0, sm.ids, 0, lane, status);
-    __syncwarp();
-    const unsigned char m0 = g.cpb == 1 ? 1 : 3;
-    for (int e = lane; e < n; e += 32) sm.mask[e] = m0;
-    if (g.cpb == 1 && hvalid1) {
-      const int32_t* row1 = block_idx + ((long long)u * g.m + hb1) * g.topk;
-      const int n0 = n;
-      const int n1 = warp_attended(g, row1, hb1, sm.ids, n0, lane, status) - n0;  // staged behind list 0
-      __syncwarp();
-      // entries of list 1 (at most 2 per lane): shared with list 0 -> mark, else keep (compacted)
-      int mine[2], pos[2];
-#pragma unroll
-      for (int r = 0; r < 2; ++r) {
-        const int e = lane + 32 * r;
-        mine[r] = e < n1 ? sm.ids[n0 + e] : -1;
-        pos[r] = -1;
-      }
-      for (int a = 0; a < n0; ++a) {
-        const int id = sm.ids[a];
-        pos[0] = id == mine[0] ? a : pos[0];
-        pos[1] = id == mine[1] ? a : pos[1];
-      }
-      __syncwarp();
-#pragma unroll
-      for (int r = 0; r < 2; ++r) {
-        const bool have = mine[r] >= 0, fresh = have && pos[r] < 0;
-        if (have && pos[r] >= 0) sm.mask[pos[r]] |= 2;
-        const unsigned fm = __ballot_sync(0xffffffffu, fresh);
-        if (fresh) {
-          const int at = n + __popc(fm & ((1u << lane) - 1u));
-          sm.ids[at] = mine[r];
-          sm.mask[at] = 2;
-        }
-        n += __popc(fm);
-        __syncwarp();
-      }
-    }
-    if (lane == 0) sm.nlist = n;
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
 
   const uint32_t tmem = sm.tmem_base;
-  const int nch = sm.nlist * g.cpb;
   volatile int* abort = &sm.abort;
 
-  if (warp == 4) {
-    // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      for (int it = 0; it < nch; ++it) {
-        const int st = it % NST, j = sm.ids[it / g.cpb], c = it % g.cpb;
-        if (!mbar_wait(s32(&sm.kv_empty[st]), ((it / NST) & 1) ^ 1, abort, status)) break;
-        const int by = j / g.nbw, bx = j - by * g.nbw;
-        mbar_expect_tx(s32(&sm.kv_full[st]), 2 * kTile);
-        tma_load_4d(s32(sm.kv[st][0]), &map_k, s32(&sm.kv_full[st]), 0, bx * g.bw, by * g.bh + c * g.crows, u);
-        tma_load_4d(s32(sm.kv[st][1]), &map_v, s32(&sm.kv_full[st]), 0, bx * g.bw, by * g.bh + c * g.crows, u);
+  if (warp == 8) {
+    // ------------------------------------------------------------- key lists + TMA producer
+    long long step = 0;  // key/value chunks issued so far (ring position)
+    for (int it = 0;; ++it) {
+      const int buf = it & 1;
+      int item = 0;
+      if (lane == 0) item = atomicAdd(work_counter, 1);
+      item = __shfl_sync(0xffffffffu, item, 0);
+      bool ok = true;
+      if (lane == 0) ok = mbar_wait(s32(&sm.list_empty[buf]), ((it >> 1) & 1) ^ 1, abort, status);
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      if (item >= total_items) {
+        if (lane == 0) { sm.info[buf].n = -1; mbar_arrive(s32(&sm.list_full[buf])); }
+        break;
       }
+      const int u = item / ipu;
+      int hb[4], hc[4];
+      const int valid = item_halves(g, item - u * ipu, hb, hc);
+      int n = 0;
+#pragma unroll
+      for (int h = 0; h < 4; ++h) {
+        if (!((valid >> h) & 1)) continue;
+        bool first = true;  // first half of its block: merge the block's list once, for all its halves
+        unsigned char bits = 0;
+#pragma unroll
+        for (int h2 = 0; h2 < 4; ++h2) {
+          if (((valid >> h2) & 1) && hb[h2] == hb[h]) {
+            if (h2 < h) first = false;
+            bits |= (unsigned char)(1 << h2);
+          }
+        }
+        if (first) n = merge_block(g, block_idx, u, hb[h], bits, sm.ids[buf], sm.mask[buf], n, lane, status);
+      }
+      if (lane == 0) {
+        ItemInfo& inf = sm.info[buf];
+        inf.n = n; inf.unit = u; inf.hvalid = valid;
+#pragma unroll
+        for (int h = 0; h < 4; ++h) { inf.hb[h] = hb[h]; inf.hc[h] = hc[h]; }
+      }
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(s32(&sm.list_full[buf]));
+        // query tiles: free once the tile's last QK^T of the previous item has completed
+        for (int t = 0; t < 2 && ok; ++t) {
+          ok = mbar_wait(s32(&sm.q_empty[t]), (it & 1) ^ 1, abort, status);
+          if (!ok) break;
+          mbar_expect_tx(s32(&sm.q_full[t]), 2 * kTile);
+          for (int hh = 0; hh < 2; ++hh) {
+            const int h = 2 * t + hh, by = hb[h] / g.nbw, bx = hb[h] - by * g.nbw;
+            tma_load_4d(s32(sm.q[t] + hh * kTile), &map_q, s32(&sm.q_full[t]), 0, bx * g.bw,
+                        by * g.bh + hc[h] * g.crows, u);
+          }
+        }
+        for (int e = 0; e < n && ok; ++e) {
+          const int j = sm.ids[buf][e], by = j / g.nbw, bx = j - by * g.nbw;
+          for (int c = 0; c < g.cpb; ++c, ++step) {
+            const int st = (int)(step % kStages);
+            ok = mbar_wait(s32(&sm.kv_empty[st]), (uint32_t)((step / kStages) & 1) ^ 1, abort, status);
+            if (!ok) break;
+            mbar_expect_tx(s32(&sm.kv_full[st]), 2 * kTile);
+            tma_load_4d(s32(sm.kv[st][0]), &map_k, s32(&sm.kv_full[st]), 0, bx * g.bw, by * g.bh + c * g.crows, u);
+            tma_load_4d(s32(sm.kv[st][1]), &map_v, s32(&sm.kv_full[st]), 0, bx * g.bw, by * g.bh + c * g.crows, u);
+          }
+        }
+      }
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+    }
+    if (lane == 0) {
       if (*abort) {  // give copies in flight time to land before the CTA's memory is released
         const long long t0 = clock64();
         while (clock64() - t0 < 400000) {}
+      } else {       // drain: the last uses of every ring stage have been released by both tiles
+        const long long first = step > kStages ? step - kStages : 0;
+        for (long long s = first; s < step; ++s)
+          if (!mbar_wait(s32(&sm.kv_empty[s % kStages]), (uint32_t)((s / kStages) & 1), abort, status)) break;
       }
     }
-  } else if (warp == 5) {
-    // ------------------------------------------------------------------ MMA issuer
+  } else if (warp == 9 || warp == 10) {
+    // ------------------------------------------------------------- MMA issuer of tile t
+    const int t = warp - 9;
     if (lane == 0) {
       constexpr uint32_t idesc_qk = make_idesc(false), idesc_pv = make_idesc(true);
-      const uint64_t qdesc = smem_desc(s32(sm.q));
-      bool ok = mbar_wait(s32(&sm.q_full), 0, abort, status);
-      auto issue_qk = [&](int it) {
-        const uint64_t kdesc = smem_desc(s32(sm.kv[it % NST][0]));
-        const uint32_t d = tmem + kColS + (it % SBUFS) * 64;
-#pragma unroll
-        for (int kk = 0; kk < 4; ++kk) umma_ss(d, qdesc + 2 * kk, kdesc + 2 * kk, idesc_qk, kk > 0);
-        tc_commit(s32(&sm.s_full[it % SBUFS]));
-      };
-      // S buffer of iteration `it` is free once P V of iteration it - SBUFS has completed
-      auto wait_sbuf = [&](int it) {
-        const int prev = it - SBUFS;
-        return prev < 0 || mbar_wait(s32(&sm.pv_done[prev % SBUFS]), (prev / SBUFS) & 1, abort, status);
-      };
-      if (ok && nch > 0) {
-        ok = mbar_wait(s32(&sm.kv_full[0]), 0, abort, status);
-        if (ok) { tc_fence_after(); issue_qk(0); }
-      }
-      for (int it = 0; ok && it < nch; ++it) {
-        if (SBUFS > 1 && it + 1 < nch) {
-          ok = mbar_wait(s32(&sm.kv_full[(it + 1) % NST]), ((it + 1) / NST) & 1, abort, status) && wait_sbuf(it + 1);
-          if (!ok) break;
-          tc_fence_after();
-          issue_qk(it + 1);
-        }
-        ok = mbar_wait(s32(&sm.p_full[it % SBUFS]), (it / SBUFS) & 1, abort, status);
+      const uint64_t qdesc = smem_desc(s32(sm.q[t]));
+      const uint32_t tcol_o = tmem + kColO + 64 * t, tcol_s = tmem + kColS + 64 * t;
+      const uint32_t tbits = 3u << (2 * t);
+      long long step = 0;   // ring position (all chunks, attended by this tile or not)
+      uint32_t nt = 0;      // products issued by this tile so far (phase of s_full/p_full/pv_done)
+      bool ok = true;
+      for (int it = 0; ok; ++it) {
+        const int buf = it & 1;
+        ok = mbar_wait(s32(&sm.list_full[buf]), (it >> 1) & 1, abort, status);
         if (!ok) break;
-        tc_fence_after();
-        const uint64_t vdesc = smem_desc(s32(sm.kv[it % NST][1]));
-        const uint32_t p = tmem + kColS + (it % SBUFS) * 64;
+        const int n = sm.info[buf].n;
+        if (n < 0) break;
+        int last = -1;
+        for (int e = 0; e < n; ++e)
+          if (sm.mask[buf][e] & tbits) last = e;
+        // the query tile is loaded for every item; it must have landed before its buffer is handed back
+        ok = mbar_wait(s32(&sm.q_full[t]), it & 1, abort, status);
+        if (!ok) break;
+        if (last < 0) mbar_arrive(s32(&sm.q_empty[t]));
+        bool first = true;
+        for (int e = 0; e < n && ok; ++e) {
+          const bool act = (sm.mask[buf][e] & tbits) != 0;
+          for (int c = 0; c < g.cpb; ++c, ++step) {
+            const int st = (int)(step % kStages);
+            ok = mbar_wait(s32(&sm.kv_full[st]), (uint32_t)((step / kStages) & 1), abort, status);
+            if (!ok) break;
+            if (!act) { mbar_arrive(s32(&sm.kv_empty[st])); continue; }
+            // S (aliased by P) is free once the previous P V of this tile has completed
+            if (nt > 0) {
+              ok = mbar_wait(s32(&sm.pv_done[t]), (nt - 1) & 1, abort, status);
+              if (!ok) break;
+            }
+            tc_fence_after();
+            const uint64_t kdesc = smem_desc(s32(sm.kv[st][0]));
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk)
-          umma_ts(tmem + kColO, p + 8 * kk, vdesc + (uint64_t)((2048 * kk) >> 4), idesc_pv, (it > 0 || kk > 0));
-        tc_commit(s32(&sm.kv_empty[it % NST]));
-        tc_commit(s32(&sm.pv_done[it % SBUFS]));
-        if (SBUFS == 1 && it + 1 < nch) {
-          ok = mbar_wait(s32(&sm.kv_full[(it + 1) % NST]), ((it + 1) / NST) & 1, abort, status) && wait_sbuf(it + 1);
-          if (!ok) break;
-          tc_fence_after();
-          issue_qk(it + 1);
+            for (int kk = 0; kk < 4; ++kk) umma_ss(tcol_s, qdesc + 2 * kk, kdesc + 2 * kk, idesc_qk, kk > 0);
+            tc_commit(s32(&sm.s_full[t]));
+            if (e == last && c == g.cpb - 1) tc_commit(s32(&sm.q_empty[t]));
+            ok = mbar_wait(s32(&sm.p_full[t]), nt & 1, abort, status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint64_t vdesc = smem_desc(s32(sm.kv[st][1]));
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+              umma_ts(tcol_o, tcol_s + 8 * kk, vdesc + (uint64_t)((2048 * kk) >> 4), idesc_pv, (!first || kk > 0));
+            tc_commit(s32(&sm.kv_empty[st]));
+            tc_commit(s32(&sm.pv_done[t]));
+            first = false;
+            ++nt;
+          }
         }
+        if (ok) mbar_arrive(s32(&sm.list_empty[buf]));
       }
     }
   } else {
-    // ------------------------------------------------------------------ softmax, then epilogue
-    const int h = warp >> 1;  // which 64-row half this warp's rows belong to
-    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    // ------------------------------------------------------------- softmax of tile t, then epilogue
+    const int t = warp >> 2;        // tile
+    const int hh = (warp >> 1) & 1; // 64-row half of the tile this warp's rows belong to
+    const int h = 2 * t + hh;
+    const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t ts = tmem + lane_off + kColS + 64 * t, to = tmem + lane_off + kColO + 64 * t;
+    const uint32_t tbits = 3u << (2 * t), hbit = 1u << h;
     const uint64_t scale2 = pack2(g.scale_log2, g.scale_log2);
-    float m_ref = -INFINITY, l = 0.f;
+    uint32_t nt = 0;
     bool ok = true;
-    for (int it = 0; it < nch; ++it) {
-      const int sb = it % SBUFS;
-      ok = mbar_wait(s32(&sm.s_full[sb]), (it / SBUFS) & 1, abort, status);
+    for (int it = 0; ok; ++it) {
+      const int buf = it & 1;
+      ok = mbar_wait(s32(&sm.list_full[buf]), (it >> 1) & 1, abort, status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
-      tc_fence_after();
-      const bool attends = (sm.mask[it / g.cpb] >> h) & 1;
-      const uint32_t ts = tmem + lane_off + kColS + sb * 64;
-      bool need = false;
-      float alpha = 1.f;
-      uint32_t pk[32];
-      if (attends) {
-        uint32_t sr[64];
-        tmem_ld32<0>(ts, sr);
-        tmem_ld32<32>(ts + 32, sr);
-        tmem_wait_ld();
-        float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]), mx2 = __uint_as_float(sr[2]),
-              mx3 = __uint_as_float(sr[3]);
-#pragma unroll
-        for (int c = 4; c < 64; c += 4) {
-          mx0 = fmaxf(mx0, __uint_as_float(sr[c]));
-          mx1 = fmaxf(mx1, __uint_as_float(sr[c + 1]));
-          mx2 = fmaxf(mx2, __uint_as_float(sr[c + 2]));
-          mx3 = fmaxf(mx3, __uint_as_float(sr[c + 3]));
-        }
-        const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * g.scale_log2;  // scale > 0 commutes with max
-        if (m_ref == -INFINITY) {
-          m_ref = mx;
-        } else if (mx > m_ref + kRescaleThreshold) {
-          need = true;
-          alpha = ex2(m_ref - mx);
-          m_ref = mx;
-          l *= alpha;
-        }
-        const uint64_t negm2 = pack2(-m_ref, -m_ref);
-        uint64_t sum_a = pack2(0.f, 0.f), sum_b = sum_a;
-#pragma unroll
-        for (int c = 0; c < 64; c += 4) {
-          float x0, x1, x2, x3;
-          unpack2(fma2(pack2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), scale2, negm2), x0, x1);
-          unpack2(fma2(pack2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), scale2, negm2), x2, x3);
-          const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
-          sum_a = add2(sum_a, pack2(p0, p1));
-          sum_b = add2(sum_b, pack2(p2, p3));
-          __nv_bfloat162 pa = __floats2bfloat162_rn(p0, p1), pb = __floats2bfloat162_rn(p2, p3);
-          pk[c >> 1] = *reinterpret_cast<uint32_t*>(&pa);
-          pk[(c >> 1) + 1] = *reinterpret_cast<uint32_t*>(&pb);
-        }
-        float s0, s1;
-        unpack2(add2(sum_a, sum_b), s0, s1);
-        l += s0 + s1;
-      } else {
-#pragma unroll
-        for (int c = 0; c < 32; ++c) pk[c] = 0u;
-      }
-      tmem_st32<0>(ts, pk);
-      if (__any_sync(0xffffffffu, need)) {
-        // the accumulator may only be touched between P V products
-        if (it > 0) {
-          ok = mbar_wait(s32(&sm.pv_done[(it - 1) % SBUFS]), ((it - 1) / SBUFS) & 1, abort, status);
+      const int n = sm.info[buf].n;
+      if (n < 0) break;
+      float m_ref = -INFINITY, l = 0.f;
+      uint32_t done = 0;
+      for (int e = 0; e < n && ok; ++e) {
+        const uint32_t mk = sm.mask[buf][e];
+        if (!(mk & tbits)) continue;
+        const bool attends = (mk & hbit) != 0;
+        for (int c = 0; c < g.cpb; ++c) {
+          ok = mbar_wait(s32(&sm.s_full[t]), nt & 1, abort, status);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
-        }
-        const uint32_t to = tmem + lane_off + kColO;
-        const uint64_t alpha2 = pack2(alpha, alpha);
+          if (attends) {
+            uint32_t sa[32], sb[32];
+            tmem_ld32(ts, sa);
+            tmem_wait_ld();
+            float mx0 = __uint_as_float(sa[0]), mx1 = __uint_as_float(sa[1]);
 #pragma unroll
-        for (int part = 0; part < 2; ++part) {
-          uint32_t ov[32];
-          tmem_ld32<0>(to + 32 * part, ov);
-          tmem_wait_ld();
+            for (int i = 2; i < 32; i += 4) {
+              mx0 = max3(mx0, __uint_as_float(sa[i]), __uint_as_float(sa[i + 1]));
+              if (i + 3 < 32) mx1 = max3(mx1, __uint_as_float(sa[i + 2]), __uint_as_float(sa[i + 3]));
+            }
+            tmem_ld32(ts + 32, sb);
+            tmem_wait_ld();
 #pragma unroll
-          for (int c = 0; c < 32; c += 2) {
-            float a, b;
-            unpack2(mul2(pack2(__uint_as_float(ov[c]), __uint_as_float(ov[c + 1])), alpha2), a, b);
-            ov[c] = __float_as_uint(a);
-            ov[c + 1] = __float_as_uint(b);
+            for (int i = 0; i < 32; i += 4) {
+              mx0 = max3(mx0, __uint_as_float(sb[i]), __uint_as_float(sb[i + 1]));
+              mx1 = max3(mx1, __uint_as_float(sb[i + 2]), __uint_as_float(sb[i + 3]));
+            }
+            const float mx = fmaxf(mx0, mx1) * g.scale_log2;  // scale > 0 commutes with max
+            bool need = false;
+            float alpha = 1.f;
+            if (m_ref == -INFINITY) {
+              m_ref = mx;
+            } else if (mx > m_ref + kRescaleThreshold) {
+              need = true;
+              alpha = ex2(m_ref - mx);
+              m_ref = mx;
+              l *= alpha;
+            }
+            const uint64_t negm2 = pack2(-m_ref, -m_ref);
+            uint64_t sum_a = pack2(0.f, 0.f), sum_b = sum_a;
+            uint32_t pk[16];
+            // columns 32..63 first (they are in registers), then columns 0..31 again from TMEM
+#pragma unroll
+            for (int i = 0; i < 32; i += 4) {
+              float x0, x1, x2, x3;
+              unpack2(fma2(pack2(__uint_as_float(sb[i]), __uint_as_float(sb[i + 1])), scale2, negm2), x0, x1);
+              unpack2(fma2(pack2(__uint_as_float(sb[i + 2]), __uint_as_float(sb[i + 3])), scale2, negm2), x2, x3);
+              const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
+              sum_a = add2(sum_a, pack2(p0, p1));
+              sum_b = add2(sum_b, pack2(p2, p3));
+              pk[i >> 1] = bf16x2(p0, p1);
+              pk[(i >> 1) + 1] = bf16x2(p2, p3);
+            }
+            tmem_ld32(ts, sa);          // S columns 0..31 are still intact: P has not been written yet
+            tmem_wait_ld();
+            tmem_st16(ts + 16, pk);     // P columns 32..63 (bf16 pairs) = 32-bit columns 16..31
+#pragma unroll
+            for (int i = 0; i < 32; i += 4) {
+              float x0, x1, x2, x3;
+              unpack2(fma2(pack2(__uint_as_float(sa[i]), __uint_as_float(sa[i + 1])), scale2, negm2), x0, x1);
+              unpack2(fma2(pack2(__uint_as_float(sa[i + 2]), __uint_as_float(sa[i + 3])), scale2, negm2), x2, x3);
+              const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
+              sum_a = add2(sum_a, pack2(p0, p1));
+              sum_b = add2(sum_b, pack2(p2, p3));
+              pk[i >> 1] = bf16x2(p0, p1);
+              pk[(i >> 1) + 1] = bf16x2(p2, p3);
+            }
+            tmem_st16(ts, pk);
+            float s0, s1;
+            unpack2(add2(sum_a, sum_b), s0, s1);
+            l += s0 + s1;
+            if (__any_sync(0xffffffffu, need)) {
+              // the previous P V of this tile completed before this S was produced: O is at rest
+              const uint64_t alpha2 = pack2(alpha, alpha);
+#pragma unroll
+              for (int part = 0; part < 2; ++part) {
+                uint32_t ov[32];
+                tmem_ld32(to + 32 * part, ov);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) {
+                  float a, b;
+                  unpack2(mul2(pack2(__uint_as_float(ov[i]), __uint_as_float(ov[i + 1])), alpha2), a, b);
+                  ov[i] = __float_as_uint(a);
+                  ov[i + 1] = __float_as_uint(b);
+                }
+                tmem_st32(to + 32 * part, ov);
+              }
+            }
+          } else {
+            uint32_t z[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) z[i] = 0u;
+            tmem_st32(ts, z);
           }
-          tmem_st32<0>(to + 32 * part, ov);
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(s32(&sm.p_full[t]));
+          ++nt;
+          ++done;
         }
       }
-      tmem_wait_st();
+      if (!ok) break;
+      if (done > 0) {
+        ok = mbar_wait(s32(&sm.pv_done[t]), (nt - 1) & 1, abort, status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        if ((sm.info[buf].hvalid >> h) & 1) {
+          const int e = tid & 63;
+          const long long tok =
+              (long long)sm.info[buf].unit * g.N + chunk_token(g, sm.info[buf].hb[h], sm.info[buf].hc[h], e);
+          const float inv = 1.f / l;
+          uint4* dst = reinterpret_cast<uint4*>(o + tok * kD);
+#pragma unroll
+          for (int part = 0; part < 2; ++part) {
+            uint32_t ov[32];
+            tmem_ld32(to + 32 * part, ov);
+            tmem_wait_ld();
+            uint32_t w[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+              w[i] = bf16x2(__uint_as_float(ov[2 * i]) * inv, __uint_as_float(ov[2 * i + 1]) * inv);
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              dst[part * 4 + i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+          }
+          lse[tok] = (m_ref + log2f(l)) * 0.6931471805599453f;
+        }
+      }
       tc_fence_before();
-      mbar_arrive(s32(&sm.p_full[sb]));
-    }
-    if (ok && nch > 0) {
-      const int last = nch - 1;
-      ok = mbar_wait(s32(&sm.pv_done[last % SBUFS]), (last / SBUFS) & 1, abort, status);
-      ok = __all_sync(0xffffffffu, ok);
-    }
-    if (ok && nch > 0 && (h == 0 || hvalid1)) {
-      tc_fence_after();
-      const int e = tid & 63;
-      const long long tok = (long long)u * g.N + chunk_token(g, h ? hb1 : hb0, h ? hc1 : hc0, e);
-      const float inv = 1.f / l;
-      const uint32_t to = tmem + lane_off + kColO;
-      uint4* dst = reinterpret_cast<uint4*>(o + tok * kD);
-#pragma unroll
-      for (int part = 0; part < 2; ++part) {
-        uint32_t ov[32];
-        tmem_ld32<0>(to + 32 * part, ov);
-        tmem_wait_ld();
-        uint32_t w[16];
-#pragma unroll
-        for (int c = 0; c < 16; ++c) {
-          __nv_bfloat162 pb =
-              __floats2bfloat162_rn(__uint_as_float(ov[2 * c]) * inv, __uint_as_float(ov[2 * c + 1]) * inv);
-          w[c] = *reinterpret_cast<uint32_t*>(&pb);
-        }
-#pragma unroll
-        for (int c = 0; c < 4; ++c) dst[part * 4 + c] = make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
-      }
-      lse[tok] = (m_ref + log2f(l)) * 0.6931471805599453f;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(s32(&sm.list_empty[buf]));
     }
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 5) {
+  if (warp == 9) {
     tc_fence_after();
     __syncwarp();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
@@ -557,34 +728,26 @@ bool make_map(CUtensorMap* map, const void* base, const Geo& g) {
 
 }  // namespace
 
-template <int NST, int SBUFS, int MINB>
-int launch_variant(const HostCtx& c, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                   const int32_t* block_idx, void* o, float* lse) {
-  const Geo& g = c.g;
-  auto kern = fwd_tc_kernel<NST, SBUFS, MINB>;
-  const size_t smem = sizeof(SmemTC<NST, SBUFS>) + 1024;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-    return MOSAIC_E_CUDA;
-  const int tiles_per_unit = g.cpb == 1 ? (g.m + 1) / 2 : g.m * (g.cpb / 2);
-  const long long grid = (long long)g.U * tiles_per_unit;
-  kern<<<(unsigned)grid, 192, smem, c.stream>>>(g, mq, mk, mv, block_idx, (__nv_bfloat16*)o, lse, c.status,
-                                                tiles_per_unit);
-  return cudaGetLastError() == cudaSuccess ? MOSAIC_OK : MOSAIC_E_CUDA;
-}
-
 int launch_fwd_tc(const HostCtx& c, const void* q, const void* k, const void* v, const int32_t* block_idx, void* o,
                   float* lse) {
   const Geo& g = c.g;
-  if (!(g.cpb == 1 || g.cpb % 2 == 0)) return MOSAIC_E_UNSUPPORTED;
   CUtensorMap mq, mk, mv;
   if (!make_map(&mq, q, g) || !make_map(&mk, k, g) || !make_map(&mv, v, g)) return MOSAIC_E_CUDA;
-  const char* var = getenv("MOSAIC_BSA_FWD_VARIANT");  // tuning aid; default below
-  const int which = var ? atoi(var) : 0;
-  switch (which) {
-    case 1: return launch_variant<3, 1, 3>(c, mq, mk, mv, block_idx, o, lse);
-    case 2: return launch_variant<2, 1, 4>(c, mq, mk, mv, block_idx, o, lse);
-    default: return launch_variant<4, 2, 2>(c, mq, mk, mv, block_idx, o, lse);
-  }
+  const size_t smem = sizeof(Smem) + 1024;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return MOSAIC_E_CUDA;
+  if (cudaFuncSetAttribute(fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return MOSAIC_E_CUDA;
+  const int ipu = items_per_unit(g);
+  const long long total = (long long)g.U * ipu;
+  if (total > 0x7fffff00ll) return MOSAIC_E_UNSUPPORTED;
+  const long long grid = total < 2ll * sms ? total : 2ll * sms;
+  // the work counter is the second word of the status block, zeroed with it when the op starts
+  fwd_tc_kernel<<<(unsigned)grid, kThreads, smem, c.stream>>>(g, mq, mk, mv, block_idx, (__nv_bfloat16*)o, lse,
+                                                             c.status, c.status + 1, ipu, (int)total);
+  return cudaGetLastError() == cudaSuccess ? MOSAIC_OK : MOSAIC_E_CUDA;
 }
 
 }  // namespace mosaic

@@ -18,9 +18,9 @@
 // both tiles of the item.
 //
 // The kernel is persistent: CTAs (two per SM) draw items from a counter in the workspace.
-// Warp roles (352 threads): warps 0-3 softmax of tile 0, warps 4-7 softmax of tile 1 (thread = query
-// row = TMEM lane), warp 8 builds key lists and issues TMA, warps 9 and 10 issue tcgen05.mma for tile 0
-// and tile 1.  Each tile is an independent chain  QK^T -> softmax -> PV  over its own TMEM columns
+// Warp roles (384 threads): warps 0-3 softmax of tile 0, warps 4-7 softmax of tile 1 (thread = query
+// row = TMEM lane), warp 8 issues TMA, warps 9 and 10 issue tcgen05.mma for tile 0 and tile 1, warp 11
+// draws items from the queue and builds their key lists one item ahead.  Each tile is an independent chain  QK^T -> softmax -> PV  over its own TMEM columns
 // (O: 64 fp32 columns, S: 64 fp32 columns; P (bf16) overwrites the first 32 columns of S and is the
 // TMEM A operand of PV), so four such chains per SM keep the MUFU exponential pipe, the limiter at
 // d = 64, busy while any one of them waits for the tensor core.
@@ -37,7 +37,7 @@ namespace {
 constexpr int kTile = 8192;                      // bytes of one 64 x 64 bf16 chunk
 constexpr int kStages = 4;                       // key/value ring depth (K + V chunk per stage)
 constexpr int kMaxUnion = 4 * kMaxList;          // most entries of an item's merged key list
-constexpr int kThreads = 352;
+constexpr int kThreads = 384;
 constexpr uint32_t kTmemCols = 256;
 constexpr uint32_t kColO = 0, kColS = 128;       // O of tile t at 64 t, S of tile t at 128 + 64 t
 constexpr long long kSpinCycles = 4000000000ll;  // bound of a single wait (~2 s)
@@ -62,6 +62,8 @@ struct Smem {
   ItemInfo info[2];
   int ids[2][kMaxUnion];
   unsigned char mask[2][kMaxUnion];
+  int tmp_ids[kMaxUnion];            // planner scratch: merged list before reordering
+  unsigned char tmp_mask[kMaxUnion];
 };
 
 __device__ __forceinline__ uint32_t s32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -352,6 +354,60 @@ __device__ __forceinline__ int merge_block(const Geo& g, const int32_t* __restri
   return n;
 }
 
+// One lane of a converged warp (the same lane every time).
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+  return pred != 0;
+}
+
+// Reorder a merged key list so that both tiles find work all along it: entries only tile 0 attends
+// (class 0), entries both attend (1) and entries only tile 1 attends (2) are spread evenly, the k-th
+// entry of a class of n getting the fractional position (4k + class) / (4n).  The order of a softmax
+// sum does not matter to the result beyond rounding; the order is a function of the list alone.
+__device__ __forceinline__ void interleave_tiles(const int* sid, const unsigned char* smask, int n, int* did,
+                                                 unsigned char* dmask, int lane) {
+  int c0 = 0, c1 = 0, c2 = 0;
+  for (int e0 = 0; e0 < n; e0 += 32) {
+    const int e = e0 + lane;
+    const unsigned m = e < n ? smask[e] : 0u;
+    const int cls = e < n ? ((m & 3u) ? ((m & 12u) ? 1 : 0) : 2) : 3;
+    c0 += __popc(__ballot_sync(0xffffffffu, cls == 0));
+    c1 += __popc(__ballot_sync(0xffffffffu, cls == 1));
+    c2 += __popc(__ballot_sync(0xffffffffu, cls == 2));
+  }
+  int b0 = 0, b1 = 0, b2 = 0;
+  for (int e0 = 0; e0 < n; e0 += 32) {
+    const int e = e0 + lane;
+    const unsigned m = e < n ? smask[e] : 0u;
+    const int cls = e < n ? ((m & 3u) ? ((m & 12u) ? 1 : 0) : 2) : 3;
+    const unsigned m0 = __ballot_sync(0xffffffffu, cls == 0), m1 = __ballot_sync(0xffffffffu, cls == 1),
+                   m2 = __ballot_sync(0xffffffffu, cls == 2);
+    if (e < n) {
+      const unsigned lower = (1u << lane) - 1u;
+      const int k = cls == 0 ? b0 + __popc(m0 & lower) : cls == 1 ? b1 + __popc(m1 & lower) : b2 + __popc(m2 & lower);
+      const int nx = cls == 0 ? c0 : cls == 1 ? c1 : c2;
+      int pos = k;
+#pragma unroll
+      for (int y = 0; y < 3; ++y) {
+        if (y == cls) continue;
+        const int ny = y == 0 ? c0 : y == 1 ? c1 : c2;
+        const int T = (4 * k + cls) * ny;
+        for (int j = 0; j < ny; ++j) {
+          const int v = (4 * j + y) * nx;
+          pos += (v < T || (v == T && y < cls)) ? 1 : 0;
+        }
+      }
+      did[pos] = sid[e];
+      dmask[pos] = (unsigned char)m;
+    }
+    b0 += __popc(m0);
+    b1 += __popc(m1);
+    b2 += __popc(m2);
+  }
+  __syncwarp();
+}
+
 }  // namespace
 
 __global__ void __launch_bounds__(kThreads, 2)
@@ -372,7 +428,7 @@ __global__ void __launch_bounds__(kThreads, 2)
       mbar_init(s32(&sm.p_full[t]), 128);
       mbar_init(s32(&sm.pv_done[t]), 1);
       mbar_init(s32(&sm.list_full[t]), 1);
-      mbar_init(s32(&sm.list_empty[t]), 10);  // 8 softmax warps + 2 MMA warps
+      mbar_init(s32(&sm.list_empty[t]), 11);  // 8 softmax warps + 2 MMA warps + TMA producer
     }
     sm.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -392,9 +448,8 @@ __global__ void __launch_bounds__(kThreads, 2)
   const uint32_t tmem = sm.tmem_base;
   volatile int* abort = &sm.abort;
 
-  if (warp == 8) {
-    // ------------------------------------------------------------- key lists + TMA producer
-    long long step = 0;  // key/value chunks issued so far (ring position)
+  if (warp == 11) {
+    // ------------------------------------------------------------- planner: work queue + key lists
     for (int it = 0;; ++it) {
       const int buf = it & 1;
       int item = 0;
@@ -424,8 +479,9 @@ __global__ void __launch_bounds__(kThreads, 2)
             bits |= (unsigned char)(1 << h2);
           }
         }
-        if (first) n = merge_block(g, block_idx, u, hb[h], bits, sm.ids[buf], sm.mask[buf], n, lane, status);
+        if (first) n = merge_block(g, block_idx, u, hb[h], bits, sm.tmp_ids, sm.tmp_mask, n, lane, status);
       }
+      interleave_tiles(sm.tmp_ids, sm.tmp_mask, n, sm.ids[buf], sm.mask[buf], lane);
       if (lane == 0) {
         ItemInfo& inf = sm.info[buf];
         inf.n = n; inf.unit = u; inf.hvalid = valid;
@@ -433,17 +489,29 @@ __global__ void __launch_bounds__(kThreads, 2)
         for (int h = 0; h < 4; ++h) { inf.hb[h] = hb[h]; inf.hc[h] = hc[h]; }
       }
       __syncwarp();
-      if (lane == 0) {
-        mbar_arrive(s32(&sm.list_full[buf]));
+      if (lane == 0) mbar_arrive(s32(&sm.list_full[buf]));
+    }
+  } else if (warp == 8) {
+    // ------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      long long step = 0;  // key/value chunks issued so far (ring position)
+      bool ok = true;
+      for (int it = 0; ok; ++it) {
+        const int buf = it & 1;
+        ok = mbar_wait(s32(&sm.list_full[buf]), (it >> 1) & 1, abort, status);
+        if (!ok) break;
+        const ItemInfo& inf = sm.info[buf];
+        const int n = inf.n, u = inf.unit;
+        if (n < 0) break;
         // query tiles: free once the tile's last QK^T of the previous item has completed
         for (int t = 0; t < 2 && ok; ++t) {
           ok = mbar_wait(s32(&sm.q_empty[t]), (it & 1) ^ 1, abort, status);
           if (!ok) break;
           mbar_expect_tx(s32(&sm.q_full[t]), 2 * kTile);
           for (int hh = 0; hh < 2; ++hh) {
-            const int h = 2 * t + hh, by = hb[h] / g.nbw, bx = hb[h] - by * g.nbw;
+            const int h = 2 * t + hh, by = inf.hb[h] / g.nbw, bx = inf.hb[h] - by * g.nbw;
             tma_load_4d(s32(sm.q[t] + hh * kTile), &map_q, s32(&sm.q_full[t]), 0, bx * g.bw,
-                        by * g.bh + hc[h] * g.crows, u);
+                        by * g.bh + inf.hc[h] * g.crows, u);
           }
         }
         for (int e = 0; e < n && ok; ++e) {
@@ -457,11 +525,8 @@ __global__ void __launch_bounds__(kThreads, 2)
             tma_load_4d(s32(sm.kv[st][1]), &map_v, s32(&sm.kv_full[st]), 0, bx * g.bw, by * g.bh + c * g.crows, u);
           }
         }
+        if (ok) mbar_arrive(s32(&sm.list_empty[buf]));
       }
-      ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (!ok) break;
-    }
-    if (lane == 0) {
       if (*abort) {  // give copies in flight time to land before the CTA's memory is released
         const long long t0 = clock64();
         while (clock64() - t0 < 400000) {}
@@ -473,62 +538,72 @@ __global__ void __launch_bounds__(kThreads, 2)
     }
   } else if (warp == 9 || warp == 10) {
     // ------------------------------------------------------------- MMA issuer of tile t
+    // The whole warp walks the loop (waits are cheap polls); one elected lane issues the tensor-core
+    // instructions, so operands that are the same for the warp stay in uniform registers.
     const int t = warp - 9;
-    if (lane == 0) {
-      constexpr uint32_t idesc_qk = make_idesc(false), idesc_pv = make_idesc(true);
-      const uint64_t qdesc = smem_desc(s32(sm.q[t]));
-      const uint32_t tcol_o = tmem + kColO + 64 * t, tcol_s = tmem + kColS + 64 * t;
-      const uint32_t tbits = 3u << (2 * t);
-      long long step = 0;   // ring position (all chunks, attended by this tile or not)
-      uint32_t nt = 0;      // products issued by this tile so far (phase of s_full/p_full/pv_done)
-      bool ok = true;
-      for (int it = 0; ok; ++it) {
-        const int buf = it & 1;
-        ok = mbar_wait(s32(&sm.list_full[buf]), (it >> 1) & 1, abort, status);
-        if (!ok) break;
-        const int n = sm.info[buf].n;
-        if (n < 0) break;
-        int last = -1;
-        for (int e = 0; e < n; ++e)
-          if (sm.mask[buf][e] & tbits) last = e;
-        // the query tile is loaded for every item; it must have landed before its buffer is handed back
-        ok = mbar_wait(s32(&sm.q_full[t]), it & 1, abort, status);
-        if (!ok) break;
-        if (last < 0) mbar_arrive(s32(&sm.q_empty[t]));
-        bool first = true;
-        for (int e = 0; e < n && ok; ++e) {
-          const bool act = (sm.mask[buf][e] & tbits) != 0;
-          for (int c = 0; c < g.cpb; ++c, ++step) {
-            const int st = (int)(step % kStages);
-            ok = mbar_wait(s32(&sm.kv_full[st]), (uint32_t)((step / kStages) & 1), abort, status);
+    constexpr uint32_t idesc_qk = make_idesc(false), idesc_pv = make_idesc(true);
+    const uint64_t qdesc = smem_desc(s32(sm.q[t]));
+    const uint32_t tcol_o = tmem + kColO + 64 * t, tcol_s = tmem + kColS + 64 * t;
+    const uint32_t tbits = 3u << (2 * t);
+    long long step = 0;   // ring position (all chunks, attended by this tile or not)
+    uint32_t nt = 0;      // products issued by this tile so far (phase of s_full/p_full/pv_done)
+    bool ok = true;
+    for (int it = 0; ok; ++it) {
+      const int buf = it & 1;
+      ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.list_full[buf]), (it >> 1) & 1, abort, status));
+      if (!ok) break;
+      const int n = sm.info[buf].n;
+      if (n < 0) break;
+      int last = -1;
+      for (int e = 0; e < n; ++e)
+        if (sm.mask[buf][e] & tbits) last = e;
+      // the query tile is loaded for every item; it must have landed before its buffer is handed back
+      ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.q_full[t]), it & 1, abort, status));
+      if (!ok) break;
+      if (last < 0 && elect_one()) mbar_arrive(s32(&sm.q_empty[t]));
+      bool first = true;
+      for (int e = 0; e < n && ok; ++e) {
+        const bool act = (sm.mask[buf][e] & tbits) != 0;
+        for (int c = 0; c < g.cpb; ++c, ++step) {
+          const int st = (int)(step % kStages);
+          ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.kv_full[st]), (uint32_t)((step / kStages) & 1), abort, status));
+          if (!ok) break;
+          if (!act) {
+            if (elect_one()) mbar_arrive(s32(&sm.kv_empty[st]));
+            continue;
+          }
+          // S (aliased by P) is free once the previous P V of this tile has completed
+          if (nt > 0) {
+            ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.pv_done[t]), (nt - 1) & 1, abort, status));
             if (!ok) break;
-            if (!act) { mbar_arrive(s32(&sm.kv_empty[st])); continue; }
-            // S (aliased by P) is free once the previous P V of this tile has completed
-            if (nt > 0) {
-              ok = mbar_wait(s32(&sm.pv_done[t]), (nt - 1) & 1, abort, status);
-              if (!ok) break;
-            }
-            tc_fence_after();
-            const uint64_t kdesc = smem_desc(s32(sm.kv[st][0]));
+          }
+          tc_fence_after();
+          const uint64_t kdesc = smem_desc(s32(sm.kv[st][0]));
+          const bool release_q = e == last && c == g.cpb - 1;
+          if (elect_one()) {
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk) umma_ss(tcol_s, qdesc + 2 * kk, kdesc + 2 * kk, idesc_qk, kk > 0);
             tc_commit(s32(&sm.s_full[t]));
-            if (e == last && c == g.cpb - 1) tc_commit(s32(&sm.q_empty[t]));
-            ok = mbar_wait(s32(&sm.p_full[t]), nt & 1, abort, status);
-            if (!ok) break;
-            tc_fence_after();
-            const uint64_t vdesc = smem_desc(s32(sm.kv[st][1]));
+            if (release_q) tc_commit(s32(&sm.q_empty[t]));
+          }
+          __syncwarp();
+          ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.p_full[t]), nt & 1, abort, status));
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t vdesc = smem_desc(s32(sm.kv[st][1]));
+          if (elect_one()) {
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)
               umma_ts(tcol_o, tcol_s + 8 * kk, vdesc + (uint64_t)((2048 * kk) >> 4), idesc_pv, (!first || kk > 0));
             tc_commit(s32(&sm.kv_empty[st]));
             tc_commit(s32(&sm.pv_done[t]));
-            first = false;
-            ++nt;
           }
+          __syncwarp();
+          first = false;
+          ++nt;
         }
-        if (ok) mbar_arrive(s32(&sm.list_empty[buf]));
       }
+      if (ok && elect_one()) mbar_arrive(s32(&sm.list_empty[buf]));
     }
   } else {
     // ------------------------------------------------------------- softmax of tile t, then epilogue

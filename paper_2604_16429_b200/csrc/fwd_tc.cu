@@ -35,11 +35,11 @@ namespace mosaic {
 namespace {
 
 constexpr int kTile = 8192;                      // bytes of one 64 x 64 bf16 chunk
-constexpr int kStages = 4;                       // key/value ring depth (K + V chunk per stage)
+constexpr int kStages = 8;                       // key/value ring depth (K + V chunk per stage)
 constexpr int kMaxUnion = 4 * kMaxList;          // most entries of an item's merged key list
 constexpr int kThreads = 384;
-constexpr uint32_t kTmemCols = 256;
-constexpr uint32_t kColO = 0, kColS = 128;       // O of tile t at 64 t, S of tile t at 128 + 64 t
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kColO = 0, kColS = 128;       // O of tile t at 64 t; S buffer b of tile t at 128 + 128 t + 64 b
 constexpr long long kSpinCycles = 4000000000ll;  // bound of a single wait (~2 s)
 constexpr float kRescaleThreshold = 8.0f;        // log2 units: P stays below 2^8
 
@@ -55,7 +55,8 @@ struct Smem {
   unsigned char q[2][2 * kTile];           // [tile][128 rows x 128 B]
   unsigned char kv[kStages][2][kTile];     // [stage][K, V]
   unsigned long long kv_full[kStages], kv_empty[kStages];
-  unsigned long long q_full[2], q_empty[2], s_full[2], p_full[2], pv_done[2];
+  unsigned long long q_full[2], q_empty[2];
+  unsigned long long s_full[2][2], p_full[2][2], pv_done[2][2];  // [tile][S buffer]
   unsigned long long list_full[2], list_empty[2];
   uint32_t tmem_base;
   int abort;
@@ -410,7 +411,7 @@ __device__ __forceinline__ void interleave_tiles(const int* sid, const unsigned 
 
 }  // namespace
 
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 1)
     fwd_tc_kernel(const Geo g, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_v, const int32_t* __restrict__ block_idx,
                   __nv_bfloat16* __restrict__ o, float* __restrict__ lse, int* status, int* work_counter,
@@ -424,9 +425,11 @@ __global__ void __launch_bounds__(kThreads, 2)
     for (int t = 0; t < 2; ++t) {
       mbar_init(s32(&sm.q_full[t]), 1);
       mbar_init(s32(&sm.q_empty[t]), 1);
-      mbar_init(s32(&sm.s_full[t]), 1);
-      mbar_init(s32(&sm.p_full[t]), 128);
-      mbar_init(s32(&sm.pv_done[t]), 1);
+      for (int b = 0; b < 2; ++b) {
+        mbar_init(s32(&sm.s_full[t][b]), 1);
+        mbar_init(s32(&sm.p_full[t][b]), 128);
+        mbar_init(s32(&sm.pv_done[t][b]), 1);
+      }
       mbar_init(s32(&sm.list_full[t]), 1);
       mbar_init(s32(&sm.list_empty[t]), 11);  // 8 softmax warps + 2 MMA warps + TMA producer
     }
@@ -540,14 +543,33 @@ __global__ void __launch_bounds__(kThreads, 2)
     // ------------------------------------------------------------- MMA issuer of tile t
     // The whole warp walks the loop (waits are cheap polls); one elected lane issues the tensor-core
     // instructions, so operands that are the same for the warp stay in uniform registers.
+    // S is double-buffered: QK^T of product n+1 is issued before P V of product n, so the tensor core
+    // fills the next S while the softmax warps work on the current one.
     const int t = warp - 9;
     constexpr uint32_t idesc_qk = make_idesc(false), idesc_pv = make_idesc(true);
     const uint64_t qdesc = smem_desc(s32(sm.q[t]));
-    const uint32_t tcol_o = tmem + kColO + 64 * t, tcol_s = tmem + kColS + 64 * t;
+    const uint32_t tcol_o = tmem + kColO + 64 * t, tcol_s = tmem + kColS + 128 * t;
     const uint32_t tbits = 3u << (2 * t);
     long long step = 0;   // ring position (all chunks, attended by this tile or not)
-    uint32_t nt = 0;      // products issued by this tile so far (phase of s_full/p_full/pv_done)
+    uint32_t nt = 0;      // products issued by this tile so far: buffer nt & 1, phase (nt >> 1) & 1
     bool ok = true;
+    // P V of product `pn` (its V chunk sits in ring stage `pst`); `pfirst` starts a new accumulation
+    auto issue_pv = [&](uint32_t pn, int pst, bool pfirst) {
+      const uint32_t b = pn & 1;
+      ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.p_full[t][b]), (pn >> 1) & 1, abort, status));
+      if (!ok) return;
+      tc_fence_after();
+      const uint64_t vdesc = smem_desc(s32(sm.kv[pst][1]));
+      const uint32_t pcol = tcol_s + 64 * b;
+      if (elect_one()) {
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+          umma_ts(tcol_o, pcol + 8 * kk, vdesc + (uint64_t)((2048 * kk) >> 4), idesc_pv, (!pfirst || kk > 0));
+        tc_commit(s32(&sm.kv_empty[pst]));
+        tc_commit(s32(&sm.pv_done[t][b]));
+      }
+      __syncwarp();
+    };
     for (int it = 0; ok; ++it) {
       const int buf = it & 1;
       ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.list_full[buf]), (it >> 1) & 1, abort, status));
@@ -561,20 +583,25 @@ __global__ void __launch_bounds__(kThreads, 2)
       ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.q_full[t]), it & 1, abort, status));
       if (!ok) break;
       if (last < 0 && elect_one()) mbar_arrive(s32(&sm.q_empty[t]));
-      bool first = true;
+      bool first = true, pend = false, pend_first = false;
+      uint32_t pend_n = 0;
+      int pend_st = 0;
       for (int e = 0; e < n && ok; ++e) {
         const bool act = (sm.mask[buf][e] & tbits) != 0;
-        for (int c = 0; c < g.cpb; ++c, ++step) {
+        for (int c = 0; c < g.cpb && ok; ++c, ++step) {
           const int st = (int)(step % kStages);
-          ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.kv_full[st]), (uint32_t)((step / kStages) & 1), abort, status));
+          ok = __all_sync(0xffffffffu,
+                          mbar_wait(s32(&sm.kv_full[st]), (uint32_t)((step / kStages) & 1), abort, status));
           if (!ok) break;
           if (!act) {
             if (elect_one()) mbar_arrive(s32(&sm.kv_empty[st]));
             continue;
           }
-          // S (aliased by P) is free once the previous P V of this tile has completed
-          if (nt > 0) {
-            ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.pv_done[t]), (nt - 1) & 1, abort, status));
+          // S buffer nt & 1 (aliased by P) is free once P V of product nt - 2 has completed
+          const uint32_t b = nt & 1;
+          if (nt >= 2) {
+            ok = __all_sync(0xffffffffu,
+                            mbar_wait(s32(&sm.pv_done[t][b]), ((nt - 2) >> 1) & 1, abort, status));
             if (!ok) break;
           }
           tc_fence_after();
@@ -582,27 +609,19 @@ __global__ void __launch_bounds__(kThreads, 2)
           const bool release_q = e == last && c == g.cpb - 1;
           if (elect_one()) {
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) umma_ss(tcol_s, qdesc + 2 * kk, kdesc + 2 * kk, idesc_qk, kk > 0);
-            tc_commit(s32(&sm.s_full[t]));
+            for (int kk = 0; kk < 4; ++kk)
+              umma_ss(tcol_s + 64 * b, qdesc + 2 * kk, kdesc + 2 * kk, idesc_qk, kk > 0);
+            tc_commit(s32(&sm.s_full[t][b]));
             if (release_q) tc_commit(s32(&sm.q_empty[t]));
           }
           __syncwarp();
-          ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.p_full[t]), nt & 1, abort, status));
-          if (!ok) break;
-          tc_fence_after();
-          const uint64_t vdesc = smem_desc(s32(sm.kv[st][1]));
-          if (elect_one()) {
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-              umma_ts(tcol_o, tcol_s + 8 * kk, vdesc + (uint64_t)((2048 * kk) >> 4), idesc_pv, (!first || kk > 0));
-            tc_commit(s32(&sm.kv_empty[st]));
-            tc_commit(s32(&sm.pv_done[t]));
-          }
-          __syncwarp();
+          if (pend) issue_pv(pend_n, pend_st, pend_first);
+          pend = true; pend_n = nt; pend_st = st; pend_first = first;
           first = false;
           ++nt;
         }
       }
+      if (ok && pend) issue_pv(pend_n, pend_st, pend_first);  // the item's last product
       if (ok && elect_one()) mbar_arrive(s32(&sm.list_empty[buf]));
     }
   } else {
@@ -611,7 +630,7 @@ __global__ void __launch_bounds__(kThreads, 2)
     const int hh = (warp >> 1) & 1; // 64-row half of the tile this warp's rows belong to
     const int h = 2 * t + hh;
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t ts = tmem + lane_off + kColS + 64 * t, to = tmem + lane_off + kColO + 64 * t;
+    const uint32_t ts = tmem + lane_off + kColS + 128 * t, to = tmem + lane_off + kColO + 64 * t;
     const uint32_t tbits = 3u << (2 * t), hbit = 1u << h;
     const uint64_t scale2 = pack2(g.scale_log2, g.scale_log2);
     uint32_t nt = 0;
@@ -630,28 +649,29 @@ __global__ void __launch_bounds__(kThreads, 2)
         if (!(mk & tbits)) continue;
         const bool attends = (mk & hbit) != 0;
         for (int c = 0; c < g.cpb; ++c) {
-          ok = mbar_wait(s32(&sm.s_full[t]), nt & 1, abort, status);
+          const uint32_t b = nt & 1, tsb = ts + 64 * b;
+          ok = mbar_wait(s32(&sm.s_full[t][b]), (nt >> 1) & 1, abort, status);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
           if (attends) {
             uint32_t sa[32], sb[32];
-            tmem_ld32(ts, sa);
+            tmem_ld32(tsb, sa);
+            tmem_ld32(tsb + 32, sb);
             tmem_wait_ld();
-            float mx0 = __uint_as_float(sa[0]), mx1 = __uint_as_float(sa[1]);
+            float mx0 = __uint_as_float(sa[0]), mx1 = __uint_as_float(sa[1]), mx2 = __uint_as_float(sb[0]),
+                  mx3 = __uint_as_float(sb[1]);
 #pragma unroll
-            for (int i = 2; i < 32; i += 4) {
-              mx0 = max3(mx0, __uint_as_float(sa[i]), __uint_as_float(sa[i + 1]));
-              if (i + 3 < 32) mx1 = max3(mx1, __uint_as_float(sa[i + 2]), __uint_as_float(sa[i + 3]));
+            for (int i = 2; i < 32; i += 2) {
+              if (i & 2) {
+                mx0 = max3(mx0, __uint_as_float(sa[i]), __uint_as_float(sa[i + 1]));
+                mx2 = max3(mx2, __uint_as_float(sb[i]), __uint_as_float(sb[i + 1]));
+              } else {
+                mx1 = max3(mx1, __uint_as_float(sa[i]), __uint_as_float(sa[i + 1]));
+                mx3 = max3(mx3, __uint_as_float(sb[i]), __uint_as_float(sb[i + 1]));
+              }
             }
-            tmem_ld32(ts + 32, sb);
-            tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; i += 4) {
-              mx0 = max3(mx0, __uint_as_float(sb[i]), __uint_as_float(sb[i + 1]));
-              mx1 = max3(mx1, __uint_as_float(sb[i + 2]), __uint_as_float(sb[i + 3]));
-            }
-            const float mx = fmaxf(mx0, mx1) * g.scale_log2;  // scale > 0 commutes with max
+            const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * g.scale_log2;  // scale > 0 commutes with max
             bool need = false;
             float alpha = 1.f;
             if (m_ref == -INFINITY) {
@@ -664,22 +684,7 @@ __global__ void __launch_bounds__(kThreads, 2)
             }
             const uint64_t negm2 = pack2(-m_ref, -m_ref);
             uint64_t sum_a = pack2(0.f, 0.f), sum_b = sum_a;
-            uint32_t pk[16];
-            // columns 32..63 first (they are in registers), then columns 0..31 again from TMEM
-#pragma unroll
-            for (int i = 0; i < 32; i += 4) {
-              float x0, x1, x2, x3;
-              unpack2(fma2(pack2(__uint_as_float(sb[i]), __uint_as_float(sb[i + 1])), scale2, negm2), x0, x1);
-              unpack2(fma2(pack2(__uint_as_float(sb[i + 2]), __uint_as_float(sb[i + 3])), scale2, negm2), x2, x3);
-              const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
-              sum_a = add2(sum_a, pack2(p0, p1));
-              sum_b = add2(sum_b, pack2(p2, p3));
-              pk[i >> 1] = bf16x2(p0, p1);
-              pk[(i >> 1) + 1] = bf16x2(p2, p3);
-            }
-            tmem_ld32(ts, sa);          // S columns 0..31 are still intact: P has not been written yet
-            tmem_wait_ld();
-            tmem_st16(ts + 16, pk);     // P columns 32..63 (bf16 pairs) = 32-bit columns 16..31
+            uint32_t pk[32];
 #pragma unroll
             for (int i = 0; i < 32; i += 4) {
               float x0, x1, x2, x3;
@@ -691,12 +696,29 @@ __global__ void __launch_bounds__(kThreads, 2)
               pk[i >> 1] = bf16x2(p0, p1);
               pk[(i >> 1) + 1] = bf16x2(p2, p3);
             }
-            tmem_st16(ts, pk);
+#pragma unroll
+            for (int i = 0; i < 32; i += 4) {
+              float x0, x1, x2, x3;
+              unpack2(fma2(pack2(__uint_as_float(sb[i]), __uint_as_float(sb[i + 1])), scale2, negm2), x0, x1);
+              unpack2(fma2(pack2(__uint_as_float(sb[i + 2]), __uint_as_float(sb[i + 3])), scale2, negm2), x2, x3);
+              const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
+              sum_a = add2(sum_a, pack2(p0, p1));
+              sum_b = add2(sum_b, pack2(p2, p3));
+              pk[16 + (i >> 1)] = bf16x2(p0, p1);
+              pk[16 + (i >> 1) + 1] = bf16x2(p2, p3);
+            }
+            tmem_st32(tsb, pk);  // P (bf16 pairs) over the first 32 columns of this S buffer
             float s0, s1;
             unpack2(add2(sum_a, sum_b), s0, s1);
             l += s0 + s1;
             if (__any_sync(0xffffffffu, need)) {
-              // the previous P V of this tile completed before this S was produced: O is at rest
+              // the accumulator may only be touched between P V products: wait for the previous one
+              if (done > 0) {
+                ok = mbar_wait(s32(&sm.pv_done[t][b ^ 1]), ((nt - 1) >> 1) & 1, abort, status);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+              }
               const uint64_t alpha2 = pack2(alpha, alpha);
 #pragma unroll
               for (int part = 0; part < 2; ++part) {
@@ -705,10 +727,10 @@ __global__ void __launch_bounds__(kThreads, 2)
                 tmem_wait_ld();
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
-                  float a, b;
-                  unpack2(mul2(pack2(__uint_as_float(ov[i]), __uint_as_float(ov[i + 1])), alpha2), a, b);
+                  float a, bb;
+                  unpack2(mul2(pack2(__uint_as_float(ov[i]), __uint_as_float(ov[i + 1])), alpha2), a, bb);
                   ov[i] = __float_as_uint(a);
-                  ov[i + 1] = __float_as_uint(b);
+                  ov[i + 1] = __float_as_uint(bb);
                 }
                 tmem_st32(to + 32 * part, ov);
               }
@@ -717,18 +739,18 @@ __global__ void __launch_bounds__(kThreads, 2)
             uint32_t z[32];
 #pragma unroll
             for (int i = 0; i < 32; ++i) z[i] = 0u;
-            tmem_st32(ts, z);
+            tmem_st32(tsb, z);
           }
           tmem_wait_st();
           tc_fence_before();
-          mbar_arrive(s32(&sm.p_full[t]));
+          mbar_arrive(s32(&sm.p_full[t][b]));
           ++nt;
           ++done;
         }
       }
       if (!ok) break;
       if (done > 0) {
-        ok = mbar_wait(s32(&sm.pv_done[t]), (nt - 1) & 1, abort, status);
+        ok = mbar_wait(s32(&sm.pv_done[t][(nt - 1) & 1]), ((nt - 1) >> 1) & 1, abort, status);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
@@ -818,7 +840,7 @@ int launch_fwd_tc(const HostCtx& c, const void* q, const void* k, const void* v,
   const int ipu = items_per_unit(g);
   const long long total = (long long)g.U * ipu;
   if (total > 0x7fffff00ll) return MOSAIC_E_UNSUPPORTED;
-  const long long grid = total < 2ll * sms ? total : 2ll * sms;
+  const long long grid = total < (long long)sms ? total : (long long)sms;
   // the work counter is the second word of the status block, zeroed with it when the op starts
   fwd_tc_kernel<<<(unsigned)grid, kThreads, smem, c.stream>>>(g, mq, mk, mv, block_idx, (__nv_bfloat16*)o, lse,
                                                              c.status, c.status + 1, ipu, (int)total);

@@ -14,49 +14,58 @@
 namespace mosaic {
 
 // ------------------------------------------------------------------------------------------
-// pool_kernel: one warp per (tensor, unit, block); lane owns channels 2*lane, 2*lane+1.
-// HBM-bound: reads 2*U*N*d*2 bytes once, every warp request is one full 128-byte line.
+// pool_kernel: eight lanes per (tensor, unit, block), four blocks per warp; a lane owns eight
+// consecutive channels (one 16-byte load per token) and adds them in token order, row-major inside
+// the block, so every channel is one sequential fp64 chain.  HBM-bound: reads 2*U*N*d*2 bytes once;
+// the loads of a whole block row are in flight together.
 // ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) pool_kernel(Geo g, const uint32_t* __restrict__ q,
-                                                   const uint32_t* __restrict__ k, float* __restrict__ pq,
-                                                   float* __restrict__ pk) {
-  const int lane = threadIdx.x & 31;
-  const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+template <int BW>
+__global__ void __launch_bounds__(256) pool_kernel(Geo g, const uint4* __restrict__ q, const uint4* __restrict__ k,
+                                                   float* __restrict__ pq, float* __restrict__ pk) {
+  const int sub = threadIdx.x & 7;  // which 8 channels
+  const long long grp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 3;
   const long long per_tensor = (long long)g.U * g.m;
-  if (warp >= 2 * per_tensor) return;
-  const int which = warp >= per_tensor;
-  const long long w = warp - which * per_tensor;
+  if (grp >= 2 * per_tensor) return;
+  const int which = grp >= per_tensor;
+  const long long w = grp - which * per_tensor;
   const int u = (int)(w / g.m), j = (int)(w - (long long)u * g.m);
-  const uint32_t* src = (which ? k : q) + (long long)u * g.N * (kD / 2) + lane;
+  const uint4* src = (which ? k : q) + (long long)u * g.N * (kD / 8) + sub;
   const int by = j / g.nbw, bx = j - by * g.nbw;
-  double a0 = 0.0, a1 = 0.0;
+  double acc[8];
+#pragma unroll
+  for (int c = 0; c < 8; ++c) acc[c] = 0.0;
   for (int r = 0; r < g.bh; ++r) {
-    const uint32_t* row = src + ((long long)(by * g.bh + r) * g.nlon + bx * g.bw) * (kD / 2);
-    // bw is 8 or 16: issue the row's loads together, then add in token order
-    uint32_t v[16];
+    const uint4* row = src + ((long long)(by * g.bh + r) * g.nlon + bx * BW) * (kD / 8);
+    uint4 v[BW];
 #pragma unroll
-    for (int c = 0; c < 16; ++c)
-      if (c < g.bw) v[c] = __ldg(row + c * (kD / 2));
+    for (int c = 0; c < BW; ++c) v[c] = __ldg(row + c * (kD / 8));
 #pragma unroll
-    for (int c = 0; c < 16; ++c)
-      if (c < g.bw) {
-        a0 += (double)__uint_as_float(v[c] << 16);
-        a1 += (double)__uint_as_float(v[c] & 0xffff0000u);
+    for (int c = 0; c < BW; ++c) {
+      const uint32_t x[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        acc[2 * e] += (double)__uint_as_float(x[e] << 16);
+        acc[2 * e + 1] += (double)__uint_as_float(x[e] & 0xffff0000u);
       }
+    }
   }
-  float* dst = (which ? pk : pq) + ((long long)u * g.m + j) * kD + 2 * lane;
-  *reinterpret_cast<float2*>(dst) = make_float2((float)a0, (float)a1);
+  float4* dst = reinterpret_cast<float4*>((which ? pk : pq) + ((long long)u * g.m + j) * kD + 8 * sub);
+  dst[0] = make_float4((float)acc[0], (float)acc[1], (float)acc[2], (float)acc[3]);
+  dst[1] = make_float4((float)acc[4], (float)acc[5], (float)acc[6], (float)acc[7]);
 }
 
 // ------------------------------------------------------------------------------------------
-// topk_kernel: a CTA owns TQ query blocks of one unit and streams the pooled keys in chunks
-// of JC blocks through shared memory.  Thread t scores key block (chunk*JC + t) against the
-// TQ pooled queries (fp64 FMA chain over channels); then one warp per query row merges the
-// chunk into a sorted k-entry list held one entry per lane.
+// topk_kernel<TI>: a CTA owns TI query blocks of one unit and streams the pooled keys in chunks of
+// JT blocks through shared memory (as fp64, channel-major).  The TI x JT scores of a chunk are a
+// register-tiled fp64 product: thread (ty, tx) holds the scores of rows ty + 16a and keys tx + 16b
+// and runs one FMA chain over channels 0..d-1 per score, so each score is the sequential sum the
+// selection is defined by.  Scores become sortable keys; a key that cannot enter its row's list
+// (worse than the row's current k-th best) is dropped at once.
+// Merge: one warp per query row keeps the sorted k-entry list, one entry per lane; the rows of a warp
+// advance in lockstep so that their reductions overlap.
 // ------------------------------------------------------------------------------------------
-constexpr int TQ = 16;
-constexpr int JC = 256;
-constexpr int KPAD = kD + 1;
+constexpr int JT = 64;
+constexpr int KSTR = JT + 1;  // padded row of the key tile: conflict-free transposing stores
 
 // Total-order key: larger key = better score.  0 = not a candidate, 1 = NaN.
 __device__ __forceinline__ unsigned long long score_key(double s) {
@@ -71,94 +80,163 @@ __device__ __forceinline__ bool ranks_before(unsigned long long ka, int ia, unsi
   return ka > kb || (ka == kb && ia < ib);
 }
 
-__global__ void __launch_bounds__(JC) topk_kernel(Geo g, const float* __restrict__ pq,
-                                                  const float* __restrict__ pk, int32_t* __restrict__ block_idx) {
+template <int TI>
+struct TopkSmem {
+  double qs[kD][TI];                   // pooled queries of this CTA, channel-major
+  double ks[kD][KSTR];                 // pooled keys of the current chunk, channel-major
+  unsigned long long keys[TI][JT];     // candidate keys of the current chunk (0 = none)
+  unsigned long long thr[TI];          // key of the row's current k-th best (0 while the list is short)
+  int flag[TI];                        // the row has a candidate in this chunk
+  short iy[TI], ix[TI], jy[JT], jx[JT];  // block coordinates of the rows and of the chunk's keys
+};
+
+template <int TI>
+__global__ void __launch_bounds__(256) topk_kernel(Geo g, const float* __restrict__ pq,
+                                                   const float* __restrict__ pk, int32_t* __restrict__ block_idx) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  double* qs = reinterpret_cast<double*>(smem_raw);                         // [TQ][kD]
-  unsigned long long* keys = reinterpret_cast<unsigned long long*>(qs + TQ * kD);  // [TQ][JC]
-  float* ks = reinterpret_cast<float*>(keys + TQ * JC);                     // [JC][KPAD]
+  TopkSmem<TI>& sm = *reinterpret_cast<TopkSmem<TI>*>(smem_raw);
+  constexpr int RI = TI / 16;                 // query rows per thread
+  constexpr int RPW = TI / 8;                 // query rows per warp in the merge
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int tiles = (g.m + TQ - 1) / TQ;
-  const int u = blockIdx.x / tiles, i0 = (blockIdx.x - u * tiles) * TQ;
+  const int tx = tid & 15, ty = tid >> 4;
+  const int tiles = (g.m + TI - 1) / TI;
+  const int u = blockIdx.x / tiles, i0 = (blockIdx.x - u * tiles) * TI;
   const float* pq_u = pq + (long long)u * g.m * kD;
   const float* pk_u = pk + (long long)u * g.m * kD;
 
-  for (int e = tid; e < TQ * kD; e += JC) {
-    int r = e / kD, i = i0 + r;
-    qs[e] = i < g.m ? (double)pq_u[(long long)i * kD + (e - r * kD)] : 0.0;
+  for (int e = tid; e < TI * kD; e += 256) {
+    const int r = e / kD, c = e - r * kD, i = i0 + r;
+    sm.qs[c][r] = i < g.m ? (double)pq_u[(long long)i * kD + c] : 0.0;
+  }
+  for (int r = tid; r < TI; r += 256) {
+    const int i = min(i0 + r, g.m - 1);
+    sm.thr[r] = 0ull;
+    sm.iy[r] = (short)(i / g.nbw);
+    sm.ix[r] = (short)(i - (i / g.nbw) * g.nbw);
   }
 
   // sorted list of the best candidates so far: entry `lane` of each row this warp owns
-  constexpr int RPW = TQ / (JC / 32);  // rows per warp
   unsigned long long lkey[RPW];
   int lid[RPW];
 #pragma unroll
   for (int r = 0; r < RPW; ++r) { lkey[r] = 0ull; lid[r] = -1; }
 
-  for (int j0 = 0; j0 < g.m; j0 += JC) {
-    __syncthreads();  // previous chunk fully merged (and qs written on the first pass)
-    const int nj = min(JC, g.m - j0);
-    for (int e = tid; e < nj * kD; e += JC) {
-      int jj = e / kD;
-      ks[jj * KPAD + (e - jj * kD)] = pk_u[(long long)j0 * kD + e];
+  for (int j0 = 0; j0 < g.m; j0 += JT) {
+    __syncthreads();  // previous chunk fully merged (and qs, thr written on the first pass)
+    const int nj = min(JT, g.m - j0);
+#pragma unroll
+    for (int e = tid; e < JT * kD / 4; e += 256) {
+      const int jj = e / (kD / 4), c4 = (e - jj * (kD / 4)) * 4;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (jj < nj) v = __ldg(reinterpret_cast<const float4*>(pk_u + (long long)(j0 + jj) * kD + c4));
+      sm.ks[c4][jj] = (double)v.x;
+      sm.ks[c4 + 1][jj] = (double)v.y;
+      sm.ks[c4 + 2][jj] = (double)v.z;
+      sm.ks[c4 + 3][jj] = (double)v.w;
     }
+    if (tid < JT) {
+      const int j = min(j0 + tid, g.m - 1);
+      sm.jy[tid] = (short)(j / g.nbw);
+      sm.jx[tid] = (short)(j - (j / g.nbw) * g.nbw);
+    }
+    for (int r = tid; r < TI; r += 256) sm.flag[r] = 0;
     __syncthreads();
     {
-      const int j = j0 + tid;
-      double acc[TQ];
+      double acc[RI][4];
 #pragma unroll
-      for (int r = 0; r < TQ; ++r) acc[r] = 0.0;
-      if (tid < nj) {
-        for (int c = 0; c < kD; ++c) {
-          const double kc = (double)ks[tid * KPAD + c];
+      for (int a = 0; a < RI; ++a)
 #pragma unroll
-          for (int r = 0; r < TQ; ++r) acc[r] = fma(qs[r * kD + c], kc, acc[r]);
-        }
+        for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
+#pragma unroll 8
+      for (int c = 0; c < kD; ++c) {
+        double qv[RI], kv[4];
+#pragma unroll
+        for (int a = 0; a < RI; ++a) qv[a] = sm.qs[c][ty + 16 * a];
+#pragma unroll
+        for (int b = 0; b < 4; ++b) kv[b] = sm.ks[c][tx + 16 * b];
+#pragma unroll
+        for (int a = 0; a < RI; ++a)
+#pragma unroll
+          for (int b = 0; b < 4; ++b) acc[a][b] = fma(qv[a], kv[b], acc[a][b]);
       }
 #pragma unroll
-      for (int r = 0; r < TQ; ++r) {
-        const int i = i0 + r;
-        const bool cand = tid < nj && i < g.m && !is_local(g, i, j);
-        keys[r * JC + tid] = cand ? score_key(acc[r]) : 0ull;
+      for (int a = 0; a < RI; ++a) {
+        const int r = ty + 16 * a, i = i0 + r;
+        const unsigned long long th = sm.thr[r];
+        const int iy = sm.iy[r], ix = sm.ix[r];
+        bool any = false;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+          const int jj = tx + 16 * b;
+          int dx = sm.jx[jj] - ix;
+          dx += dx < 0 ? g.nbw : 0;  // (jx - ix) mod nbw
+          const bool local = abs(sm.jy[jj] - iy) <= g.rlat && (dx <= g.rlon || g.nbw - dx <= g.rlon);
+          unsigned long long key = 0ull;
+          if (jj < nj && i < g.m && !local) {
+            key = score_key(acc[a][b]);
+            if (key < th) key = 0ull;  // cannot enter the list (an equal key may: lower id wins)
+          }
+          sm.keys[r][jj] = key;
+          any |= key != 0ull;
+        }
+        if (any) sm.flag[r] = 1;
       }
     }
     __syncthreads();
-    // merge: repeatedly take the best remaining chunk entry while it still enters the list
+    // merge, all rows of this warp in lockstep: repeatedly take each row's best remaining chunk entry
+    // while it still enters the row's list
+    unsigned live = 0;
+#pragma unroll
+    for (int rr = 0; rr < RPW; ++rr) live |= (sm.flag[warp * RPW + rr] ? 1u : 0u) << rr;
+    for (int round = 0; round < g.topk && live; ++round) {
+      unsigned long long bk[RPW];
+      int bj[RPW];
+#pragma unroll
+      for (int rr = 0; rr < RPW; ++rr) {
+        bk[rr] = 0ull;
+        bj[rr] = 0x7fffffff;
+        if ((live >> rr) & 1) {
+          const unsigned long long* row = sm.keys[warp * RPW + rr];
+#pragma unroll
+          for (int s = 0; s < JT / 32; ++s) {
+            const unsigned long long kk = row[lane + 32 * s];
+            const int jj = j0 + lane + 32 * s;
+            if (kk != 0ull && ranks_before(kk, jj, bk[rr], bj[rr])) { bk[rr] = kk; bj[rr] = jj; }
+          }
+        }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+        for (int rr = 0; rr < RPW; ++rr) {
+          const unsigned long long ok = __shfl_xor_sync(0xffffffffu, bk[rr], o);
+          const int oj = __shfl_xor_sync(0xffffffffu, bj[rr], o);
+          if (ok != 0ull && ranks_before(ok, oj, bk[rr], bj[rr])) { bk[rr] = ok; bj[rr] = oj; }
+        }
+      }
+#pragma unroll
+      for (int rr = 0; rr < RPW; ++rr) {
+        // list is sorted best-first; its last wanted entry sits in lane topk-1
+        const unsigned long long tk = __shfl_sync(0xffffffffu, lkey[rr], g.topk - 1);
+        const int ti = __shfl_sync(0xffffffffu, lid[rr], g.topk - 1);
+        const bool enters = bk[rr] != 0ull && (tk == 0ull || ranks_before(bk[rr], bj[rr], tk, ti));
+        if (!enters) { live &= ~(1u << rr); continue; }  // chunk exhausted for this row
+        // insert at position p = number of entries ranking before the new one
+        const bool before = lkey[rr] != 0ull && ranks_before(lkey[rr], lid[rr], bk[rr], bj[rr]);
+        const int p = __popc(__ballot_sync(0xffffffffu, before));
+        const unsigned long long uk = __shfl_up_sync(0xffffffffu, lkey[rr], 1);
+        const int ui = __shfl_up_sync(0xffffffffu, lid[rr], 1);
+        if (lane == p) { lkey[rr] = bk[rr]; lid[rr] = bj[rr]; }
+        else if (lane > p) { lkey[rr] = uk; lid[rr] = ui; }
+        if (lane == ((bj[rr] - j0) & 31)) sm.keys[warp * RPW + rr][bj[rr] - j0] = 0ull;  // taken
+      }
+      __syncwarp();
+    }
 #pragma unroll
     for (int rr = 0; rr < RPW; ++rr) {
-      const int r = warp * RPW + rr;
-      unsigned long long* row = keys + r * JC;
-      for (int round = 0; round < g.topk; ++round) {
-        unsigned long long bk = 0ull;
-        int bj = 0x7fffffff;
-#pragma unroll
-        for (int s = 0; s < JC / 32; ++s) {
-          unsigned long long kk = row[lane + 32 * s];
-          int jj = j0 + lane + 32 * s;
-          if (kk != 0ull && ranks_before(kk, jj, bk, bj)) { bk = kk; bj = jj; }
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-          unsigned long long ok = __shfl_xor_sync(0xffffffffu, bk, o);
-          int oj = __shfl_xor_sync(0xffffffffu, bj, o);
-          if (ok != 0ull && ranks_before(ok, oj, bk, bj)) { bk = ok; bj = oj; }
-        }
-        if (bk == 0ull) break;  // chunk exhausted
-        // list is sorted best-first; its last wanted entry sits in lane topk-1
-        unsigned long long tk = __shfl_sync(0xffffffffu, lkey[rr], g.topk - 1);
-        int ti = __shfl_sync(0xffffffffu, lid[rr], g.topk - 1);
-        if (tk != 0ull && !ranks_before(bk, bj, tk, ti)) break;  // nothing left that enters
-        // insert at position p = number of entries ranking before the new one
-        bool before = lkey[rr] != 0ull && ranks_before(lkey[rr], lid[rr], bk, bj);
-        int p = __popc(__ballot_sync(0xffffffffu, before));
-        unsigned long long uk = __shfl_up_sync(0xffffffffu, lkey[rr], 1);
-        int ui = __shfl_up_sync(0xffffffffu, lid[rr], 1);
-        if (lane == p) { lkey[rr] = bk; lid[rr] = bj; }
-        else if (lane > p) { lkey[rr] = uk; lid[rr] = ui; }
-        if (lane == ((bj - j0) & 31)) row[bj - j0] = 0ull;  // taken
-        __syncwarp();
-      }
+      const unsigned long long tk = __shfl_sync(0xffffffffu, lkey[rr], g.topk - 1);
+      if (lane == 0) sm.thr[warp * RPW + rr] = tk;  // 0 until the list holds topk entries
     }
   }
 #pragma unroll
@@ -169,28 +247,36 @@ __global__ void __launch_bounds__(JC) topk_kernel(Geo g, const float* __restrict
   }
 }
 
+template <int TI>
+int launch_topk(const HostCtx& c, const float* pooled_q, const float* pooled_k, int32_t* block_idx) {
+  const Geo& g = c.g;
+  const size_t smem = sizeof(TopkSmem<TI>);
+  if (cudaFuncSetAttribute(topk_kernel<TI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return MOSAIC_E_CUDA;
+  const int tiles = (g.m + TI - 1) / TI;
+  topk_kernel<TI><<<(unsigned)(g.U * tiles), 256, smem, c.stream>>>(g, pooled_q, pooled_k, block_idx);
+  return cudaGetLastError() == cudaSuccess ? MOSAIC_OK : MOSAIC_E_CUDA;
+}
+
 int launch_select(const HostCtx& c, const void* q, const void* k, int32_t* block_idx, float* pooled_q,
                   float* pooled_k) {
   const Geo& g = c.g;
   {
-    long long warps = 2ll * g.U * g.m;
-    int wpb = 8;
-    long long blocks = (warps + wpb - 1) / wpb;
-    pool_kernel<<<(unsigned)blocks, wpb * 32, 0, c.stream>>>(g, (const uint32_t*)q, (const uint32_t*)k,
-                                                             pooled_q, pooled_k);
+    const long long threads = 2ll * g.U * g.m * 8;
+    const unsigned blocks = (unsigned)((threads + 255) / 256);
+    if (g.bw == 8)
+      pool_kernel<8><<<blocks, 256, 0, c.stream>>>(g, (const uint4*)q, (const uint4*)k, pooled_q, pooled_k);
+    else
+      pool_kernel<16><<<blocks, 256, 0, c.stream>>>(g, (const uint4*)q, (const uint4*)k, pooled_q, pooled_k);
     if (cudaGetLastError() != cudaSuccess) return MOSAIC_E_CUDA;
   }
   if (g.topk > 0) {
-    size_t smem = sizeof(double) * TQ * kD + sizeof(unsigned long long) * TQ * JC + sizeof(float) * JC * KPAD;
-    static bool attr_set = false;
-    if (!attr_set) {
-      if (cudaFuncSetAttribute(topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-        return MOSAIC_E_CUDA;
-      attr_set = true;
-    }
-    int tiles = (g.m + TQ - 1) / TQ;
-    topk_kernel<<<(unsigned)(g.U * tiles), JC, smem, c.stream>>>(g, pooled_q, pooled_k, block_idx);
-    if (cudaGetLastError() != cudaSuccess) return MOSAIC_E_CUDA;
+    // the most query blocks per CTA (64, 32, 16) that still gives every SM two CTAs; 16 otherwise
+    auto ctas = [&](int ti) { return (long long)g.U * ((g.m + ti - 1) / ti); };
+    const int rc = ctas(64) >= 296 ? launch_topk<64>(c, pooled_q, pooled_k, block_idx)
+                 : ctas(32) >= 296 ? launch_topk<32>(c, pooled_q, pooled_k, block_idx)
+                                   : launch_topk<16>(c, pooled_q, pooled_k, block_idx);
+    if (rc) return rc;
   }
   return MOSAIC_OK;
 }

@@ -206,14 +206,16 @@ __global__ void __launch_bounds__(256) topk_kernel(Geo g, const float* __restric
           }
         }
       }
+      // warp-wide best of each row: maximum of the key's high word, then of the low word among the
+      // lanes that hold that high word, then the lowest block id among the lanes that hold the key
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-#pragma unroll
-        for (int rr = 0; rr < RPW; ++rr) {
-          const unsigned long long ok = __shfl_xor_sync(0xffffffffu, bk[rr], o);
-          const int oj = __shfl_xor_sync(0xffffffffu, bj[rr], o);
-          if (ok != 0ull && ranks_before(ok, oj, bk[rr], bj[rr])) { bk[rr] = ok; bj[rr] = oj; }
-        }
+      for (int rr = 0; rr < RPW; ++rr) {
+        const unsigned hi = (unsigned)(bk[rr] >> 32), lo = (unsigned)bk[rr];
+        const unsigned mh = __reduce_max_sync(0xffffffffu, hi);
+        const unsigned ml = __reduce_max_sync(0xffffffffu, hi == mh ? lo : 0u);
+        const bool mine = bk[rr] != 0ull && hi == mh && lo == ml;
+        bj[rr] = __reduce_min_sync(0xffffffffu, mine ? bj[rr] : 0x7fffffff);
+        bk[rr] = ((unsigned long long)mh << 32) | ml;
       }
 #pragma unroll
       for (int rr = 0; rr < RPW; ++rr) {

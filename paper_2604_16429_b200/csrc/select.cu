@@ -210,6 +210,7 @@ __global__ void __launch_bounds__(256) topk_kernel(Geo g, const float* __restric
       // lanes that hold that high word, then the lowest block id among the lanes that hold the key
 #pragma unroll
       for (int rr = 0; rr < RPW; ++rr) {
+        if (!((live >> rr) & 1)) continue;  // warp-uniform
         const unsigned hi = (unsigned)(bk[rr] >> 32), lo = (unsigned)bk[rr];
         const unsigned mh = __reduce_max_sync(0xffffffffu, hi);
         const unsigned ml = __reduce_max_sync(0xffffffffu, hi == mh ? lo : 0u);
@@ -220,6 +221,7 @@ __global__ void __launch_bounds__(256) topk_kernel(Geo g, const float* __restric
 #pragma unroll
       for (int rr = 0; rr < RPW; ++rr) {
         // list is sorted best-first; its last wanted entry sits in lane topk-1
+        if (!((live >> rr) & 1)) continue;
         const unsigned long long tk = __shfl_sync(0xffffffffu, lkey[rr], g.topk - 1);
         const int ti = __shfl_sync(0xffffffffu, lid[rr], g.topk - 1);
         const bool enters = bk[rr] != 0ull && (tk == 0ull || ranks_before(bk[rr], bj[rr], tk, ti));

@@ -17,13 +17,19 @@
 // operand layout for S = Q K^T and the MN-major operand layout for O += P V.  A staged chunk serves
 // both tiles of the item.
 //
-// The kernel is persistent: CTAs (two per SM) draw items from a counter in the workspace.
+// The kernel is persistent: one CTA per SM draws items from a counter in the workspace.
 // Warp roles (384 threads): warps 0-3 softmax of tile 0, warps 4-7 softmax of tile 1 (thread = query
-// row = TMEM lane), warp 8 issues TMA, warps 9 and 10 issue tcgen05.mma for tile 0 and tile 1, warp 11
-// draws items from the queue and builds their key lists one item ahead.  Each tile is an independent chain  QK^T -> softmax -> PV  over its own TMEM columns
-// (O: 64 fp32 columns, S: 64 fp32 columns; P (bf16) overwrites the first 32 columns of S and is the
-// TMEM A operand of PV), so four such chains per SM keep the MUFU exponential pipe, the limiter at
-// d = 64, busy while any one of them waits for the tensor core.
+// row = TMEM lane), warp 8 issues TMA, warps 9 and 10 issue tcgen05.mma for tile 0 and tile 1 (the whole
+// warp walks the loop, one elected lane issues), warp 11 draws items from the queue and builds their key
+// lists one item ahead, interleaved so that both tiles find work all along a list.
+// TMEM (512 columns): O of tile t at 64 t (fp32, 64 columns); two S buffers per tile at 128 + 128 t + 64 b
+// (fp32, 64 columns each).  P (bf16) overwrites the first 32 columns of its S buffer and is the TMEM A
+// operand of PV.  QK^T of product n+1 is issued before P V of product n, so the tensor core fills one S
+// buffer while the softmax warps work on the other.
+// Softmax: fp32, base-2 exponentials with the scale folded in, running maximum moved only when it grows by
+// more than 2^8 (then O is rescaled, between two P V products), packed two-lane fp32 arithmetic, and a
+// quarter of the exponentials evaluated by a cubic on the FMA pipe because at d = 64 the MUFU pipe
+// (16 ex2 per clock per SM against 8192 tensor FLOP per clock) is the limiter, not the tensor core.
 // Every mbarrier wait is bounded; on expiry the CTA records MOSAIC_E_DEVICE_TIMEOUT and drains.
 #include <cuda.h>
 #include <cuda_bf16.h>

@@ -625,13 +625,10 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (elect_one()) mbar_arrive(s32(&sm.kv_empty[st]));
             continue;
           }
-          // S buffer nt & 1 (aliased by P) is free once P V of product nt - 2 has completed
+          // S buffer nt & 1 (aliased by P) was last read by P V of product nt - 2, which this warp issued
+          // earlier: tensor-core operations of one thread execute in issue order, so this QK^T cannot
+          // overwrite the buffer before that product has consumed it, and no wait is needed here
           const uint32_t b = nt & 1;
-          if (nt >= 2) {
-            ok = __all_sync(0xffffffffu,
-                            mbar_wait(s32(&sm.pv_done[t][b]), ((nt - 2) >> 1) & 1, abort, status));
-            if (!ok) break;
-          }
           tc_fence_after();
           const uint64_t kdesc = smem_desc(s32(sm.kv[st][0]));
           const bool release_q = e == last && c == g.cpb - 1;

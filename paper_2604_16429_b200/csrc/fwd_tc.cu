@@ -59,10 +59,10 @@ struct ItemInfo {
 };
 
 struct Smem {
-  unsigned char q[2][2 * kTile];           // [tile][128 rows x 128 B]
+  unsigned char q[2][2][2 * kTile];        // [item parity][tile][128 rows x 128 B]
   unsigned char kv[kStages][2][kTile];     // [stage][K, V]
   unsigned long long kv_full[kStages], kv_empty[kStages];
-  unsigned long long q_full[2], q_empty[2];
+  unsigned long long q_full[2][2], q_empty[2][2];  // [item parity][tile]
   unsigned long long s_full[2][2], p_full[2][2], pv_done[2][2];  // [tile][S buffer]
   unsigned long long list_full[2], list_empty[2];
   uint32_t tmem_base;
@@ -451,8 +451,10 @@ __global__ void __launch_bounds__(kThreads, 1)
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(s32(&sm.kv_full[s]), 1); mbar_init(s32(&sm.kv_empty[s]), 2); }
     for (int t = 0; t < 2; ++t) {
-      mbar_init(s32(&sm.q_full[t]), 1);
-      mbar_init(s32(&sm.q_empty[t]), 1);
+      for (int b = 0; b < 2; ++b) {
+        mbar_init(s32(&sm.q_full[b][t]), 1);
+        mbar_init(s32(&sm.q_empty[b][t]), 1);
+      }
       for (int b = 0; b < 2; ++b) {
         mbar_init(s32(&sm.s_full[t][b]), 1);
         mbar_init(s32(&sm.p_full[t][b]), 128);
@@ -534,14 +536,15 @@ __global__ void __launch_bounds__(kThreads, 1)
         const ItemInfo& inf = sm.info[buf];
         const int n = inf.n, u = inf.unit;
         if (n < 0) break;
-        // query tiles: free once the tile's last QK^T of the previous item has completed
+        // query tiles (double-buffered by item parity): free once the tile's last QK^T of the item before
+        // the previous one has completed, so this load runs while the previous item still computes
         for (int t = 0; t < 2 && ok; ++t) {
-          ok = mbar_wait(s32(&sm.q_empty[t]), (it & 1) ^ 1, abort, status);
+          ok = mbar_wait(s32(&sm.q_empty[buf][t]), ((it >> 1) & 1) ^ 1, abort, status);
           if (!ok) break;
-          mbar_expect_tx(s32(&sm.q_full[t]), 2 * kTile);
+          mbar_expect_tx(s32(&sm.q_full[buf][t]), 2 * kTile);
           for (int hh = 0; hh < 2; ++hh) {
             const int h = 2 * t + hh, by = inf.hb[h] / g.nbw, bx = inf.hb[h] - by * g.nbw;
-            tma_load_4d(s32(sm.q[t] + hh * kTile), &map_q, s32(&sm.q_full[t]), 0, bx * g.bw,
+            tma_load_4d(s32(sm.q[buf][t] + hh * kTile), &map_q, s32(&sm.q_full[buf][t]), 0, bx * g.bw,
                         by * g.bh + inf.hc[h] * g.crows, u);
           }
         }
@@ -575,7 +578,6 @@ __global__ void __launch_bounds__(kThreads, 1)
     // fills the next S while the softmax warps work on the current one.
     const int t = warp - 9;
     constexpr uint32_t idesc_qk = make_idesc(false), idesc_pv = make_idesc(true);
-    const uint64_t qdesc = smem_desc(s32(sm.q[t]));
     const uint32_t tcol_o = tmem + kColO + 64 * t, tcol_s = tmem + kColS + 128 * t;
     const uint32_t tbits = 3u << (2 * t);
     long long step = 0;   // ring position (all chunks, attended by this tile or not)
@@ -608,9 +610,10 @@ __global__ void __launch_bounds__(kThreads, 1)
       for (int e = 0; e < n; ++e)
         if (sm.mask[buf][e] & tbits) last = e;
       // the query tile is loaded for every item; it must have landed before its buffer is handed back
-      ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.q_full[t]), it & 1, abort, status));
+      ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.q_full[buf][t]), (it >> 1) & 1, abort, status));
+      const uint64_t qdesc = smem_desc(s32(sm.q[buf][t]));
       if (!ok) break;
-      if (last < 0 && elect_one()) mbar_arrive(s32(&sm.q_empty[t]));
+      if (last < 0 && elect_one()) mbar_arrive(s32(&sm.q_empty[buf][t]));
       bool first = true, pend = false, pend_first = false;
       uint32_t pend_n = 0;
       int pend_st = 0;
@@ -637,7 +640,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             for (int kk = 0; kk < 4; ++kk)
               umma_ss(tcol_s + 64 * b, qdesc + 2 * kk, kdesc + 2 * kk, idesc_qk, kk > 0);
             tc_commit(s32(&sm.s_full[t][b]));
-            if (release_q) tc_commit(s32(&sm.q_empty[t]));
+            if (release_q) tc_commit(s32(&sm.q_empty[buf][t]));
           }
           __syncwarp();
           if (pend) issue_pv(pend_n, pend_st, pend_first);

@@ -43,6 +43,7 @@ namespace {
 constexpr int kTile = 8192;                      // bytes of one 64 x 64 bf16 chunk
 constexpr int kStages = 8;                       // key/value ring depth (K + V chunk per stage)
 constexpr int kMaxUnion = 4 * kMaxList;          // most entries of an item's merged key list
+constexpr int kLists = 4;                        // key lists in flight (the planner runs this far ahead)
 constexpr int kThreads = 384;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColO = 0, kColS = 128;       // O of tile t at 64 t; S buffer b of tile t at 128 + 128 t + 64 b
@@ -64,12 +65,12 @@ struct Smem {
   unsigned long long kv_full[kStages], kv_empty[kStages];
   unsigned long long q_full[2][2], q_empty[2][2];  // [item parity][tile]
   unsigned long long s_full[2][2], p_full[2][2], pv_done[2][2];  // [tile][S buffer]
-  unsigned long long list_full[2], list_empty[2];
+  unsigned long long list_full[kLists], list_empty[kLists];
   uint32_t tmem_base;
   int abort;
-  ItemInfo info[2];
-  int ids[2][kMaxUnion];
-  unsigned char mask[2][kMaxUnion];
+  ItemInfo info[kLists];
+  int ids[kLists][kMaxUnion];
+  unsigned char mask[kLists][kMaxUnion];
   int tmp_ids[kMaxUnion];            // planner scratch: merged list before reordering
   unsigned char tmp_mask[kMaxUnion];
 };
@@ -316,8 +317,7 @@ __host__ __device__ inline int items_per_unit(const Geo& g) {
 
 // Warp-cooperative attended list of query block i (local set, then valid selected ids) written to
 // ids[n0..); returns the new count.
-__device__ __forceinline__ int warp_attended(const Geo& g, const int32_t* __restrict__ idx_row, int i, int* ids,
-                                             int n0, int lane, int* status) {
+__device__ __forceinline__ int warp_attended(const Geo& g, int j, int i, int* ids, int n0, int lane, int* status) {
   const int by = i / g.nbw, bx = i - by * g.nbw;
   const int wl = 2 * g.rlon + 1, nl = (2 * g.rlat + 1) * wl;
   int id = -1 - lane;
@@ -333,7 +333,6 @@ __device__ __forceinline__ int warp_attended(const Geo& g, const int32_t* __rest
   const unsigned km = __ballot_sync(0xffffffffu, keep);
   if (keep) ids[n0 + __popc(km & ((1u << lane) - 1u))] = id;
   int n = n0 + __popc(km);
-  int j = lane < g.topk ? __ldg(idx_row + lane) : -1;
   if (j < -1 || j >= g.m) { set_status(status, MOSAIC_E_DEVICE_BAD_INDEX); j = -1; }
   const unsigned sm_ = __ballot_sync(0xffffffffu, j >= 0);
   if (j >= 0) ids[n + __popc(sm_ & ((1u << lane) - 1u))] = j;
@@ -342,12 +341,11 @@ __device__ __forceinline__ int warp_attended(const Geo& g, const int32_t* __rest
 
 // Merge the attended list of query block `blk` into the item's list (ids/mask, n entries so far):
 // entries already present get `bits` OR-ed into their mask, new ones are appended.  Returns the new n.
-__device__ __forceinline__ int merge_block(const Geo& g, const int32_t* __restrict__ block_idx, int u, int blk,
-                                           unsigned char bits, int* ids, unsigned char* mask, int n, int lane,
-                                           int* status) {
-  const int32_t* row = block_idx + ((long long)u * g.m + blk) * g.topk;
+// `jsel` is this lane's entry of the block's row of block_idx (-1 beyond top-k).
+__device__ __forceinline__ int merge_block(const Geo& g, int jsel, int blk, unsigned char bits, int* ids,
+                                           unsigned char* mask, int n, int lane, int* status) {
   const int n0 = n;
-  const int nb = warp_attended(g, row, blk, ids, n0, lane, status) - n0;  // staged behind the list
+  const int nb = warp_attended(g, jsel, blk, ids, n0, lane, status) - n0;  // staged behind the list
   __syncwarp();
   if (n0 == 0) {
     for (int e = lane; e < nb; e += 32) mask[e] = bits;
@@ -460,8 +458,10 @@ __global__ void __launch_bounds__(kThreads, 1)
         mbar_init(s32(&sm.p_full[t][b]), 128);
         mbar_init(s32(&sm.pv_done[t][b]), 1);
       }
-      mbar_init(s32(&sm.list_full[t]), 1);
-      mbar_init(s32(&sm.list_empty[t]), 11);  // 8 softmax warps + 2 MMA warps + TMA producer
+    }
+    for (int i = 0; i < kLists; ++i) {
+      mbar_init(s32(&sm.list_full[i]), 1);
+      mbar_init(s32(&sm.list_empty[i]), 11);  // 8 softmax warps + 2 MMA warps + TMA producer
     }
     sm.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -484,12 +484,12 @@ __global__ void __launch_bounds__(kThreads, 1)
   if (warp == 11) {
     // ------------------------------------------------------------- planner: work queue + key lists
     for (int it = 0;; ++it) {
-      const int buf = it & 1;
+      const int buf = it % kLists;
       int item = 0;
       if (lane == 0) item = atomicAdd(work_counter, 1);
       item = __shfl_sync(0xffffffffu, item, 0);
       bool ok = true;
-      if (lane == 0) ok = mbar_wait(s32(&sm.list_empty[buf]), ((it >> 1) & 1) ^ 1, abort, status);
+      if (lane == 0) ok = mbar_wait(s32(&sm.list_empty[buf]), ((it / kLists) & 1) ^ 1, abort, status);
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
       if (item >= total_items) {
@@ -499,6 +499,10 @@ __global__ void __launch_bounds__(kThreads, 1)
       const int u = item / ipu;
       int hb[4], hc[4];
       const int valid = item_halves(g, item - u * ipu, hb, hc);
+      int jsel[4];  // the four rows of block_idx, fetched together
+#pragma unroll
+      for (int h = 0; h < 4; ++h)
+        jsel[h] = lane < g.topk ? __ldg(block_idx + ((long long)u * g.m + hb[h]) * g.topk + lane) : -1;
       int n = 0;
 #pragma unroll
       for (int h = 0; h < 4; ++h) {
@@ -512,7 +516,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             bits |= (unsigned char)(1 << h2);
           }
         }
-        if (first) n = merge_block(g, block_idx, u, hb[h], bits, sm.tmp_ids, sm.tmp_mask, n, lane, status);
+        if (first) n = merge_block(g, jsel[h], hb[h], bits, sm.tmp_ids, sm.tmp_mask, n, lane, status);
       }
       interleave_tiles(sm.tmp_ids, sm.tmp_mask, n, sm.ids[buf], sm.mask[buf], lane);
       if (lane == 0) {
@@ -530,8 +534,8 @@ __global__ void __launch_bounds__(kThreads, 1)
       long long step = 0;  // key/value chunks issued so far (ring position)
       bool ok = true;
       for (int it = 0; ok; ++it) {
-        const int buf = it & 1;
-        ok = mbar_wait(s32(&sm.list_full[buf]), (it >> 1) & 1, abort, status);
+        const int buf = it % kLists, qb = it & 1;
+        ok = mbar_wait(s32(&sm.list_full[buf]), (it / kLists) & 1, abort, status);
         if (!ok) break;
         const ItemInfo& inf = sm.info[buf];
         const int n = inf.n, u = inf.unit;
@@ -539,12 +543,12 @@ __global__ void __launch_bounds__(kThreads, 1)
         // query tiles (double-buffered by item parity): free once the tile's last QK^T of the item before
         // the previous one has completed, so this load runs while the previous item still computes
         for (int t = 0; t < 2 && ok; ++t) {
-          ok = mbar_wait(s32(&sm.q_empty[buf][t]), ((it >> 1) & 1) ^ 1, abort, status);
+          ok = mbar_wait(s32(&sm.q_empty[qb][t]), ((it >> 1) & 1) ^ 1, abort, status);
           if (!ok) break;
-          mbar_expect_tx(s32(&sm.q_full[buf][t]), 2 * kTile);
+          mbar_expect_tx(s32(&sm.q_full[qb][t]), 2 * kTile);
           for (int hh = 0; hh < 2; ++hh) {
             const int h = 2 * t + hh, by = inf.hb[h] / g.nbw, bx = inf.hb[h] - by * g.nbw;
-            tma_load_4d(s32(sm.q[buf][t] + hh * kTile), &map_q, s32(&sm.q_full[buf][t]), 0, bx * g.bw,
+            tma_load_4d(s32(sm.q[qb][t] + hh * kTile), &map_q, s32(&sm.q_full[qb][t]), 0, bx * g.bw,
                         by * g.bh + inf.hc[h] * g.crows, u);
           }
         }
@@ -601,8 +605,8 @@ __global__ void __launch_bounds__(kThreads, 1)
       __syncwarp();
     };
     for (int it = 0; ok; ++it) {
-      const int buf = it & 1;
-      ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.list_full[buf]), (it >> 1) & 1, abort, status));
+      const int buf = it % kLists, qb = it & 1;
+      ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.list_full[buf]), (it / kLists) & 1, abort, status));
       if (!ok) break;
       const int n = sm.info[buf].n;
       if (n < 0) break;
@@ -610,10 +614,10 @@ __global__ void __launch_bounds__(kThreads, 1)
       for (int e = 0; e < n; ++e)
         if (sm.mask[buf][e] & tbits) last = e;
       // the query tile is loaded for every item; it must have landed before its buffer is handed back
-      ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.q_full[buf][t]), (it >> 1) & 1, abort, status));
-      const uint64_t qdesc = smem_desc(s32(sm.q[buf][t]));
+      ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.q_full[qb][t]), (it >> 1) & 1, abort, status));
+      const uint64_t qdesc = smem_desc(s32(sm.q[qb][t]));
       if (!ok) break;
-      if (last < 0 && elect_one()) mbar_arrive(s32(&sm.q_empty[buf][t]));
+      if (last < 0 && elect_one()) mbar_arrive(s32(&sm.q_empty[qb][t]));
       bool first = true, pend = false, pend_first = false;
       uint32_t pend_n = 0;
       int pend_st = 0;
@@ -640,7 +644,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             for (int kk = 0; kk < 4; ++kk)
               umma_ss(tcol_s + 64 * b, qdesc + 2 * kk, kdesc + 2 * kk, idesc_qk, kk > 0);
             tc_commit(s32(&sm.s_full[t][b]));
-            if (release_q) tc_commit(s32(&sm.q_empty[buf][t]));
+            if (release_q) tc_commit(s32(&sm.q_empty[qb][t]));
           }
           __syncwarp();
           if (pend) issue_pv(pend_n, pend_st, pend_first);
@@ -664,8 +668,8 @@ __global__ void __launch_bounds__(kThreads, 1)
     uint32_t nt = 0;
     bool ok = true;
     for (int it = 0; ok; ++it) {
-      const int buf = it & 1;
-      ok = mbar_wait(s32(&sm.list_full[buf]), (it >> 1) & 1, abort, status);
+      const int buf = it % kLists;
+      ok = mbar_wait(s32(&sm.list_full[buf]), (it / kLists) & 1, abort, status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       const int n = sm.info[buf].n;

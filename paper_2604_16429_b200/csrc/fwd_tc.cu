@@ -49,6 +49,7 @@ constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColO = 0, kColS = 128;       // O of tile t at 64 t; S buffer b of tile t at 128 + 128 t + 64 b
 constexpr long long kSpinCycles = 4000000000ll;  // bound of a single wait (~2 s)
 constexpr int kPolyEvery = 2;                   // one pair in every kPolyEvery groups of four logits takes the FMA-pipe exp2
+constexpr uint32_t kSuspendHintNs = 20000;       // longest park of one mbarrier poll
 constexpr float kRescaleThreshold = 8.0f;        // log2 units: P stays below 2^8
 
 struct ItemInfo {
@@ -86,12 +87,14 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// One poll.  The time hint lets the hardware park the thread for up to that long (it wakes as soon as the
+// phase completes), so warps that wait do not take issue slots from warps that work.
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
-      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity)
+      : "r"(bar), "r"(parity), "r"(kSuspendHintNs)
       : "memory");
   return ok != 0;
 }
@@ -486,7 +489,8 @@ __global__ void __launch_bounds__(kThreads, 1)
     for (int it = 0;; ++it) {
       const int buf = it % kLists;
       int item = 0;
-      if (lane == 0) item = atomicAdd(work_counter, 1);
+      // the first item of a CTA is its own index; later ones come from the queue, which counts from 0
+      if (lane == 0) item = it == 0 ? (int)blockIdx.x : atomicAdd(work_counter, 1) + (int)gridDim.x;
       item = __shfl_sync(0xffffffffu, item, 0);
       bool ok = true;
       if (lane == 0) ok = mbar_wait(s32(&sm.list_empty[buf]), ((it / kLists) & 1) ^ 1, abort, status);

@@ -64,8 +64,6 @@ __global__ void __launch_bounds__(256) pool_kernel(Geo g, const uint4* __restric
 // Merge: one warp per query row keeps the sorted k-entry list, one entry per lane; the rows of a warp
 // advance in lockstep so that their reductions overlap.
 // ------------------------------------------------------------------------------------------
-constexpr int JT = 64;
-constexpr int KSTR = JT + 1;  // padded row of the key tile: conflict-free transposing stores
 
 // Total-order key: larger key = better score.  0 = not a candidate, 1 = NaN.
 __device__ __forceinline__ unsigned long long score_key(double s) {
@@ -80,8 +78,9 @@ __device__ __forceinline__ bool ranks_before(unsigned long long ka, int ia, unsi
   return ka > kb || (ka == kb && ia < ib);
 }
 
-template <int TI>
+template <int TI, int JT>
 struct TopkSmem {
+  static constexpr int KSTR = JT + 1;  // padded row of the key tile: conflict-free transposing stores
   double qs[kD][TI];                   // pooled queries of this CTA, channel-major
   double ks[kD][KSTR];                 // pooled keys of the current chunk, channel-major
   unsigned long long keys[TI][JT];     // candidate keys of the current chunk (0 = none)
@@ -90,11 +89,12 @@ struct TopkSmem {
   short iy[TI], ix[TI], jy[JT], jx[JT];  // block coordinates of the rows and of the chunk's keys
 };
 
-template <int TI>
+template <int TI, int JT>
 __global__ void __launch_bounds__(256) topk_kernel(Geo g, const float* __restrict__ pq,
                                                    const float* __restrict__ pk, int32_t* __restrict__ block_idx) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  TopkSmem<TI>& sm = *reinterpret_cast<TopkSmem<TI>*>(smem_raw);
+  TopkSmem<TI, JT>& sm = *reinterpret_cast<TopkSmem<TI, JT>*>(smem_raw);
+  constexpr int RJ = JT / 16;                 // keys per thread
   constexpr int RI = TI / 16;                 // query rows per thread
   constexpr int RPW = TI / 8;                 // query rows per warp in the merge
 
@@ -143,22 +143,22 @@ __global__ void __launch_bounds__(256) topk_kernel(Geo g, const float* __restric
     for (int r = tid; r < TI; r += 256) sm.flag[r] = 0;
     __syncthreads();
     {
-      double acc[RI][4];
+      double acc[RI][RJ];
 #pragma unroll
       for (int a = 0; a < RI; ++a)
 #pragma unroll
-        for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
+        for (int b = 0; b < RJ; ++b) acc[a][b] = 0.0;
 #pragma unroll 8
       for (int c = 0; c < kD; ++c) {
-        double qv[RI], kv[4];
+        double qv[RI], kv[RJ];
 #pragma unroll
         for (int a = 0; a < RI; ++a) qv[a] = sm.qs[c][ty + 16 * a];
 #pragma unroll
-        for (int b = 0; b < 4; ++b) kv[b] = sm.ks[c][tx + 16 * b];
+        for (int b = 0; b < RJ; ++b) kv[b] = sm.ks[c][tx + 16 * b];
 #pragma unroll
         for (int a = 0; a < RI; ++a)
 #pragma unroll
-          for (int b = 0; b < 4; ++b) acc[a][b] = fma(qv[a], kv[b], acc[a][b]);
+          for (int b = 0; b < RJ; ++b) acc[a][b] = fma(qv[a], kv[b], acc[a][b]);
       }
 #pragma unroll
       for (int a = 0; a < RI; ++a) {
@@ -167,7 +167,7 @@ __global__ void __launch_bounds__(256) topk_kernel(Geo g, const float* __restric
         const int iy = sm.iy[r], ix = sm.ix[r];
         bool any = false;
 #pragma unroll
-        for (int b = 0; b < 4; ++b) {
+        for (int b = 0; b < RJ; ++b) {
           const int jj = tx + 16 * b;
           int dx = sm.jx[jj] - ix;
           dx += dx < 0 ? g.nbw : 0;  // (jx - ix) mod nbw
@@ -251,14 +251,14 @@ __global__ void __launch_bounds__(256) topk_kernel(Geo g, const float* __restric
   }
 }
 
-template <int TI>
+template <int TI, int JT>
 int launch_topk(const HostCtx& c, const float* pooled_q, const float* pooled_k, int32_t* block_idx) {
   const Geo& g = c.g;
-  const size_t smem = sizeof(TopkSmem<TI>);
-  if (cudaFuncSetAttribute(topk_kernel<TI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+  const size_t smem = sizeof(TopkSmem<TI, JT>);
+  if (cudaFuncSetAttribute(topk_kernel<TI, JT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return MOSAIC_E_CUDA;
   const int tiles = (g.m + TI - 1) / TI;
-  topk_kernel<TI><<<(unsigned)(g.U * tiles), 256, smem, c.stream>>>(g, pooled_q, pooled_k, block_idx);
+  topk_kernel<TI, JT><<<(unsigned)(g.U * tiles), 256, smem, c.stream>>>(g, pooled_q, pooled_k, block_idx);
   return cudaGetLastError() == cudaSuccess ? MOSAIC_OK : MOSAIC_E_CUDA;
 }
 
@@ -277,9 +277,10 @@ int launch_select(const HostCtx& c, const void* q, const void* k, int32_t* block
   if (g.topk > 0) {
     // the most query blocks per CTA (64, 32, 16) that still gives every SM two CTAs; 16 otherwise
     auto ctas = [&](int ti) { return (long long)g.U * ((g.m + ti - 1) / ti); };
-    const int rc = ctas(64) >= 296 ? launch_topk<64>(c, pooled_q, pooled_k, block_idx)
-                 : ctas(32) >= 296 ? launch_topk<32>(c, pooled_q, pooled_k, block_idx)
-                                   : launch_topk<16>(c, pooled_q, pooled_k, block_idx);
+    // small problems (16 rows per CTA) take keys in chunks of 128 to halve the number of merge passes
+    const int rc = ctas(64) >= 296 ? launch_topk<64, 64>(c, pooled_q, pooled_k, block_idx)
+                 : ctas(32) >= 296 ? launch_topk<32, 64>(c, pooled_q, pooled_k, block_idx)
+                                   : launch_topk<16, 128>(c, pooled_q, pooled_k, block_idx);
     if (rc) return rc;
   }
   return MOSAIC_OK;

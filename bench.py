@@ -125,8 +125,9 @@ def sample_flops(w, g, blocks) -> float:
 
 
 def cpu_baseline(w, x, idx_gpu, o_gpu, lse_gpu) -> dict:
-    """Time the oracle, as it stands, on a bounded sample of the workload (about 10-30 core-seconds):
-    two whole units for 64-token blocks, 64 query blocks of one unit for larger blocks.  The sample
+    """Time the oracle, as it stands, on a bounded sample of the workload (a few seconds to about ten on 16
+    host cores): up to 40 whole units for 64-token blocks (the whole 1.5-degree workload has 8), 640 query
+    blocks of one unit for larger blocks.  The sample
     doubles as a parity spot check of the launch configuration that was just timed."""
     import oracle
     from oracle import Geom
@@ -134,11 +135,11 @@ def cpu_baseline(w, x, idx_gpu, o_gpu, lse_gpu) -> dict:
     g = Geom(w.nlat, w.nlon, d=w.d, bh=w.bh, bw=w.bw, rlat=w.rlat, rlon=w.rlon, topk=w.topk)
     rng = np.random.default_rng(0)
     if w.b <= 64:
-        units = [(u // w.H, u % w.H) for u in range(min(2, w.U))]
+        units = [(u // w.H, u % w.H) for u in range(min(40, w.U))]
         blocks = np.arange(w.m, dtype=np.int32)
     else:
         units = [(0, 0)]
-        blocks = np.sort(rng.choice(w.m, size=min(w.m, 64), replace=False)).astype(np.int32)
+        blocks = np.sort(rng.choice(w.m, size=min(w.m, 640), replace=False)).astype(np.int32)
     oracle.local_set(g, 0)                                       # load the library before timing
     fl, dt, worst = 0.0, 0.0, 0.0
     for (b, h) in units:

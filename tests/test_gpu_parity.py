@@ -21,6 +21,8 @@ SELECT_CASES = [
     synth.small_case(40, 48, 8, 8, 5, B=1, H=3, seed=24, rlat=2, rlon=1),
     synth.small_case(32, 16, 8, 8, 2, B=1, H=1, seed=25),                       # 2 block columns: neighbourhood de-duplicates
     synth.small_case(48, 64, 8, 8, 0, B=1, H=1, seed=26, rlat=0, rlon=0),       # nothing selected
+    synth.small_case(240, 320, 8, 8, 8, B=1, H=8, kind="smooth", seed=28),      # m = 1200, 8 units: the 32-rows-per-CTA ranking path
+    synth.small_case(32, 64, 8, 16, 3, B=1, H=1, kind="smooth", seed=29),       # 8 x 16 blocks
 ]
 
 
@@ -56,6 +58,12 @@ FWD_CASES = [
     (synth.small_case(48, 64, 8, 8, 0, B=1, H=1, seed=33, rlat=0, rlon=0), 0.0),   # block-diagonal
     (synth.small_case(40, 48, 8, 8, 6, B=2, H=1, kind="smooth", seed=34, rlat=2, rlon=2), 0.3),
     (synth.small_case(16, 16, 8, 8, 4, B=1, H=1, seed=35), 0.0),                # 2x2 blocks: everything local, all -1
+    # every way a 256-row work item is put together
+    (synth.small_case(40, 56, 8, 8, 5, B=1, H=2, kind="smooth", seed=51), 0.0),   # 5 x 7 blocks: odd last row (1x4 groups), odd width
+    (synth.small_case(32, 64, 8, 16, 3, B=1, H=1, kind="smooth", seed=52), 0.0),  # 128-token blocks (8 x 16): two blocks per item
+    (synth.small_case(48, 40, 16, 8, 2, B=1, H=2, seed=53), 0.0),                  # 128-token blocks (16 x 8), 5 block columns: lone block
+    (synth.small_case(64, 32, 32, 8, 2, B=1, H=1, seed=54), 0.0),                  # 256-token blocks (32 x 8): one item per block
+    (synth.small_case(48, 64, 24, 16, 2, B=1, H=1, kind="smooth", seed=55), 0.0), # 384-token blocks: second item of a block is half empty
 ]
 
 
@@ -124,6 +132,8 @@ BWD_CASES = [
     synth.small_case(24, 40, 8, 8, 3, B=1, H=1, kind="smooth", seed=42, backward=True),
     synth.small_case(32, 64, 16, 16, 2, B=1, H=1, kind="smooth", seed=43, backward=True),
     synth.small_case(48, 64, 8, 8, 0, B=1, H=1, seed=44, rlat=0, rlon=0, backward=True),
+    synth.small_case(32, 64, 8, 16, 3, B=1, H=1, kind="smooth", seed=46, backward=True),   # 128-token blocks
+    synth.small_case(40, 56, 8, 8, 5, B=1, H=1, kind="smooth", seed=47, backward=True),    # odd block grid
 ]
 
 

@@ -362,6 +362,7 @@ __device__ __forceinline__ int merge_block(const Geo& g, int jsel, int blk, unsi
     mine[r] = e < nb ? ids[n0 + e] : -1;
     pos[r] = -1;
   }
+#pragma unroll 8
   for (int a = 0; a < n0; ++a) {
     const int id = ids[a];
     pos[0] = id == mine[0] ? a : pos[0];
@@ -422,11 +423,13 @@ __device__ __forceinline__ void interleave_tiles(const int* sid, const unsigned 
       for (int y = 0; y < 3; ++y) {
         if (y == cls) continue;
         const int ny = y == 0 ? c0 : y == 1 ? c1 : c2;
-        const int T = (4 * k + cls) * ny;
-        for (int j = 0; j < ny; ++j) {
-          const int v = (4 * j + y) * nx;
-          pos += (v < T || (v == T && y < cls)) ? 1 : 0;
-        }
+        if (ny == 0) continue;
+        // entries j of class y that come first: (4j + y) nx < (4k + cls) ny, ties to the lower class
+        const int R = (4 * k + cls) * ny - y * nx;  // 4 j nx < R, or <= R when y < cls
+        int cnt = 0;
+        if (y < cls) cnt = R >= 0 ? R / (4 * nx) + 1 : 0;
+        else cnt = R > 0 ? (R + 4 * nx - 1) / (4 * nx) : 0;
+        pos += min(cnt, ny);
       }
       did[pos] = sid[e];
       dmask[pos] = (unsigned char)m;

@@ -6,7 +6,8 @@
 // log-sum-exp, following the memory-efficient formulation the paper adopts).
 //
 // With w = exp(scale*q.k - LSE), dP = dO.v, D = dO.O, dS = w*(dP - D):
-//   dQ_l = scale * sum_t dS_lt k_t       (query-block stationary, same traversal as the forward)
+//   dQ_l = scale * sum_t dS_lt k_t       (query-block stationary, same traversal as the forward;
+//                                         tensor-core kernel in bwd_dq_tc.cu)
 //   dV_t = sum_l w_lt dO_l ; dK_t = scale * sum_l dS_lt q_l   (key-block stationary over the
 //          transposed pattern: local neighbours by geometry + a CSR list of selecting query blocks)
 // Summation order is fixed (no floating-point atomics), so results are deterministic.
@@ -89,93 +90,6 @@ __global__ void __launch_bounds__(256) csr_kernel(Geo g, const int32_t* __restri
       }
       __syncwarp();
     }
-  }
-}
-
-// ------------------------------------------------------------------------------------------
-// dQ kernel: one CTA (4 warps x 16 rows) per 64-row query tile; streams the attended chunks.
-// ------------------------------------------------------------------------------------------
-struct RowFrag {  // this thread's two rows of a 16-row warp tile: lane/4 and lane/4 + 8
-  float v[2];
-};
-
-__global__ void __launch_bounds__(128) dq_kernel(Geo g, const __nv_bfloat16* __restrict__ q,
-                                                 const __nv_bfloat16* __restrict__ k,
-                                                 const __nv_bfloat16* __restrict__ v,
-                                                 const __nv_bfloat16* __restrict__ d_o,
-                                                 const float* __restrict__ lse, const float* __restrict__ D,
-                                                 const int32_t* __restrict__ block_idx,
-                                                 __nv_bfloat16* __restrict__ dq, int* status) {
-  __shared__ __align__(128) unsigned char tiles[4 * kTileBytes];
-  __shared__ int list[kMaxList];
-  __shared__ int nlist;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int qc = blockIdx.x % g.cpb;
-  const int i = (blockIdx.x / g.cpb) % g.m;
-  const int u = blockIdx.x / (g.cpb * g.m);
-  const long long ubase = (long long)u * g.N;
-  const uint32_t Qs = smem_u32(tiles), dOs = Qs + kTileBytes, Ks = dOs + kTileBytes, Vs = Ks + kTileBytes;
-
-  if (tid == 0) nlist = attended_list(g, block_idx + ((long long)u * g.m + i) * g.topk, i, list, status);
-  load_tile<128>(Qs, q + ubase * kD, g, i, qc, tid);
-  load_tile<128>(dOs, d_o + ubase * kD, g, i, qc, tid);
-  cp_async_commit();
-  cp_async_wait<0>();
-  __syncthreads();
-
-  uint32_t qa[4][4], da[4][4];
-#pragma unroll
-  for (int kk = 0; kk < 4; ++kk) {
-    load_A(Qs, warp * 16, kk, lane, qa[kk]);
-    load_A(dOs, warp * 16, kk, lane, da[kk]);
-  }
-  const int r0 = warp * 16 + (lane >> 2);
-  const long long tok0 = ubase + chunk_token(g, i, qc, r0), tok1 = ubase + chunk_token(g, i, qc, r0 + 8);
-  const float lse0 = lse[tok0] * kLog2e, lse1 = lse[tok1] * kLog2e;
-  const float D0 = D[tok0], D1 = D[tok1];
-
-  float acc[8][4];
-#pragma unroll
-  for (int n = 0; n < 8; ++n)
-#pragma unroll
-    for (int e = 0; e < 4; ++e) acc[n][e] = 0.f;
-
-  const int nchunks = nlist * g.cpb;
-  for (int it = 0; it < nchunks; ++it) {
-    const int j = list[it / g.cpb], c = it % g.cpb;
-    __syncthreads();  // all warps finished with the previous K/V tiles
-    load_tile<128>(Ks, k + ubase * kD, g, j, c, tid);
-    load_tile<128>(Vs, v + ubase * kD, g, j, c, tid);
-    cp_async_commit();
-    cp_async_wait<0>();
-    __syncthreads();
-
-    float s[8][4], dp[8][4];
-#pragma unroll
-    for (int n = 0; n < 8; ++n)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) { s[n][e] = 0.f; dp[n][e] = 0.f; }
-    gemm_nt(s, qa, Ks, lane);
-    gemm_nt(dp, da, Vs, lane);
-#pragma unroll
-    for (int n = 0; n < 8; ++n) {
-      float p0 = exp2f(s[n][0] * g.scale_log2 - lse0), p1 = exp2f(s[n][1] * g.scale_log2 - lse0);
-      float p2 = exp2f(s[n][2] * g.scale_log2 - lse1), p3 = exp2f(s[n][3] * g.scale_log2 - lse1);
-      s[n][0] = p0 * (dp[n][0] - D0);
-      s[n][1] = p1 * (dp[n][1] - D0);
-      s[n][2] = p2 * (dp[n][2] - D1);
-      s[n][3] = p3 * (dp[n][3] - D1);
-    }
-    uint32_t dsa[4][4];
-    acc_to_A(s, dsa);
-    gemm_nn(acc, dsa, Ks, lane);
-  }
-  __nv_bfloat16* out0 = dq + tok0 * kD + 2 * (lane & 3);
-  __nv_bfloat16* out1 = dq + tok1 * kD + 2 * (lane & 3);
-#pragma unroll
-  for (int n = 0; n < 8; ++n) {
-    *reinterpret_cast<uint32_t*>(out0 + 8 * n) = pack_bf16(acc[n][0] * g.scale, acc[n][1] * g.scale);
-    *reinterpret_cast<uint32_t*>(out1 + 8 * n) = pack_bf16(acc[n][2] * g.scale, acc[n][3] * g.scale);
   }
 }
 
@@ -304,10 +218,12 @@ int launch_bwd(const HostCtx& c, const void* q, const void* k, const void* v, co
   }
   if (cudaGetLastError() != cudaSuccess) return MOSAIC_E_CUDA;
   const unsigned grid = (unsigned)((long long)g.U * g.m * g.cpb);
-  dq_kernel<<<grid, 128, 0, c.stream>>>(g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k,
-                                        (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, lse, Dbuf, block_idx,
-                                        (__nv_bfloat16*)dq, c.status);
-  if (cudaGetLastError() != cudaSuccess) return MOSAIC_E_CUDA;
+  {
+    // dQ on the tcgen05 path; its work queue counts in the second word of the status block (zeroed when the
+    // op started)
+    const int rc = launch_dq_tc(c, q, k, v, d_o, lse, Dbuf, block_idx, dq, c.status + 1);
+    if (rc) return rc;
+  }
   dkdv_kernel<<<grid, 128, 0, c.stream>>>(g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k,
                                           (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, lse, Dbuf, csr_off,
                                           csr_q, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv);

@@ -104,6 +104,8 @@ int launch_select(const HostCtx& c, const void* q, const void* k, int32_t* block
                   float* pooled_k);
 int launch_fwd_tc(const HostCtx& c, const void* q, const void* k, const void* v, const int32_t* block_idx,
                   void* o, float* lse);
+int launch_dq_tc(const HostCtx& c, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
+                 const float* D, const int32_t* block_idx, void* dq, int* work_counter);
 int launch_bwd(const HostCtx& c, const void* q, const void* k, const void* v, const void* o, const float* lse,
                const void* d_o, const int32_t* block_idx, void* dq, void* dk, void* dv, float* Dbuf,
                int32_t* csr_off, int32_t* csr_cur, int32_t* csr_q);

@@ -40,13 +40,14 @@ int validate(const mosaic_bsa_params* p, Geo* g) {
 
 namespace {
 
-struct BwdWs { size_t D, off, cur, q, total; };
+struct BwdWs { size_t D, negD, nlse2, off, q, total; };
 BwdWs bwd_layout(const Geo& g) {
   BwdWs w;
   size_t at = kStatusBytes;
   w.D = at; at = align256(at + sizeof(float) * (size_t)g.U * g.N);
+  w.negD = at; at = align256(at + sizeof(float) * (size_t)g.U * g.N);
+  w.nlse2 = at; at = align256(at + sizeof(float) * (size_t)g.U * g.N);
   w.off = at; at = align256(at + sizeof(int32_t) * (size_t)g.U * (g.m + 1));
-  w.cur = at;  // reserved
   w.q = at; at = align256(at + sizeof(int32_t) * (size_t)g.U * g.m * (g.topk > 0 ? g.topk : 1));
   w.total = at;
   return w;
@@ -143,7 +144,8 @@ int mosaic_bsa_bwd(const mosaic_bsa_params* p, const void* q, const void* k, con
   if ((rc = begin(p, ws, ws_bytes, w.total, cuda_stream, &c))) return rc;
   char* base = (char*)ws;
   return launch_bwd(c, q, k, v, o, lse, d_o, block_idx, dq, dk, dv, (float*)(base + w.D),
-                    (int32_t*)(base + w.off), (int32_t*)(base + w.cur), (int32_t*)(base + w.q));
+                    (float*)(base + w.negD), (float*)(base + w.nlse2), (int32_t*)(base + w.off),
+                    (int32_t*)(base + w.q));
 }
 
 int mosaic_bsa_last_status(const void* ws, void* cuda_stream) {

@@ -9,19 +9,23 @@
 //   dQ_l = scale * sum_t dS_lt k_t       (query-block stationary, same traversal as the forward;
 //                                         tensor-core kernel in bwd_dq_tc.cu)
 //   dV_t = sum_l w_lt dO_l ; dK_t = scale * sum_l dS_lt q_l   (key-block stationary over the
-//          transposed pattern: local neighbours by geometry + a CSR list of selecting query blocks)
+//          transposed pattern: local neighbours by geometry + a CSR list of selecting query blocks;
+//          tensor-core kernel in bwd_dkdv_tc.cu)
 // Summation order is fixed (no floating-point atomics), so results are deterministic.
-#include "mma_util.cuh"
+#include "common.cuh"
 
 namespace mosaic {
 
 constexpr float kLog2e = 1.4426950408889634f;
 
 // ------------------------------------------------------------------------------------------
-// D_l = sum_c dO_lc * O_lc.  HBM-bound: 8 lanes per token, 16 bytes of each tensor per lane.
+// D_l = sum_c dO_lc * O_lc (also stored negated, with the negated base-2 log-sum-exp beside it).
+// HBM-bound: 8 lanes per token, 16 bytes of each tensor per lane.
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) rowdot_kernel(long long tokens, const uint4* __restrict__ o,
-                                                     const uint4* __restrict__ d_o, float* __restrict__ D) {
+                                                     const uint4* __restrict__ d_o, const float* __restrict__ lse,
+                                                     float* __restrict__ D, float* __restrict__ neg_d,
+                                                     float* __restrict__ neg_lse2) {
   long long t = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 3;
   int part = threadIdx.x & 7;
   float acc = 0.f;
@@ -37,7 +41,11 @@ __global__ void __launch_bounds__(256) rowdot_kernel(long long tokens, const uin
   acc += __shfl_xor_sync(0xffffffffu, acc, 1);
   acc += __shfl_xor_sync(0xffffffffu, acc, 2);
   acc += __shfl_xor_sync(0xffffffffu, acc, 4);
-  if (part == 0 && t < tokens) D[t] = acc;
+  if (part == 0 && t < tokens) {
+    D[t] = acc;
+    neg_d[t] = -acc;                     // the key-stationary kernel reads these per query column
+    neg_lse2[t] = -lse[t] * kLog2e;      // log-sum-exp in base-2 units, negated
+  }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -93,116 +101,16 @@ __global__ void __launch_bounds__(256) csr_kernel(Geo g, const int32_t* __restri
   }
 }
 
-// ------------------------------------------------------------------------------------------
-// dK/dV kernel: one CTA per 64-token key/value chunk; visits the connected query blocks in a
-// fixed order (local neighbours by geometry -- the neighbourhood relation is symmetric -- then
-// the ascending CSR list) and accumulates dK, dV in registers.
-// ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(128) dkdv_kernel(Geo g, const __nv_bfloat16* __restrict__ q,
-                                                   const __nv_bfloat16* __restrict__ k,
-                                                   const __nv_bfloat16* __restrict__ v,
-                                                   const __nv_bfloat16* __restrict__ d_o,
-                                                   const float* __restrict__ lse, const float* __restrict__ D,
-                                                   const int32_t* __restrict__ csr_off,
-                                                   const int32_t* __restrict__ csr_q,
-                                                   __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv) {
-  __shared__ __align__(128) unsigned char tiles[4 * kTileBytes];
-  __shared__ float lse_s[kChunk], D_s[kChunk];
-  __shared__ int loc[kMaxList];
-  __shared__ int nloc;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int c = blockIdx.x % g.cpb;
-  const int j = (blockIdx.x / g.cpb) % g.m;
-  const int u = blockIdx.x / (g.cpb * g.m);
-  const long long ubase = (long long)u * g.N;
-  const uint32_t Ks = smem_u32(tiles), Vs = Ks + kTileBytes, Qs = Vs + kTileBytes, dOs = Qs + kTileBytes;
-
-  if (tid == 0) nloc = local_set(g, j, loc);
-  load_tile<128>(Ks, k + ubase * kD, g, j, c, tid);
-  load_tile<128>(Vs, v + ubase * kD, g, j, c, tid);
-  cp_async_commit();
-  cp_async_wait<0>();
-  __syncthreads();
-  uint32_t ka[4][4], va[4][4];
-#pragma unroll
-  for (int kk = 0; kk < 4; ++kk) {
-    load_A(Ks, warp * 16, kk, lane, ka[kk]);
-    load_A(Vs, warp * 16, kk, lane, va[kk]);
-  }
-  float acck[8][4], accv[8][4];
-#pragma unroll
-  for (int n = 0; n < 8; ++n)
-#pragma unroll
-    for (int e = 0; e < 4; ++e) { acck[n][e] = 0.f; accv[n][e] = 0.f; }
-
-  const int32_t* offs = csr_off + (long long)u * (g.m + 1);
-  const int s_beg = offs[j], s_end = offs[j + 1];
-  const int32_t* sel = csr_q + (long long)u * g.m * g.topk;
-  const int nq = nloc + (s_end - s_beg);
-
-  for (int qi = 0; qi < nq; ++qi) {
-    const int i = qi < nloc ? loc[qi] : sel[s_beg + qi - nloc];
-    for (int qc = 0; qc < g.cpb; ++qc) {
-      __syncthreads();
-      load_tile<128>(Qs, q + ubase * kD, g, i, qc, tid);
-      load_tile<128>(dOs, d_o + ubase * kD, g, i, qc, tid);
-      cp_async_commit();
-      if (tid < kChunk) {
-        long long t = ubase + chunk_token(g, i, qc, tid);
-        lse_s[tid] = lse[t] * kLog2e;
-        D_s[tid] = D[t];
-      }
-      cp_async_wait<0>();
-      __syncthreads();
-
-      float st[8][4], dpt[8][4];
-#pragma unroll
-      for (int n = 0; n < 8; ++n)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) { st[n][e] = 0.f; dpt[n][e] = 0.f; }
-      gemm_nt(st, ka, Qs, lane);    // S^T = K Q^T : rows = keys, columns = queries
-      gemm_nt(dpt, va, dOs, lane);  // dP^T = V dO^T
-      uint32_t pa[4][4];
-#pragma unroll
-      for (int n = 0; n < 8; ++n) {
-        const int col = 8 * n + 2 * (lane & 3);
-        const float l0 = lse_s[col], l1 = lse_s[col + 1], d0 = D_s[col], d1 = D_s[col + 1];
-        float p0 = exp2f(st[n][0] * g.scale_log2 - l0), p1 = exp2f(st[n][1] * g.scale_log2 - l1);
-        float p2 = exp2f(st[n][2] * g.scale_log2 - l0), p3 = exp2f(st[n][3] * g.scale_log2 - l1);
-        dpt[n][0] = p0 * (dpt[n][0] - d0);
-        dpt[n][1] = p1 * (dpt[n][1] - d1);
-        dpt[n][2] = p2 * (dpt[n][2] - d0);
-        dpt[n][3] = p3 * (dpt[n][3] - d1);
-        st[n][0] = p0; st[n][1] = p1; st[n][2] = p2; st[n][3] = p3;
-      }
-      acc_to_A(st, pa);
-      gemm_nn(accv, pa, dOs, lane);  // dV += P^T dO
-      acc_to_A(dpt, pa);
-      gemm_nn(acck, pa, Qs, lane);   // dK += dS^T Q
-    }
-  }
-  const int r0 = warp * 16 + (lane >> 2);
-  const long long tok0 = ubase + chunk_token(g, j, c, r0), tok1 = ubase + chunk_token(g, j, c, r0 + 8);
-#pragma unroll
-  for (int n = 0; n < 8; ++n) {
-    const int col = 8 * n + 2 * (lane & 3);
-    *reinterpret_cast<uint32_t*>(dk + tok0 * kD + col) = pack_bf16(acck[n][0] * g.scale, acck[n][1] * g.scale);
-    *reinterpret_cast<uint32_t*>(dk + tok1 * kD + col) = pack_bf16(acck[n][2] * g.scale, acck[n][3] * g.scale);
-    *reinterpret_cast<uint32_t*>(dv + tok0 * kD + col) = pack_bf16(accv[n][0], accv[n][1]);
-    *reinterpret_cast<uint32_t*>(dv + tok1 * kD + col) = pack_bf16(accv[n][2], accv[n][3]);
-  }
-}
-
 int launch_bwd(const HostCtx& c, const void* q, const void* k, const void* v, const void* o, const float* lse,
-               const void* d_o, const int32_t* block_idx, void* dq, void* dk, void* dv, float* Dbuf,
-               int32_t* csr_off, int32_t* csr_cur, int32_t* csr_q) {
-  (void)csr_cur;
+               const void* d_o, const int32_t* block_idx, void* dq, void* dk, void* dv, float* Dbuf, float* neg_d,
+               float* neg_lse2,
+               int32_t* csr_off, int32_t* csr_q) {
   const Geo& g = c.g;
   const long long tokens = (long long)g.U * g.N;
   {
     long long threads = tokens * 8;
     rowdot_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, c.stream>>>(tokens, (const uint4*)o,
-                                                                           (const uint4*)d_o, Dbuf);
+                                                                           (const uint4*)d_o, lse, Dbuf, neg_d, neg_lse2);
     if (cudaGetLastError() != cudaSuccess) return MOSAIC_E_CUDA;
   }
   if (g.topk > 0) {
@@ -217,17 +125,17 @@ int launch_bwd(const HostCtx& c, const void* q, const void* k, const void* v, co
       return MOSAIC_E_CUDA;
   }
   if (cudaGetLastError() != cudaSuccess) return MOSAIC_E_CUDA;
-  const unsigned grid = (unsigned)((long long)g.U * g.m * g.cpb);
   {
     // dQ on the tcgen05 path; its work queue counts in the second word of the status block (zeroed when the
     // op started)
     const int rc = launch_dq_tc(c, q, k, v, d_o, lse, Dbuf, block_idx, dq, c.status + 1);
     if (rc) return rc;
   }
-  dkdv_kernel<<<grid, 128, 0, c.stream>>>(g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k,
-                                          (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, lse, Dbuf, csr_off,
-                                          csr_q, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv);
-  if (cudaGetLastError() != cudaSuccess) return MOSAIC_E_CUDA;
+  {
+    // dK, dV on the tcgen05 path; its work queue counts in the third word of the status block
+    const int rc = launch_dkdv_tc(c, q, k, v, d_o, neg_lse2, neg_d, csr_off, csr_q, dk, dv, c.status + 2);
+    if (rc) return rc;
+  }
   return MOSAIC_OK;
 }
 

@@ -106,8 +106,11 @@ int launch_fwd_tc(const HostCtx& c, const void* q, const void* k, const void* v,
                   void* o, float* lse);
 int launch_dq_tc(const HostCtx& c, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
                  const float* D, const int32_t* block_idx, void* dq, int* work_counter);
+int launch_dkdv_tc(const HostCtx& c, const void* q, const void* k, const void* v, const void* d_o,
+                   const float* neg_lse2, const float* neg_d, const int32_t* csr_off, const int32_t* csr_q, void* dk,
+                   void* dv, int* work_counter);
 int launch_bwd(const HostCtx& c, const void* q, const void* k, const void* v, const void* o, const float* lse,
-               const void* d_o, const int32_t* block_idx, void* dq, void* dk, void* dv, float* Dbuf,
-               int32_t* csr_off, int32_t* csr_cur, int32_t* csr_q);
+               const void* d_o, const int32_t* block_idx, void* dq, void* dk, void* dv, float* Dbuf, float* neg_d,
+               float* neg_lse2, int32_t* csr_off, int32_t* csr_q);
 
 }  // namespace mosaic

@@ -23,6 +23,7 @@ struct ItemInfo {
   int hvalid;   // bit h: half h exists
   int hb[4];    // query block of half h
   int hc[4];    // 64-token chunk of that block
+  int more;     // 1: the item's list continues in the next list buffer (lists longer than a buffer)
 };
 
 __device__ __forceinline__ uint32_t s32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -438,7 +439,7 @@ __device__ __forceinline__ void planner_loop(SM& sm, const Geo& g, const int32_t
     interleave_tiles(sm.tmp_ids, sm.tmp_mask, n, sm.ids[buf], sm.mask[buf], lane);
     if (lane == 0) {
       ItemInfo& inf = sm.info[buf];
-      inf.n = n; inf.unit = u; inf.hvalid = valid;
+      inf.n = n; inf.unit = u; inf.hvalid = valid; inf.more = 0;
 #pragma unroll
       for (int h = 0; h < 4; ++h) { inf.hb[h] = hb[h]; inf.hc[h] = hc[h]; }
     }
@@ -477,6 +478,28 @@ bool make_map(CUtensorMap* map, const void* base, const Geo& g) {
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+
+// [U, nlat, nlon] fp32 view (one value per token), box = the 64 tokens of one chunk {bw, 64/bw, 1}, no swizzle.
+bool make_map_rows(CUtensorMap* map, const void* base, const Geo& g) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)g.nlon, (cuuint64_t)g.nlat, (cuuint64_t)g.U};
+  cuuint64_t strides[2] = {(cuuint64_t)g.nlon * 4, (cuuint64_t)g.N * 4};
+  cuuint32_t box[3] = {(cuuint32_t)g.bw, (cuuint32_t)g.crows, 1u};
+  cuuint32_t estr[3] = {1u, 1u, 1u};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                            int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], "
+      "[%2];" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
 }  // namespace
 
 }  // namespace mosaic

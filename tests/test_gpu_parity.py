@@ -157,6 +157,33 @@ def test_backward_matches_oracle(w):
                 assert np.abs(gh - want).mean() <= 0.1 * max(np.abs(want).mean(), 1e-3), name
 
 
+def test_backward_popular_key_blocks_lists_span_several_buffers():
+    """Two key blocks that (almost) every query block selects: their lists of connected query blocks are longer
+    than one list buffer of the key-stationary kernel, which then continues an item over several buffers."""
+    w = synth.small_case(120, 160, 8, 8, 4, B=1, H=1, seed=48, backward=True)      # m = 300
+    x = synth.make_inputs(w)
+    kf = synth.bf16_bits_to_f32(x["k"]).reshape(1, 1, 120, 160, 64).copy()
+    qf = synth.bf16_bits_to_f32(x["q"]).reshape(1, 1, 120, 160, 64).copy()
+    qf[..., 0] = np.abs(qf[..., 0]) + 1.0                       # every query likes channel 0 ...
+    kf[:, :, 56:64, 72:88, 0] = 6.0                             # ... which two neighbouring key blocks carry
+    x["k"] = synth.to_bf16_bits(kf.reshape(1, 1, -1, 64))
+    x["q"] = synth.to_bf16_bits(qf.reshape(1, 1, -1, 64))
+    dx = G.device_inputs(x)
+    idx = G.gpu_select(w, dx)
+    idx_h = idx.cpu().numpy()[0, 0]
+    popular = 7 * 20 + 9
+    assert (idx_h == popular).any(axis=1).sum() > 260           # in-degree beyond one list buffer (256 entries)
+    o, lse = G.gpu_fwd(w, dx, idx)
+    dq, dk, dv = G.gpu_bwd(w, dx, o, lse, idx)
+    dQ, dK, dV, _, _ = oracle.bwd(G.geom_of(w), x["q"][0, 0], x["k"][0, 0], x["v"][0, 0], x["do"][0, 0], idx_h)
+    for name, got, want in (("dQ", dq, dQ), ("dK", dk, dK), ("dV", dv, dV)):
+        gh = got[0, 0].float().cpu().numpy().astype(np.float64)
+        assert np.isfinite(gh).all(), name
+        # dK and dV of the popular blocks sum several hundred bf16-rounded terms: compare relative to the scale
+        err = np.abs(gh - want)
+        assert (err <= G.BWD_MAX_ABS + 1e-2 * np.abs(want)).all(), f"{name} max-abs {err.max():.4g}"
+
+
 def test_backward_is_deterministic():
     w = BWD_CASES[0]
     dx = G.device_inputs(synth.make_inputs(w))

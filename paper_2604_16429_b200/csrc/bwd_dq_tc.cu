@@ -10,10 +10,10 @@
 // 128-row tiles, four 64-row halves) from a queue; a planner warp merges the key lists of the item's
 // query blocks; a producer warp streams 64-token K and V chunks through a ring; one warp per tile issues
 // the tensor-core work; two groups of four warps (thread = query row = TMEM lane) turn S and dP into dS.
-// Per product and tile: S = Q K^T and dP = dO V^T (eight MMAs into two 64-column TMEM buffers), then the
-// row threads write dS (bf16) over the start of the dP buffer, then dQ += dS K (dS is the TMEM A operand,
-// the K chunk in shared memory is read as the MN-major B operand).  Tensor-core operations of one thread
-// execute in issue order, so the next product may overwrite S and dP without waiting for dQ += dS K.
+// Per product and tile: S = Q K^T and dP = dO V^T (eight MMAs into two 64-column TMEM buffers); the row
+// threads pull both into registers and hand the buffers back at once, so the next product's S and dP are
+// computed while they form dS (bf16, its own 32 TMEM columns); then dQ += dS K (dS is the TMEM A operand,
+// the K chunk in shared memory is read as the MN-major B operand), issued one product behind.
 // Every mbarrier wait is bounded; on expiry the CTA records MOSAIC_E_DEVICE_TIMEOUT and drains.
 #include "tc_common.cuh"
 
@@ -24,14 +24,15 @@ namespace {
 constexpr int kStages = 6;       // key/value ring depth (K + V chunk per stage)
 constexpr int kThreads = 384;
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColDQ = 0, kColS = 128;  // dQ of tile t at 64 t; S of tile t at 128 + 128 t, dP right after it
+// dQ of tile t at 64 t; S of tile t at 128 + 128 t, dP right after it; dS (bf16) of tile t at 384 + 32 t
+constexpr uint32_t kColDQ = 0, kColS = 128, kColDS = 384;
 
 struct Smem {
   unsigned char q[2][2 * kTile];           // [tile][128 rows x 128 B]
   unsigned char d_o[2][2 * kTile];         // [tile][128 rows x 128 B]
   unsigned char kv[kStages][2][kTile];     // [stage][K, V]
   unsigned long long kv_full[kStages], kv_empty[kStages];
-  unsigned long long q_full[2], q_empty[2], s_full[2], p_full[2], pv_done[2];  // [tile]
+  unsigned long long q_full[2], q_empty[2], s_full[2], sdp_free[2], p_full[2], pv_done[2];  // [tile]
   unsigned long long list_full[kLists], list_empty[kLists];
   uint32_t tmem_base;
   int abort;
@@ -59,6 +60,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       mbar_init(s32(&sm.q_full[t]), 1);
       mbar_init(s32(&sm.q_empty[t]), 1);
       mbar_init(s32(&sm.s_full[t]), 1);
+      mbar_init(s32(&sm.sdp_free[t]), 128);
       mbar_init(s32(&sm.p_full[t]), 128);
       mbar_init(s32(&sm.pv_done[t]), 1);
     }
@@ -140,10 +142,26 @@ __global__ void __launch_bounds__(kThreads, 1)
     constexpr uint32_t idesc_nt = make_idesc(false), idesc_nn = make_idesc(true);
     const uint64_t qdesc = smem_desc(s32(sm.q[t])), dodesc = smem_desc(s32(sm.d_o[t]));
     const uint32_t tcol_dq = tmem + kColDQ + 64 * t, tcol_s = tmem + kColS + 128 * t, tcol_dp = tcol_s + 64;
+    const uint32_t tcol_ds = tmem + kColDS + 32 * t;
     const uint32_t tbits = 3u << (2 * t);
     long long step = 0;   // ring position (all chunks, attended by this tile or not)
-    uint32_t nt = 0;      // products issued by this tile so far (phase of s_full / p_full / pv_done)
+    uint32_t nt = 0;      // products started by this tile so far (phase of the per-product barriers)
     bool ok = true;
+    // dQ += dS K of the product whose K chunk sits in ring stage `pst` (the previous product of this tile)
+    auto issue_dq = [&](int pst, bool pfirst) {
+      ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.p_full[t]), (nt - 1) & 1, abort, status));
+      if (!ok) return;
+      tc_fence_after();
+      const uint64_t kmn = smem_desc(s32(sm.kv[pst][0]));
+      if (elect_one()) {
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+          umma_ts(tcol_dq, tcol_ds + 8 * kk, kmn + (uint64_t)((2048 * kk) >> 4), idesc_nn, (!pfirst || kk > 0));
+        tc_commit(s32(&sm.kv_empty[pst]));
+        tc_commit(s32(&sm.pv_done[t]));
+      }
+      __syncwarp();
+    };
     for (int it = 0; ok; ++it) {
       const int buf = it % kLists;
       ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.list_full[buf]), (it / kLists) & 1, abort, status));
@@ -157,7 +175,8 @@ __global__ void __launch_bounds__(kThreads, 1)
       ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.q_full[t]), it & 1, abort, status));
       if (!ok) break;
       if (last < 0 && elect_one()) mbar_arrive(s32(&sm.q_empty[t]));
-      bool first = true;
+      bool first = true, pend = false, pend_first = false;
+      int pend_st = 0;
       for (int e = 0; e < n && ok; ++e) {
         const bool act = (sm.mask[buf][e] & tbits) != 0;
         for (int c = 0; c < g.cpb && ok; ++c, ++step) {
@@ -169,8 +188,11 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (elect_one()) mbar_arrive(s32(&sm.kv_empty[st]));
             continue;
           }
-          // S and dP were last read by this warp's previous dQ += dS K (dS aliases dP) and, before that, by
-          // the row threads, which arrived on p_full: in-order execution makes overwriting them safe
+          // S and dP may be overwritten once the row threads hold the previous product's values in registers
+          if (nt > 0) {
+            ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.sdp_free[t]), (nt - 1) & 1, abort, status));
+            if (!ok) break;
+          }
           tc_fence_after();
           const uint64_t kdesc = smem_desc(s32(sm.kv[st][0])), vdesc = smem_desc(s32(sm.kv[st][1]));
           const bool release_q = e == last && c == g.cpb - 1;
@@ -183,21 +205,14 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (release_q) tc_commit(s32(&sm.q_empty[t]));
           }
           __syncwarp();
-          ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.p_full[t]), nt & 1, abort, status));
+          if (pend) issue_dq(pend_st, pend_first);  // previous product: its dS is ready or about to be
           if (!ok) break;
-          tc_fence_after();
-          if (elect_one()) {
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-              umma_ts(tcol_dq, tcol_dp + 8 * kk, kdesc + (uint64_t)((2048 * kk) >> 4), idesc_nn, (!first || kk > 0));
-            tc_commit(s32(&sm.kv_empty[st]));
-            tc_commit(s32(&sm.pv_done[t]));
-          }
-          __syncwarp();
+          pend = true; pend_st = st; pend_first = first;
           first = false;
           ++nt;
         }
       }
+      if (ok && pend) issue_dq(pend_st, pend_first);  // the item's last product
       if (ok && elect_one()) mbar_arrive(s32(&sm.list_empty[buf]));
     }
   } else {
@@ -207,6 +222,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     const int h = 2 * t + hh;
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t ts = tmem + lane_off + kColS + 128 * t, tdp = ts + 64, tdq = tmem + lane_off + kColDQ + 64 * t;
+    const uint32_t tds = tmem + lane_off + kColDS + 32 * t;
     const uint32_t tbits = 3u << (2 * t), hbit = 1u << h;
     const uint64_t scale2 = pack2(g.scale_log2, g.scale_log2);
     uint32_t nt = 0;
@@ -235,31 +251,39 @@ __global__ void __launch_bounds__(kThreads, 1)
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
+          uint32_t pk[32];
           if (attends) {
-            // two pieces of 32 key columns; piece p writes dS (bf16 pairs) over dP columns 16p .. 16p+15, which
-            // hold fp32 values of key columns this thread has already consumed
+            // all 64 + 64 values into registers, then S and dP are handed back to the tensor core at once
+            uint32_t sv[64], dp[64];
+            tmem_ld32(ts, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
+            tmem_ld32(ts + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
+            tmem_ld32(tdp, *reinterpret_cast<uint32_t(*)[32]>(&dp[0]));
+            tmem_ld32(tdp + 32, *reinterpret_cast<uint32_t(*)[32]>(&dp[32]));
+            tmem_wait_ld();
+            tc_fence_before();
+            mbar_arrive(s32(&sm.sdp_free[t]));
 #pragma unroll
-            for (int piece = 0; piece < 2; ++piece) {
-              uint32_t sv[32], dp[32], pk[16];
-              tmem_ld32(ts + 32 * piece, sv);
-              tmem_ld32(tdp + 32 * piece, dp);
-              tmem_wait_ld();
-#pragma unroll
-              for (int i = 0; i < 32; i += 2) {
-                float x0, x1, d0, d1;
-                unpack2(fma2(pack2(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])), scale2, neg_lse2), x0, x1);
-                const uint64_t dmd = add2(pack2(__uint_as_float(dp[i]), __uint_as_float(dp[i + 1])), neg_d2);
-                unpack2(mul2(pack2(ex2(x0), ex2(x1)), dmd), d0, d1);
-                pk[i >> 1] = bf16x2(d0, d1);
-              }
-              tmem_st16(tdp + 16 * piece, pk);
+            for (int i = 0; i < 64; i += 2) {
+              float x0, x1, d0, d1;
+              unpack2(fma2(pack2(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])), scale2, neg_lse2), x0, x1);
+              const uint64_t dmd = add2(pack2(__uint_as_float(dp[i]), __uint_as_float(dp[i + 1])), neg_d2);
+              unpack2(mul2(pack2(ex2(x0), ex2(x1)), dmd), d0, d1);
+              pk[i >> 1] = bf16x2(d0, d1);
             }
           } else {
-            uint32_t z[32];
+            tc_fence_before();
+            mbar_arrive(s32(&sm.sdp_free[t]));
 #pragma unroll
-            for (int i = 0; i < 32; ++i) z[i] = 0u;
-            tmem_st32(tdp, z);
+            for (int i = 0; i < 32; ++i) pk[i] = 0u;
           }
+          // dS has one buffer: the previous product's dQ += dS K must have consumed it
+          if (done > 0) {
+            ok = mbar_wait(s32(&sm.pv_done[t]), (nt - 1) & 1, abort, status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+          }
+          tmem_st32(tds, pk);
           tmem_wait_st();
           tc_fence_before();
           mbar_arrive(s32(&sm.p_full[t]));

@@ -7,15 +7,17 @@
 // The connected query blocks of key block j are its local neighbours (the neighbourhood relation is
 // symmetric, so they follow from geometry) and the query blocks that selected j (transposed pattern, CSR).
 //
-// Key/value-stationary mirror of the forward kernel: a persistent CTA per SM draws 256-row items of KEY
-// rows (two 128-row tiles, four 64-row halves, each half one 64-token chunk of a key block); the K and V
-// tiles stay in shared memory, query-side chunks (Q, dO, and per query row -LSE*log2(e) and -D) stream
-// through a ring.  Per product and tile:  S^T = K Q^T and dP^T = V dO^T (eight MMAs into two 64-column TMEM
-// buffers), the row threads (thread = key row = TMEM lane) write P^T over the start of the S^T buffer and
-// dS^T over the start of the dP^T buffer (bf16), then dV += P^T dO and dK += dS^T Q with those buffers as
-// TMEM A operands and the staged dO and Q chunks as MN-major B operands.
-// Lists: the planner merges the local neighbourhoods of the item's key blocks (entries carry a mask of
-// the halves they are connected to) and appends each block's CSR list; a list longer than a list buffer
+// Key/value-stationary: a persistent CTA per SM draws items of 128 KEY rows (one tile = two 64-row halves,
+// each half one 64-token chunk of a key block; tile t of the 256-row items the other kernels use).  The K
+// and V tiles stay in shared memory; query-side chunks (Q, dO, and per query row -LSE*log2(e) and -D)
+// stream through a ring.  Per product:  S^T = K Q^T and dP^T = V dO^T (eight MMAs into two 64-column TMEM
+// buffers); the row threads (TMEM lane = key row, two threads per row, each half of the query columns; the
+// backward has no reduction along a row, so they never talk) pull their share into registers and hand the
+// buffers back at once, so the next product's S^T and dP^T are computed while they form P^T and dS^T (bf16,
+// own TMEM columns); then dV += P^T dO and dK += dS^T Q (TMEM A operands, the staged dO and Q chunks as
+// MN-major B operands), issued one product behind.
+// Lists: the planner merges the local neighbourhoods of the tile's key blocks (entries carry a mask of the
+// halves they are connected to) and appends each block's CSR list; a list longer than a list buffer
 // continues in the next buffer (ItemInfo::more).  The order of a list is a function of the pattern alone,
 // so the summation order, and with it the result, is deterministic.
 // Every mbarrier wait is bounded; on expiry the CTA records MOSAIC_E_DEVICE_TIMEOUT and drains.
@@ -26,10 +28,10 @@ namespace mosaic {
 namespace {
 
 constexpr int kStages = 6;       // ring depth of query-side chunks
-constexpr int kThreads = 384;
+constexpr int kThreads = 384;    // warps 0-7 row threads, 8 TMA producer, 9 MMA issuer, 10 idle, 11 planner
 constexpr uint32_t kTmemCols = 512;
-// tile t: dK at 256 t, dV at 256 t + 64, S^T (then P^T) at 256 t + 128, dP^T (then dS^T) at 256 t + 192
-constexpr uint32_t kColDK = 0, kColDV = 64, kColS = 128, kColDP = 192, kTileCols = 256;
+// dK, dV accumulators; S^T and dP^T (fp32); P^T and dS^T (bf16 pairs)
+constexpr uint32_t kColDK = 0, kColDV = 64, kColS = 128, kColDP = 192, kColP = 256, kColDS = 288;
 constexpr uint32_t kStageBytes = 2 * kTile + 2 * 64 * 4;
 
 struct Stage {
@@ -41,23 +43,21 @@ struct Stage {
 };
 
 struct Smem {
-  unsigned char k[2][2 * kTile];           // [tile][128 key rows x 128 B]
-  unsigned char v[2][2 * kTile];
+  unsigned char k[2 * kTile];              // 128 key rows x 128 B
+  unsigned char v[2 * kTile];
   Stage ring[kStages];
   unsigned long long ring_full[kStages], ring_empty[kStages];
-  unsigned long long kv_full[2], kv_empty[2], s_full[2], p_full[2], pv_done[2];  // [tile]
+  unsigned long long kv_full, kv_empty, s_full, sdp_free, p_full, pv_done;
   unsigned long long list_full[kLists], list_empty[kLists];
   uint32_t tmem_base;
   int abort;
-  ItemInfo info[kLists];
+  ItemInfo info[kLists];             // hb/hc/hvalid entries 0 and 1 describe the tile's two halves
   int ids[kLists][kMaxUnion];
   unsigned char mask[kLists][kMaxUnion];
-  int tmp_ids[kMaxUnion];            // planner scratch: merged list before reordering
-  unsigned char tmp_mask[kMaxUnion];
 };
 
-// Planner of the key-stationary kernel: per item, the merged local neighbourhoods of its key blocks, then
-// each block's list of selecting query blocks, cut into list buffers.
+// Planner of the key-stationary kernel: per item (tile), the merged local neighbourhoods of its key blocks,
+// then each block's list of selecting query blocks, cut into list buffers.
 __device__ __forceinline__ void planner_kv_loop(Smem& sm, const Geo& g, const int32_t* __restrict__ csr_off,
                                                 const int32_t* __restrict__ csr_q, int* work_counter, int ipu,
                                                 int total_items, int lane, volatile int* abort, int* status) {
@@ -77,50 +77,41 @@ __device__ __forceinline__ void planner_kv_loop(Smem& sm, const Geo& g, const in
       if (lane == 0) { sm.info[lb % kLists].n = -1; mbar_arrive(s32(&sm.list_full[lb % kLists])); }
       break;
     }
-    const int u = item / ipu;
-    int hb[4], hc[4];
-    const int valid = item_halves(g, item - u * ipu, hb, hc);
+    // item = 2 * (256-row item) + tile
+    const int i256 = item >> 1, t = item & 1;
+    const int u = i256 / ipu;
+    int hb4[4], hc4[4];
+    const int valid4 = item_halves(g, i256 - u * ipu, hb4, hc4);
+    const int hb[2] = {hb4[2 * t], hb4[2 * t + 1]}, hc[2] = {hc4[2 * t], hc4[2 * t + 1]};
+    const int valid = (valid4 >> (2 * t)) & 3;
     int n = 0;
-    auto publish = [&](int more) {  // reorder the scratch list into buffer lb and hand it over
+    auto publish = [&](int more) {
       const int buf = lb % kLists;
-      interleave_tiles(sm.tmp_ids, sm.tmp_mask, n, sm.ids[buf], sm.mask[buf], lane);
       if (lane == 0) {
         ItemInfo& inf = sm.info[buf];
         inf.n = n; inf.unit = u; inf.hvalid = valid; inf.more = more;
-#pragma unroll
-        for (int h = 0; h < 4; ++h) { inf.hb[h] = hb[h]; inf.hc[h] = hc[h]; }
+        inf.hb[0] = hb[0]; inf.hb[1] = hb[1]; inf.hc[0] = hc[0]; inf.hc[1] = hc[1];
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(s32(&sm.list_full[buf]));
       ++lb;
       n = 0;
     };
-    // the halves of one key block are merged once, with all their bits
-    unsigned char bits_of[4];
-    bool first_of[4];
-#pragma unroll
-    for (int h = 0; h < 4; ++h) {
-      first_of[h] = ((valid >> h) & 1) != 0;
-      bits_of[h] = 0;
-#pragma unroll
-      for (int h2 = 0; h2 < 4; ++h2) {
-        if (((valid >> h2) & 1) && ((valid >> h) & 1) && hb[h2] == hb[h]) {
-          if (h2 < h) first_of[h] = false;
-          bits_of[h] |= (unsigned char)(1 << h2);
-        }
-      }
-    }
-    // local neighbourhoods (at most 64 entries per block, merged with masks)
-#pragma unroll
-    for (int h = 0; h < 4; ++h)
-      if (first_of[h]) n = merge_block(g, -1, hb[h], bits_of[h], sm.tmp_ids, sm.tmp_mask, n, lane, status);
+    // the two halves are either two key blocks (one bit each) or two chunks of one block (both bits)
+    const bool same = (valid == 3) && hb[0] == hb[1];
+    const unsigned char bits0 = same ? 3 : 1, bits1 = 2;
+    const bool use0 = (valid & 1) != 0, use1 = (valid & 2) != 0 && !same;
+    // local neighbourhoods (at most 64 entries per block, merged with masks), straight into the list buffer
+    if (use0) n = merge_block(g, -1, hb[0], bits0, sm.ids[lb % kLists], sm.mask[lb % kLists], n, lane, status);
+    if (use1) n = merge_block(g, -1, hb[1], bits1, sm.ids[lb % kLists], sm.mask[lb % kLists], n, lane, status);
     // query blocks that selected the key block (ascending ids), appended 32 at a time
     const int32_t* off = csr_off + (long long)u * (g.m + 1);
     const int32_t* sel = csr_q + (long long)u * g.m * g.topk;
 #pragma unroll
-    for (int h = 0; h < 4 && ok; ++h) {
-      if (!first_of[h]) continue;
-      const int s_beg = __ldg(off + hb[h]), s_end = __ldg(off + hb[h] + 1);
+    for (int hh = 0; hh < 2 && ok; ++hh) {
+      if (!(hh == 0 ? use0 : use1)) continue;
+      const unsigned char bits = hh == 0 ? bits0 : bits1;
+      const int s_beg = __ldg(off + hb[hh]), s_end = __ldg(off + hb[hh] + 1);
       for (int base = s_beg; base < s_end && ok; base += 32) {
         if (n + 32 > kMaxUnion) {
           publish(1);
@@ -129,8 +120,8 @@ __device__ __forceinline__ void planner_kv_loop(Smem& sm, const Geo& g, const in
         }
         const int e = base + lane;
         if (e < s_end) {
-          sm.tmp_ids[n + lane] = __ldg(sel + e);
-          sm.tmp_mask[n + lane] = bits_of[h];
+          sm.ids[lb % kLists][n + lane] = __ldg(sel + e);
+          sm.mask[lb % kLists][n + lane] = bits;
         }
         n += min(32, s_end - base);
         __syncwarp();
@@ -155,17 +146,16 @@ __global__ void __launch_bounds__(kThreads, 1)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(s32(&sm.ring_full[s]), 1); mbar_init(s32(&sm.ring_empty[s]), 2); }
-    for (int t = 0; t < 2; ++t) {
-      mbar_init(s32(&sm.kv_full[t]), 1);
-      mbar_init(s32(&sm.kv_empty[t]), 1);
-      mbar_init(s32(&sm.s_full[t]), 1);
-      mbar_init(s32(&sm.p_full[t]), 128);
-      mbar_init(s32(&sm.pv_done[t]), 1);
-    }
+    for (int s = 0; s < kStages; ++s) { mbar_init(s32(&sm.ring_full[s]), 1); mbar_init(s32(&sm.ring_empty[s]), 1); }
+    mbar_init(s32(&sm.kv_full), 1);
+    mbar_init(s32(&sm.kv_empty), 1);
+    mbar_init(s32(&sm.s_full), 1);
+    mbar_init(s32(&sm.sdp_free), 256);
+    mbar_init(s32(&sm.p_full), 256);
+    mbar_init(s32(&sm.pv_done), 1);
     for (int i = 0; i < kLists; ++i) {
       mbar_init(s32(&sm.list_full[i]), 1);
-      mbar_init(s32(&sm.list_empty[i]), 11);  // 8 row-thread warps + 2 MMA warps + TMA producer
+      mbar_init(s32(&sm.list_empty[i]), 10);  // 8 row-thread warps + MMA warp + TMA producer
     }
     sm.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -202,17 +192,15 @@ __global__ void __launch_bounds__(kThreads, 1)
         if (n < 0) break;
         if (fresh) {
           // K and V tiles: free once every product of the previous item has completed
-          for (int t = 0; t < 2 && ok; ++t) {
-            ok = mbar_wait(s32(&sm.kv_empty[t]), (items & 1) ^ 1, abort, status);
-            if (!ok) break;
-            mbar_expect_tx(s32(&sm.kv_full[t]), 4 * kTile);
-            for (int hh = 0; hh < 2; ++hh) {
-              const int h = 2 * t + hh, by = inf.hb[h] / g.nbw, bx = inf.hb[h] - by * g.nbw;
-              tma_load_4d(s32(sm.k[t] + hh * kTile), &map_k, s32(&sm.kv_full[t]), 0, bx * g.bw,
-                          by * g.bh + inf.hc[h] * g.crows, u);
-              tma_load_4d(s32(sm.v[t] + hh * kTile), &map_v, s32(&sm.kv_full[t]), 0, bx * g.bw,
-                          by * g.bh + inf.hc[h] * g.crows, u);
-            }
+          ok = mbar_wait(s32(&sm.kv_empty), (items & 1) ^ 1, abort, status);
+          if (!ok) break;
+          mbar_expect_tx(s32(&sm.kv_full), 4 * kTile);
+          for (int hh = 0; hh < 2; ++hh) {
+            const int by = inf.hb[hh] / g.nbw, bx = inf.hb[hh] - by * g.nbw;
+            tma_load_4d(s32(sm.k + hh * kTile), &map_k, s32(&sm.kv_full), 0, bx * g.bw,
+                        by * g.bh + inf.hc[hh] * g.crows, u);
+            tma_load_4d(s32(sm.v + hh * kTile), &map_v, s32(&sm.kv_full), 0, bx * g.bw,
+                        by * g.bh + inf.hc[hh] * g.crows, u);
           }
           ++items;
         }
@@ -238,24 +226,43 @@ __global__ void __launch_bounds__(kThreads, 1)
       if (*abort) {  // give copies in flight time to land before the CTA's memory is released
         const long long t0 = clock64();
         while (clock64() - t0 < 400000) {}
-      } else {       // drain: the last uses of every ring stage have been released by both tiles
+      } else {       // drain: the last uses of every ring stage have been released
         const long long first = step > kStages ? step - kStages : 0;
         for (long long s = first; s < step; ++s)
           if (!mbar_wait(s32(&sm.ring_empty[s % kStages]), (uint32_t)((s / kStages) & 1), abort, status)) break;
       }
     }
-  } else if (warp == 9 || warp == 10) {
-    // ------------------------------------------------------------- MMA issuer of tile t
+  } else if (warp == 9) {
+    // ------------------------------------------------------------- MMA issuer
     // The whole warp walks the loop; one elected lane issues the tensor-core instructions.
-    const int t = warp - 9;
     constexpr uint32_t idesc_nt = make_idesc(false), idesc_nn = make_idesc(true);
-    const uint64_t kdesc = smem_desc(s32(sm.k[t])), vdesc = smem_desc(s32(sm.v[t]));
-    const uint32_t tbase = tmem + kTileCols * t;
-    const uint32_t tbits = 3u << (2 * t);
-    long long step = 0;   // ring position (all chunks, connected to this tile or not)
-    uint32_t nt = 0;      // products issued by this tile so far (phase of s_full / p_full / pv_done)
+    const uint64_t kdesc = smem_desc(s32(sm.k)), vdesc = smem_desc(s32(sm.v));
+    long long step = 0;   // ring position
+    uint32_t nt = 0;      // products started so far (phase of the per-product barriers)
     int items = 0;
     bool ok = true, fresh = true, first = true;
+    bool pend = false, pend_first = false;
+    int pend_st = 0;
+    // dV += P^T dO and dK += dS^T Q of the previous product (its chunks sit in ring stage `pst`)
+    auto issue_grads = [&](int pst, bool pfirst) {
+      ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.p_full), (nt - 1) & 1, abort, status));
+      if (!ok) return;
+      tc_fence_after();
+      const uint64_t qmn = smem_desc(s32(sm.ring[pst].q)), domn = smem_desc(s32(sm.ring[pst].d_o));
+      if (elect_one()) {
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+          umma_ts(tmem + kColDV, tmem + kColP + 8 * kk, domn + (uint64_t)((2048 * kk) >> 4), idesc_nn,
+                  (!pfirst || kk > 0));
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+          umma_ts(tmem + kColDK, tmem + kColDS + 8 * kk, qmn + (uint64_t)((2048 * kk) >> 4), idesc_nn,
+                  (!pfirst || kk > 0));
+        tc_commit(s32(&sm.ring_empty[pst]));
+        tc_commit(s32(&sm.pv_done));
+      }
+      __syncwarp();
+    };
     for (int lb = 0; ok; ++lb) {
       const int buf = lb % kLists;
       ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.list_full[buf]), (lb / kLists) & 1, abort, status));
@@ -264,67 +271,55 @@ __global__ void __launch_bounds__(kThreads, 1)
       if (n < 0) break;
       const bool more = sm.info[buf].more != 0;
       if (fresh) {
-        ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.kv_full[t]), items & 1, abort, status));
+        ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.kv_full), items & 1, abort, status));
         if (!ok) break;
         ++items;
         first = true;
       }
       fresh = !more;
       for (int e = 0; e < n && ok; ++e) {
-        const bool act = (sm.mask[buf][e] & tbits) != 0;
         for (int c = 0; c < g.cpb && ok; ++c, ++step) {
           const int st = (int)(step % kStages);
           ok = __all_sync(0xffffffffu,
                           mbar_wait(s32(&sm.ring_full[st]), (uint32_t)((step / kStages) & 1), abort, status));
           if (!ok) break;
-          if (!act) {
-            if (elect_one()) mbar_arrive(s32(&sm.ring_empty[st]));
-            continue;
+          // S^T and dP^T may be overwritten once the row threads hold the previous product in registers
+          if (nt > 0) {
+            ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.sdp_free), (nt - 1) & 1, abort, status));
+            if (!ok) break;
           }
-          // S^T and dP^T were last read by this warp's previous dV / dK products (P^T and dS^T alias them)
-          // and before that by the row threads, which arrived on p_full: in-order execution makes
-          // overwriting them safe
           tc_fence_after();
           const uint64_t qdesc = smem_desc(s32(sm.ring[st].q)), dodesc = smem_desc(s32(sm.ring[st].d_o));
           if (elect_one()) {
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) umma_ss(tbase + kColS, kdesc + 2 * kk, qdesc + 2 * kk, idesc_nt, kk > 0);
+            for (int kk = 0; kk < 4; ++kk) umma_ss(tmem + kColS, kdesc + 2 * kk, qdesc + 2 * kk, idesc_nt, kk > 0);
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) umma_ss(tbase + kColDP, vdesc + 2 * kk, dodesc + 2 * kk, idesc_nt, kk > 0);
-            tc_commit(s32(&sm.s_full[t]));
+            for (int kk = 0; kk < 4; ++kk) umma_ss(tmem + kColDP, vdesc + 2 * kk, dodesc + 2 * kk, idesc_nt, kk > 0);
+            tc_commit(s32(&sm.s_full));
           }
           __syncwarp();
-          ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.p_full[t]), nt & 1, abort, status));
+          if (pend) issue_grads(pend_st, pend_first);
           if (!ok) break;
-          tc_fence_after();
-          if (elect_one()) {
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-              umma_ts(tbase + kColDV, tbase + kColS + 8 * kk, dodesc + (uint64_t)((2048 * kk) >> 4), idesc_nn,
-                      (!first || kk > 0));
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-              umma_ts(tbase + kColDK, tbase + kColDP + 8 * kk, qdesc + (uint64_t)((2048 * kk) >> 4), idesc_nn,
-                      (!first || kk > 0));
-            tc_commit(s32(&sm.ring_empty[st]));
-            tc_commit(s32(&sm.pv_done[t]));
-          }
-          __syncwarp();
+          pend = true; pend_st = st; pend_first = first;
           first = false;
           ++nt;
         }
       }
-      if (ok && !more && elect_one()) tc_commit(s32(&sm.kv_empty[t]));  // all products of the item are behind it
+      if (ok && !more) {
+        if (pend) issue_grads(pend_st, pend_first);  // the item's last product
+        pend = false;
+        if (ok && elect_one()) tc_commit(s32(&sm.kv_empty));  // all products of the item are behind it
+      }
       if (ok && elect_one()) mbar_arrive(s32(&sm.list_empty[buf]));
     }
-  } else {
-    // ------------------------------------------------------------- row threads of tile t (thread = key row)
-    const int t = warp >> 2;        // tile
-    const int hh = (warp >> 1) & 1; // 64-row half of the tile this warp's rows belong to
-    const int h = 2 * t + hh;
-    const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t tbase = tmem + lane_off + kTileCols * t;
-    const uint32_t tbits = 3u << (2 * t), hbit = 1u << h;
+  } else if (warp < 8) {
+    // ------------------------------------------------------------- row threads (TMEM lane = key row)
+    const int ch = warp >> 2;        // half of the query columns (and of the output channels) this thread owns
+    const int quad = warp & 3;       // TMEM lane quadrant
+    const int hh = quad >> 1;        // 64-row half of the tile this warp's rows belong to
+    const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
+    const uint32_t tb = tmem + lane_off;
+    const uint32_t hbit = 1u << hh;
     const uint64_t scale2 = pack2(g.scale_log2, g.scale_log2);
     uint32_t nt = 0;
     long long step = 0;  // ring position, to find the stage that holds the query rows' -LSE and -D
@@ -339,14 +334,13 @@ __global__ void __launch_bounds__(kThreads, 1)
       if (n < 0) break;
       const bool more = sm.info[buf].more != 0;
       for (int e = 0; e < n && ok; ++e) {
-        const uint32_t mk = sm.mask[buf][e];
-        if (!(mk & tbits)) { step += g.cpb; continue; }
-        const bool connected = (mk & hbit) != 0;
+        const bool connected = (sm.mask[buf][e] & hbit) != 0;
         for (int c = 0; c < g.cpb; ++c, ++step) {
-          ok = mbar_wait(s32(&sm.s_full[t]), nt & 1, abort, status);  // implies the ring stage has landed
+          ok = mbar_wait(s32(&sm.s_full), nt & 1, abort, status);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
+          uint32_t pp[16], ds[16];
           if (connected) {
             const int st = (int)(step % kStages);
             // the stage landed before the MMA warp could produce this S^T; waiting on its barrier here as well
@@ -355,45 +349,48 @@ __global__ void __launch_bounds__(kThreads, 1)
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             const Stage& sg = sm.ring[st];
-            // two pieces of 32 query columns; piece p writes P^T and dS^T (bf16 pairs) over columns
-            // 16p .. 16p+15 of the S^T and dP^T buffers, which hold values this thread has already consumed
+            uint32_t sv[32], dp[32];
+            tmem_ld32(tb + kColS + 32 * ch, sv);
+            tmem_ld32(tb + kColDP + 32 * ch, dp);
+            tmem_wait_ld();
+            tc_fence_before();
+            mbar_arrive(s32(&sm.sdp_free));  // S^T and dP^T go back to the tensor core
 #pragma unroll
-            for (int piece = 0; piece < 2; ++piece) {
-              uint32_t sv[32], dp[32], pp[16], ds[16];
-              tmem_ld32(tbase + kColS + 32 * piece, sv);
-              tmem_ld32(tbase + kColDP + 32 * piece, dp);
-              tmem_wait_ld();
-#pragma unroll
-              for (int i = 0; i < 32; i += 4) {
-                // -LSE*log2(e) and -D of four query columns (the same for every thread: broadcast loads)
-                const float4 nl = *reinterpret_cast<const float4*>(&sg.neg_lse2[32 * piece + i]);
-                const float4 nd = *reinterpret_cast<const float4*>(&sg.neg_d[32 * piece + i]);
-                float x0, x1, x2, x3, d0, d1, d2, d3;
-                unpack2(fma2(pack2(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])), scale2, pack2(nl.x, nl.y)), x0, x1);
-                unpack2(fma2(pack2(__uint_as_float(sv[i + 2]), __uint_as_float(sv[i + 3])), scale2, pack2(nl.z, nl.w)), x2, x3);
-                const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
-                const uint64_t t01 = add2(pack2(__uint_as_float(dp[i]), __uint_as_float(dp[i + 1])), pack2(nd.x, nd.y));
-                const uint64_t t23 = add2(pack2(__uint_as_float(dp[i + 2]), __uint_as_float(dp[i + 3])), pack2(nd.z, nd.w));
-                unpack2(mul2(pack2(p0, p1), t01), d0, d1);
-                unpack2(mul2(pack2(p2, p3), t23), d2, d3);
-                pp[i >> 1] = bf16x2(p0, p1);
-                pp[(i >> 1) + 1] = bf16x2(p2, p3);
-                ds[i >> 1] = bf16x2(d0, d1);
-                ds[(i >> 1) + 1] = bf16x2(d2, d3);
-              }
-              tmem_st16(tbase + kColS + 16 * piece, pp);
-              tmem_st16(tbase + kColDP + 16 * piece, ds);
+            for (int i = 0; i < 32; i += 4) {
+              // -LSE*log2(e) and -D of four query columns (the same for every thread: broadcast loads)
+              const float4 nl = *reinterpret_cast<const float4*>(&sg.neg_lse2[32 * ch + i]);
+              const float4 nd = *reinterpret_cast<const float4*>(&sg.neg_d[32 * ch + i]);
+              float x0, x1, x2, x3, d0, d1, d2, d3;
+              unpack2(fma2(pack2(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])), scale2, pack2(nl.x, nl.y)), x0, x1);
+              unpack2(fma2(pack2(__uint_as_float(sv[i + 2]), __uint_as_float(sv[i + 3])), scale2, pack2(nl.z, nl.w)), x2, x3);
+              const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
+              const uint64_t t01 = add2(pack2(__uint_as_float(dp[i]), __uint_as_float(dp[i + 1])), pack2(nd.x, nd.y));
+              const uint64_t t23 = add2(pack2(__uint_as_float(dp[i + 2]), __uint_as_float(dp[i + 3])), pack2(nd.z, nd.w));
+              unpack2(mul2(pack2(p0, p1), t01), d0, d1);
+              unpack2(mul2(pack2(p2, p3), t23), d2, d3);
+              pp[i >> 1] = bf16x2(p0, p1);
+              pp[(i >> 1) + 1] = bf16x2(p2, p3);
+              ds[i >> 1] = bf16x2(d0, d1);
+              ds[(i >> 1) + 1] = bf16x2(d2, d3);
             }
           } else {
-            uint32_t z[32];
+            tc_fence_before();
+            mbar_arrive(s32(&sm.sdp_free));
 #pragma unroll
-            for (int i = 0; i < 32; ++i) z[i] = 0u;
-            tmem_st32(tbase + kColS, z);
-            tmem_st32(tbase + kColDP, z);
+            for (int i = 0; i < 16; ++i) { pp[i] = 0u; ds[i] = 0u; }
           }
+          // P^T and dS^T have one buffer each: the previous product's dV / dK updates must have consumed them
+          if (item_done > 0) {
+            ok = mbar_wait(s32(&sm.pv_done), (nt - 1) & 1, abort, status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+          }
+          tmem_st16(tb + kColP + 16 * ch, pp);
+          tmem_st16(tb + kColDS + 16 * ch, ds);
           tmem_wait_st();
           tc_fence_before();
-          mbar_arrive(s32(&sm.p_full[t]));
+          mbar_arrive(s32(&sm.p_full));
           ++nt;
           ++item_done;
         }
@@ -401,30 +398,26 @@ __global__ void __launch_bounds__(kThreads, 1)
       if (!ok) break;
       if (!more) {
         if (item_done > 0) {
-          ok = mbar_wait(s32(&sm.pv_done[t]), (nt - 1) & 1, abort, status);
+          ok = mbar_wait(s32(&sm.pv_done), (nt - 1) & 1, abort, status);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
-          if ((sm.info[buf].hvalid >> h) & 1) {
+          if ((sm.info[buf].hvalid >> hh) & 1) {
             const long long tok = (long long)sm.info[buf].unit * g.N +
-                                  chunk_token(g, sm.info[buf].hb[h], sm.info[buf].hc[h], tid & 63);
+                                  chunk_token(g, sm.info[buf].hb[hh], sm.info[buf].hc[hh], (quad & 1) * 32 + lane);
 #pragma unroll
             for (int which = 0; which < 2; ++which) {  // 0: dK (scaled), 1: dV
-              uint4* dst = reinterpret_cast<uint4*>((which ? dv : dk) + tok * kD);
+              uint4* dst = reinterpret_cast<uint4*>((which ? dv : dk) + tok * kD + 32 * ch);
               const float f = which ? 1.f : g.scale;
+              uint32_t ov[32];
+              tmem_ld32(tb + (which ? kColDV : kColDK) + 32 * ch, ov);
+              tmem_wait_ld();
+              uint32_t w[16];
 #pragma unroll
-              for (int part = 0; part < 2; ++part) {
-                uint32_t ov[32];
-                tmem_ld32(tbase + (which ? kColDV : kColDK) + 32 * part, ov);
-                tmem_wait_ld();
-                uint32_t w[16];
+              for (int i = 0; i < 16; ++i)
+                w[i] = bf16x2(__uint_as_float(ov[2 * i]) * f, __uint_as_float(ov[2 * i + 1]) * f);
 #pragma unroll
-                for (int i = 0; i < 16; ++i)
-                  w[i] = bf16x2(__uint_as_float(ov[2 * i]) * f, __uint_as_float(ov[2 * i + 1]) * f);
-#pragma unroll
-                for (int i = 0; i < 4; ++i)
-                  dst[part * 4 + i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
-              }
+              for (int i = 0; i < 4; ++i) dst[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
             }
           }
         }
@@ -461,7 +454,7 @@ int launch_dkdv_tc(const HostCtx& c, const void* q, const void* k, const void* v
   if (cudaFuncSetAttribute(dkdv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return MOSAIC_E_CUDA;
   const int ipu = items_per_unit(g);
-  const long long total = (long long)g.U * ipu;
+  const long long total = 2ll * g.U * ipu;  // one item per 128-row tile
   if (total > 0x7fffff00ll) return MOSAIC_E_UNSUPPORTED;
   const long long grid = total < (long long)sms ? total : (long long)sms;
   dkdv_tc_kernel<<<(unsigned)grid, kThreads, smem, c.stream>>>(g, mq, mdo, mk, mv, mnl, mnd, csr_off, csr_q,

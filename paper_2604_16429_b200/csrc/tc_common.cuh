@@ -436,6 +436,35 @@ __device__ __forceinline__ void planner_loop(SM& sm, const Geo& g, const int32_t
       }
       if (first) n = merge_block(g, jsel[h], hb[h], bits, sm.tmp_ids, sm.tmp_mask, n, lane, status);
     }
+    if (g.cpb == 1 && valid == 0xF) {
+      // Four different query blocks: which two share a 128-row tile is free.  Take the pairing whose tiles have
+      // the most entries in common (fewest products with a masked half); ties keep the first pairing.
+      int o01 = 0, o23 = 0, o02 = 0, o13 = 0, o03 = 0, o12 = 0;
+      for (int e0 = 0; e0 < n; e0 += 32) {
+        const unsigned mk = e0 + lane < n ? sm.tmp_mask[e0 + lane] : 0u;
+        o01 += __popc(__ballot_sync(0xffffffffu, (mk & 3u) == 3u));
+        o23 += __popc(__ballot_sync(0xffffffffu, (mk & 12u) == 12u));
+        o02 += __popc(__ballot_sync(0xffffffffu, (mk & 5u) == 5u));
+        o13 += __popc(__ballot_sync(0xffffffffu, (mk & 10u) == 10u));
+        o03 += __popc(__ballot_sync(0xffffffffu, (mk & 9u) == 9u));
+        o12 += __popc(__ballot_sync(0xffffffffu, (mk & 6u) == 6u));
+      }
+      const int s0 = o01 + o23, s1 = o02 + o13, s2 = o03 + o12;
+      const int pick = (s1 > s0 && s1 >= s2) ? 1 : (s2 > s0 && s2 > s1) ? 2 : 0;
+      if (pick != 0) {
+        // new half k is old half perm[k]: (0,2,1,3) pairs the blocks vertically, (0,3,1,2) diagonally
+        const int p1 = pick == 1 ? 2 : 3, p2 = 1, p3 = pick == 1 ? 3 : 2;
+        for (int e = lane; e < n; e += 32) {
+          const unsigned mk = sm.tmp_mask[e];
+          sm.tmp_mask[e] = (unsigned char)((mk & 1u) | (((mk >> p1) & 1u) << 1) | (((mk >> p2) & 1u) << 2) |
+                                           (((mk >> p3) & 1u) << 3));
+        }
+        const int b1 = hb[p1], b2 = hb[p2], b3 = hb[p3], c1 = hc[p1], c2 = hc[p2], c3 = hc[p3];
+        hb[1] = b1; hb[2] = b2; hb[3] = b3;
+        hc[1] = c1; hc[2] = c2; hc[3] = c3;
+        __syncwarp();
+      }
+    }
     interleave_tiles(sm.tmp_ids, sm.tmp_mask, n, sm.ids[buf], sm.mask[buf], lane);
     if (lane == 0) {
       ItemInfo& inf = sm.info[buf];

@@ -342,56 +342,63 @@ __device__ __forceinline__ bool elect_one() {
   return pred != 0;
 }
 
-// Reorder a merged key list so that both tiles find work all along it: entries only tile 0 attends
-// (class 0), entries both attend (1) and entries only tile 1 attends (2) are spread evenly, the k-th
-// entry of a class of n getting the fractional position (4k + class) / (4n).  The order of a softmax
-// sum does not matter to the result beyond rounding; the order is a function of the list alone.
+// Reorder a merged key list so that both tiles, and both 64-row halves of a tile, find work all along it.
+// Entries fall into seven classes by who attends them: tile 0 only (upper half, lower half, both halves), both
+// tiles, tile 1 only (upper, lower, both).  The k-th entry of a class of n gets the fractional position
+// (8k + class) / (8n), so every class is spread evenly; in particular products that only the upper half of a
+// tile attends alternate with products only its lower half attends, and since S is double-buffered the idle
+// half's warps run ahead into the next product.  The order of a softmax sum does not matter to the result
+// beyond rounding; the order is a function of the list alone.
+__device__ __forceinline__ int list_class(unsigned m) {
+  const unsigned t0 = m & 3u, t1 = (m >> 2) & 3u;
+  return t1 == 0u ? (int)t0 - 1 : t0 == 0u ? 3 + (int)t1 : 3;
+}
 __device__ __forceinline__ void interleave_tiles(const int* sid, const unsigned char* smask, int n, int* did,
                                                  unsigned char* dmask, int lane) {
-  int c0 = 0, c1 = 0, c2 = 0;
+  constexpr int NC = 7;
+  int cnt[NC];
+#pragma unroll
+  for (int y = 0; y < NC; ++y) cnt[y] = 0;
   for (int e0 = 0; e0 < n; e0 += 32) {
     const int e = e0 + lane;
-    const unsigned m = e < n ? smask[e] : 0u;
-    const int cls = e < n ? ((m & 3u) ? ((m & 12u) ? 1 : 0) : 2) : 3;
-    c0 += __popc(__ballot_sync(0xffffffffu, cls == 0));
-    c1 += __popc(__ballot_sync(0xffffffffu, cls == 1));
-    c2 += __popc(__ballot_sync(0xffffffffu, cls == 2));
+    const int cls = e < n ? list_class(smask[e]) : -1;
+#pragma unroll
+    for (int y = 0; y < NC; ++y) cnt[y] += __popc(__ballot_sync(0xffffffffu, cls == y));
   }
-  int b0 = 0, b1 = 0, b2 = 0;
+  int base[NC];
+#pragma unroll
+  for (int y = 0; y < NC; ++y) base[y] = 0;
   for (int e0 = 0; e0 < n; e0 += 32) {
     const int e = e0 + lane;
     const unsigned m = e < n ? smask[e] : 0u;
-    const int cls = e < n ? ((m & 3u) ? ((m & 12u) ? 1 : 0) : 2) : 3;
-    const unsigned m0 = __ballot_sync(0xffffffffu, cls == 0), m1 = __ballot_sync(0xffffffffu, cls == 1),
-                   m2 = __ballot_sync(0xffffffffu, cls == 2);
+    const int cls = e < n ? list_class(m) : -1;
+    const unsigned lower = (1u << lane) - 1u;
+    int k = 0, nx = 1;
+#pragma unroll
+    for (int y = 0; y < NC; ++y) {
+      const unsigned by = __ballot_sync(0xffffffffu, cls == y);
+      if (cls == y) { k = base[y] + __popc(by & lower); nx = cnt[y]; }
+      base[y] += __popc(by);
+    }
     if (e < n) {
-      const unsigned lower = (1u << lane) - 1u;
-      const int k = cls == 0 ? b0 + __popc(m0 & lower) : cls == 1 ? b1 + __popc(m1 & lower) : b2 + __popc(m2 & lower);
-      const int nx = cls == 0 ? c0 : cls == 1 ? c1 : c2;
       int pos = k;
 #pragma unroll
-      for (int y = 0; y < 3; ++y) {
-        if (y == cls) continue;
-        const int ny = y == 0 ? c0 : y == 1 ? c1 : c2;
-        if (ny == 0) continue;
-        // entries j of class y that come first: (4j + y) nx < (4k + cls) ny, ties to the lower class
-        const int R = (4 * k + cls) * ny - y * nx;  // 4 j nx < R, or <= R when y < cls
-        int cnt = 0;
-        if (y < cls) cnt = R >= 0 ? R / (4 * nx) + 1 : 0;
-        else cnt = R > 0 ? (R + 4 * nx - 1) / (4 * nx) : 0;
-        pos += min(cnt, ny);
+      for (int y = 0; y < NC; ++y) {
+        const int ny = cnt[y];
+        if (y == cls || ny == 0) continue;
+        // entries j of class y that come first: (8j + y) nx < (8k + cls) ny, ties to the lower class
+        const int R = (8 * k + cls) * ny - y * nx;
+        int c = 0;
+        if (y < cls) c = R >= 0 ? R / (8 * nx) + 1 : 0;
+        else c = R > 0 ? (R + 8 * nx - 1) / (8 * nx) : 0;
+        pos += min(c, ny);
       }
       did[pos] = sid[e];
       dmask[pos] = (unsigned char)m;
     }
-    b0 += __popc(m0);
-    b1 += __popc(m1);
-    b2 += __popc(m2);
   }
   __syncwarp();
 }
-
-
 
 // Planner warp: draws work items from the queue (the first item of a CTA is its own index) and builds each
 // item's merged, interleaved key list one or more items ahead of the warps that consume it.  `SM` is the

@@ -43,7 +43,7 @@ FALLBACK_HBM_GBS = 6650.0
 L2_FLUSH_BYTES = 256 << 20
 # DRAM bytes moved by one fwd_tc_kernel launch (ncu, dram__bytes_read.sum + dram__bytes_write.sum of the
 # capture summarised in profiles/fwd_tc_kernel_c2_1p5deg.md).  Workloads without a capture report null.
-FWD_TRAFFIC_BYTES = {"c2_1p5deg": 88.77e6 + 12.29e6}
+FWD_TRAFFIC_BYTES = {"c2_1p5deg": 88.69e6 + 12.58e6}
 
 
 def measured_peaks():

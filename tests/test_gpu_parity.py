@@ -184,6 +184,35 @@ def test_backward_popular_key_blocks_lists_span_several_buffers():
         assert (err <= G.BWD_MAX_ABS + 1e-2 * np.abs(want)).all(), f"{name} max-abs {err.max():.4g}"
 
 
+def test_backward_custom_scale_and_wide_neighbourhood():
+    w = synth.small_case(48, 64, 8, 8, 6, B=1, H=2, kind="smooth", seed=49, rlat=2, rlon=1, backward=True)
+    scale = 0.2
+    x = synth.make_inputs(w)
+    dx = G.device_inputs(x)
+    idx = G.gpu_select(w, dx)
+    o, lse = G.gpu_fwd(w, dx, idx, scale)
+    dq, dk, dv = G.gpu_bwd(w, dx, o, lse, idx, scale)
+    g = G.geom_of(w, scale)
+    idx_h = idx.cpu().numpy()
+    for h in range(w.H):
+        G.compare_fwd_unit(w, x, 0, h, idx_h[0, h], o, lse, scale=scale)
+        dQ, dK, dV, _, _ = oracle.bwd(g, x["q"][0, h], x["k"][0, h], x["v"][0, h], x["do"][0, h], idx_h[0, h])
+        for name, got, want in (("dQ", dq, dQ), ("dK", dk, dK), ("dV", dv, dV)):
+            err = np.abs(got[0, h].float().cpu().numpy().astype(np.float64) - want).max()
+            assert err <= G.BWD_MAX_ABS, f"{name} max-abs {err:.4g}"
+
+
+def test_forward_largest_topk_and_16x16_radius_two():
+    for w in (synth.small_case(64, 96, 8, 8, 32, B=1, H=1, kind="smooth", seed=56),                    # top-k at its limit
+              synth.small_case(96, 96, 16, 16, 5, B=1, H=1, kind="smooth", seed=57, rlat=2, rlon=2)):  # 25 local blocks
+        x = synth.make_inputs(w)
+        dx = G.device_inputs(x)
+        idx = G.gpu_select(w, dx)
+        assert np.array_equal(idx.cpu().numpy(), G.oracle_select_all(w, x))
+        o, lse = G.gpu_fwd(w, dx, idx)
+        G.compare_fwd_unit(w, x, 0, 0, idx.cpu().numpy()[0, 0], o, lse)
+
+
 def test_backward_is_deterministic():
     w = BWD_CASES[0]
     dx = G.device_inputs(synth.make_inputs(w))

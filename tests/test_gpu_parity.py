@@ -213,6 +213,26 @@ def test_forward_largest_topk_and_16x16_radius_two():
         G.compare_fwd_unit(w, x, 0, 0, idx.cpu().numpy()[0, 0], o, lse)
 
 
+@pytest.mark.parametrize("nlat,nlon", [(8, 8), (8, 16), (16, 8), (8, 40)])
+def test_degenerate_grids_forward_and_backward(nlat, nlon):
+    """One block, one row or one column of blocks: neighbourhoods collapse onto themselves, nothing can be selected."""
+    w = synth.small_case(nlat, nlon, 8, 8, 3, B=1, H=2, seed=58 + nlat + nlon, backward=True)
+    x = synth.make_inputs(w)
+    dx = G.device_inputs(x)
+    idx = G.gpu_select(w, dx)
+    want = G.oracle_select_all(w, x)
+    assert np.array_equal(idx.cpu().numpy(), want)
+    o, lse = G.gpu_fwd(w, dx, idx)
+    dq, dk, dv = G.gpu_bwd(w, dx, o, lse, idx)
+    g = G.geom_of(w)
+    for h in range(w.H):
+        G.compare_fwd_unit(w, x, 0, h, want[0, h], o, lse)
+        dQ, dK, dV, _, _ = oracle.bwd(g, x["q"][0, h], x["k"][0, h], x["v"][0, h], x["do"][0, h], want[0, h])
+        for name, got, ref in (("dQ", dq, dQ), ("dK", dk, dK), ("dV", dv, dV)):
+            err = np.abs(got[0, h].float().cpu().numpy().astype(np.float64) - ref).max()
+            assert err <= G.BWD_MAX_ABS, f"{name} max-abs {err:.4g}"
+
+
 def test_backward_is_deterministic():
     w = BWD_CASES[0]
     dx = G.device_inputs(synth.make_inputs(w))

@@ -21,7 +21,9 @@
  *     block i, best first, padded with -1.  The local set is implicit.
  *   - The caller owns every buffer, including the workspace `ws` (device memory, 256-byte
  *     aligned, at least mosaic_bsa_workspace_bytes() long).  The library allocates no
- *     device memory and keeps no state beyond a host-side cache of TMA descriptors.
+ *     device memory.  Host-side state: a small cache of TMA descriptors keyed by (device, base
+ *     pointer, geometry) and per-device launch attributes; mosaic_bsa_select_static also keeps the
+ *     device address of its fixed scratch array.
  *   - Calls enqueue work on `cuda_stream` (a cudaStream_t, NULL = default stream) and
  *     return without synchronising.  Two calls that share a workspace must be ordered
  *     on one stream.
@@ -67,7 +69,8 @@ enum {
   MOSAIC_E_CUDA = -5,               /* a CUDA runtime/driver call failed (launch, query)  */
   /* device-side status codes (mosaic_bsa_last_status) */
   MOSAIC_E_DEVICE_TIMEOUT = -16,    /* a bounded wait on an on-chip barrier ran out       */
-  MOSAIC_E_DEVICE_BAD_INDEX = -17   /* block_idx held an id outside [-1, m)               */
+  MOSAIC_E_DEVICE_BAD_INDEX = -17   /* a row of block_idx held an id outside [-1, m), an id
+                                       inside the row's local set, or the same id twice      */
 };
 
 /* Bytes of device workspace the given op needs for these params (0 on invalid params).
@@ -82,7 +85,9 @@ size_t mosaic_bsa_workspace_bytes(const mosaic_bsa_params *p, int op);
  * Arithmetic is fixed so that the result is unique: block sums accumulate in fp64 in
  * row-major order inside the block and round once to fp32; a score is the fp64 sum, in
  * channel order, of the exact products of those fp32 values; order = (score descending,
- * block id ascending); +0 and -0 tie; a NaN score ranks last.
+ * block id ascending); +0 and -0 tie; a NaN score ranks after every number, -inf included
+ * (inputs are expected to be finite; this only fixes what happens when they are not).
+ * The selection kernels detect no device-side faults and never write the status word.
  */
 int mosaic_bsa_select(const mosaic_bsa_params *p, const void *q, const void *k, int32_t *block_idx,
                       void *ws, size_t ws_bytes, void *cuda_stream);
@@ -92,7 +97,10 @@ int mosaic_bsa_select(const mosaic_bsa_params *p, const void *q, const void *k, 
  * of local and selected blocks; streaming evaluation per the "Kernel Design" paragraph).
  *   q, k, v    in   [B,H,N,d] bf16
  *   block_idx  in   [B,H,m,topk] int32 (from mosaic_bsa_select or the caller: ids in
- *                   [0,m) or -1, no repeats in a row, none inside the row's local set)
+ *                   [0,m) or -1, no repeats in a row, none inside the row's local set.  An
+ *                   entry that breaks these rules is skipped -- a block is never attended
+ *                   twice -- and MOSAIC_E_DEVICE_BAD_INDEX is recorded; the backward applies
+ *                   the same rule, so it stays the gradient of what the forward computed)
  *   o          out  [B,H,N,d] bf16
  *   lse        out  [B,H,N] fp32, natural-log sum-exp of the scaled logits of each row
  */
@@ -133,7 +141,8 @@ int mosaic_bsa_bwd(const mosaic_bsa_params *p, const void *q, const void *k, con
  *   - All calls on a device share the one array, which keeps the previous call's contents (the call
  *     clears what has to start at zero).  Two calls that overlap on the GPU -- different streams without
  *     an ordering between them -- race on it: keep calls of this entry point ordered.
- *   - Other return codes as for mosaic_bsa_select.
+ *   - Other return codes as for mosaic_bsa_select.  There is no status word to read afterwards (the
+ *     selection kernels record no device-side faults), so mosaic_bsa_last_status has no counterpart here.
  */
 #define MOSAIC_BSA_STATIC_SCRATCH_BYTES (4u << 20)
 int mosaic_bsa_select_static(const mosaic_bsa_params *p, const void *q, const void *k, int32_t *block_idx,
@@ -143,6 +152,10 @@ int mosaic_bsa_select_static(const mosaic_bsa_params *p, const void *q, const vo
  * (MOSAIC_OK, MOSAIC_E_DEVICE_*) or MOSAIC_E_CUDA if the stream reports an error.
  * Every op resets the word when it starts. */
 int mosaic_bsa_last_status(const void *ws, void *cuda_stream);
+
+/* Diagnostic: how many TMA descriptors the library has encoded so far in this process.  A call that
+ * sees the same tensors (device, base pointers, geometry) as an earlier one encodes none. */
+long long mosaic_bsa_descriptor_encodes(void);
 
 /* Static, NUL-terminated description of a return code. */
 const char *mosaic_bsa_strerror(int code);

@@ -171,6 +171,25 @@ def bwd(g: Geom, q, k, v, d_o, idx):
     return dQ, dK, dV, O, L
 
 
+def bwd_blocks(g: Geom, q, k, v, d_o, idx, qblocks, kblocks):
+    """Backward of one unit restricted to lists of blocks: dQ [nq, b, d] of the query blocks in
+    `qblocks`, dK and dV [nk, b, d] of the key/value blocks in `kblocks` (fp64, rows in row-major
+    order inside each block).  Same arithmetic as `bwd`, for sizes at which a whole unit takes too long."""
+    q, k, v, d_o = _u16(q, g), _u16(k, g), _u16(v, g), _u16(d_o, g)
+    idx = np.ascontiguousarray(idx, np.int32).reshape(g.m, g.topk)
+    qb = np.ascontiguousarray(qblocks, np.int32)
+    kb = np.ascontiguousarray(kblocks, np.int32)
+    dQ = np.zeros((max(qb.size, 1), g.b, g.d)); dK = np.zeros((max(kb.size, 1), g.b, g.d)); dV = np.zeros_like(dK)
+    gc = g.c()
+    rc = _load().mo_bwd_blocks(ctypes.byref(gc), _p(q, ctypes.c_uint16), _p(k, ctypes.c_uint16),
+                               _p(v, ctypes.c_uint16), _p(d_o, ctypes.c_uint16), _p(idx, ctypes.c_int32),
+                               ctypes.c_int32(qb.size), _p(qb, ctypes.c_int32), _p(dQ, ctypes.c_double),
+                               ctypes.c_int32(kb.size), _p(kb, ctypes.c_int32), _p(dK, ctypes.c_double),
+                               _p(dV, ctypes.c_double))
+    assert rc == 0
+    return dQ[:qb.size], dK[:kb.size], dV[:kb.size]
+
+
 def block_tokens(g: Geom, j: int) -> np.ndarray:
     """Token ids of block j in row-major order inside the block (layout helper)."""
     by, bx = divmod(j, g.nbw)

@@ -367,3 +367,121 @@ int mo_bwd_unit(const mo_geom *g, const uint16_t *q, const uint16_t *k, const ui
   free(Ob); free(Lb); free(LSE); free(D);
   return 0;
 }
+
+/*
+ * Backward restricted to lists of blocks of one unit (same arithmetic as mo_bwd_unit, for sizes at
+ * which the whole unit takes too long): dQ for the query blocks in qblocks, dK and dV for the
+ * key/value blocks in kblocks.  dQ is [nq, b, d], dK and dV are [nk, b, d], rows in row-major order
+ * inside each block.  The forward quantities a gradient needs (LSE_l and D_l = dO_l . O_l) are
+ * computed for exactly the query blocks involved: the listed ones and every query block connected
+ * to a listed key/value block.
+ */
+int mo_bwd_blocks(const mo_geom *g, const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                  const uint16_t *d_o, const int32_t *idx, int32_t nq, const int32_t *qblocks, double *dQ,
+                  int32_t nk, const int32_t *kblocks, double *dK, double *dV) {
+  if (!g_ok(g)) return -1;
+  int m = g_m(g), b = g_b(g), d = g->d;
+  int64_t N = (int64_t)g->nlat * g->nlon;
+  int max_att = MO_MAX_LOCAL + g->topk;
+  double sc = g_scale(g);
+  for (int n = 0; n < nq; ++n) if (qblocks[n] < 0 || qblocks[n] >= m) return -1;
+  for (int n = 0; n < nk; ++n) if (kblocks[n] < 0 || kblocks[n] >= m) return -1;
+  /* which query blocks are involved */
+  unsigned char *need = (unsigned char *)calloc((size_t)m, 1);
+  int32_t *att0 = (int32_t *)malloc(sizeof(int32_t) * (size_t)max_att);
+  if (!need || !att0) { free(need); free(att0); return -2; }
+  for (int n = 0; n < nq; ++n) need[qblocks[n]] = 1;
+  for (int i = 0; i < m; ++i) {
+    int na = attended(g, idx, i, att0);
+    for (int a = 0; a < na; ++a)
+      for (int n = 0; n < nk; ++n) if (att0[a] == kblocks[n]) need[i] = 1;
+  }
+  free(att0);
+  int nn = 0;
+  for (int i = 0; i < m; ++i) nn += need[i];
+  int32_t *list = (int32_t *)malloc(sizeof(int32_t) * (size_t)(nn > 0 ? nn : 1));
+  double *Ob = (double *)malloc(sizeof(double) * (size_t)(nn > 0 ? nn : 1) * b * d);
+  double *Lb = (double *)malloc(sizeof(double) * (size_t)(nn > 0 ? nn : 1) * b);
+  double *LSE = (double *)malloc(sizeof(double) * (size_t)N);
+  double *D = (double *)malloc(sizeof(double) * (size_t)N);
+  if (!list || !Ob || !Lb || !LSE || !D) { free(need); free(list); free(Ob); free(Lb); free(LSE); free(D); return -2; }
+  nn = 0;
+  for (int i = 0; i < m; ++i) if (need[i]) list[nn++] = i;
+  mo_fwd_unit(g, q, k, v, idx, nn, list, Ob, Lb);
+  /* D_l = dO_l . O_l and LSE_l of the involved rows */
+#pragma omp parallel for schedule(static)
+  for (int n = 0; n < nn; ++n)
+    for (int e = 0; e < b; ++e) {
+      int64_t l = block_token(g, list[n], e);
+      double acc = 0.0;
+      for (int c = 0; c < d; ++c) acc += bf16_widen(d_o[l * d + c]) * Ob[((size_t)n * b + e) * d + c];
+      D[l] = acc;
+      LSE[l] = Lb[(size_t)n * b + e];
+    }
+  /* dQ of the listed query blocks: every row over its attended tokens */
+#pragma omp parallel
+  {
+    int32_t *att = (int32_t *)malloc(sizeof(int32_t) * (size_t)max_att);
+    double *x = (double *)malloc(sizeof(double) * (size_t)max_att * b);
+#pragma omp for schedule(dynamic, 1)
+    for (int n = 0; n < nq; ++n) {
+      int i = qblocks[n];
+      int na = attended(g, idx, i, att);
+      for (int e = 0; e < b; ++e) {
+        int64_t l = block_token(g, i, e);
+        row_logits(g, q, k, l, att, na, x);
+        double *dq = dQ + ((size_t)n * b + e) * d;
+        for (int c = 0; c < d; ++c) dq[c] = 0.0;
+        for (int a = 0; a < na; ++a)
+          for (int e2 = 0; e2 < b; ++e2) {
+            int64_t t = block_token(g, att[a], e2);
+            double w = exp(x[(size_t)a * b + e2] - LSE[l]);
+            double dP = 0.0;
+            for (int c = 0; c < d; ++c) dP += bf16_widen(d_o[l * d + c]) * bf16_widen(v[t * d + c]);
+            double dS = w * (dP - D[l]);
+            for (int c = 0; c < d; ++c) dq[c] += sc * dS * bf16_widen(k[t * d + c]);
+          }
+      }
+    }
+    free(att);
+    free(x);
+  }
+  /* dK, dV of the listed key/value blocks: every row over the query blocks connected to its block,
+   * query blocks in ascending order (rows of a key block are independent: parallel over them) */
+  for (int n = 0; n < nk; ++n) {
+    int j = kblocks[n];
+    int32_t *conn = (int32_t *)malloc(sizeof(int32_t) * (size_t)m);
+    int32_t *att = (int32_t *)malloc(sizeof(int32_t) * (size_t)max_att);
+    int nc = 0;
+    for (int i = 0; i < m; ++i) {
+      int na = attended(g, idx, i, att), connected = 0;
+      for (int a = 0; a < na; ++a) connected |= (att[a] == j);
+      if (connected) conn[nc++] = i;
+    }
+    free(att);
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int e2 = 0; e2 < b; ++e2) {
+      int64_t t = block_token(g, j, e2);
+      double *dk = dK + ((size_t)n * b + e2) * d, *dv = dV + ((size_t)n * b + e2) * d;
+      for (int c = 0; c < d; ++c) { dk[c] = 0.0; dv[c] = 0.0; }
+      for (int ci = 0; ci < nc; ++ci)
+        for (int e = 0; e < b; ++e) {
+          int64_t l = block_token(g, conn[ci], e);
+          double s = 0.0, dP = 0.0;
+          for (int c = 0; c < d; ++c) {
+            s += bf16_widen(q[l * d + c]) * bf16_widen(k[t * d + c]);
+            dP += bf16_widen(d_o[l * d + c]) * bf16_widen(v[t * d + c]);
+          }
+          double w = exp(sc * s - LSE[l]);
+          double dS = w * (dP - D[l]);
+          for (int c = 0; c < d; ++c) {
+            dv[c] += w * bf16_widen(d_o[l * d + c]);
+            dk[c] += sc * dS * bf16_widen(q[l * d + c]);
+          }
+        }
+    }
+    free(conn);
+  }
+  free(need); free(list); free(Ob); free(Lb); free(LSE); free(D);
+  return 0;
+}

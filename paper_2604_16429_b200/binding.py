@@ -19,7 +19,8 @@ _lib = None
 
 OP_SELECT, OP_FWD, OP_BWD = 0, 1, 2
 EXPORTS = ("mosaic_bsa_workspace_bytes", "mosaic_bsa_select", "mosaic_bsa_fwd", "mosaic_bsa_bwd",
-           "mosaic_bsa_last_status", "mosaic_bsa_strerror", "mosaic_bsa_select_static")
+           "mosaic_bsa_last_status", "mosaic_bsa_strerror", "mosaic_bsa_select_static",
+           "mosaic_bsa_descriptor_encodes")
 STATIC_SCRATCH_BYTES = 4 << 20
 
 
@@ -91,6 +92,8 @@ def lib():
         L.mosaic_bsa_bwd.argtypes = [pp, vp, vp, vp, vp, fp, vp, i32p, vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.mosaic_bsa_last_status.restype = ctypes.c_int
         L.mosaic_bsa_last_status.argtypes = [vp, vp]
+        L.mosaic_bsa_descriptor_encodes.restype = ctypes.c_longlong
+        L.mosaic_bsa_descriptor_encodes.argtypes = []
         L.mosaic_bsa_strerror.restype = ctypes.c_char_p
         L.mosaic_bsa_strerror.argtypes = [ctypes.c_int]
         _lib = L
@@ -188,6 +191,10 @@ def mosaic_bsa_bwd(p: Params, q, k, v, o, lse, d_o, block_idx, dq=None, dk=None,
 
 def mosaic_bsa_last_status(ws, stream=None) -> int:
     return int(lib().mosaic_bsa_last_status(_ptr(ws), _stream(stream)))
+
+
+def descriptor_encodes() -> int:
+    return int(lib().mosaic_bsa_descriptor_encodes())
 
 
 def check_status(ws, where: str, stream=None):

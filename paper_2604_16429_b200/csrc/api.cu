@@ -165,7 +165,7 @@ const char* mosaic_bsa_strerror(int code) {
     case MOSAIC_E_MISALIGNED: return "misaligned pointer";
     case MOSAIC_E_CUDA: return "CUDA call failed";
     case MOSAIC_E_DEVICE_TIMEOUT: return "device: bounded wait ran out";
-    case MOSAIC_E_DEVICE_BAD_INDEX: return "device: block id out of range";
+    case MOSAIC_E_DEVICE_BAD_INDEX: return "device: block id out of range, inside the local set, or repeated in its row";
     default: return "unknown code";
   }
 }

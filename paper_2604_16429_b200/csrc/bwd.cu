@@ -64,8 +64,9 @@ __global__ void __launch_bounds__(256) csr_kernel(Geo g, const int32_t* __restri
   for (int j = tid; j < g.m; j += blockDim.x) cur[j] = 0;
   __syncthreads();
   for (int e = tid; e < E; e += blockDim.x) {
-    int j = idx[e];
-    if (j >= 0 && j < g.m) atomicAdd(&cur[j], 1);
+    const int i = e / g.topk;
+    bool report;
+    if (selected_entry_ok(g, idx + (long long)i * g.topk, i, e - i * g.topk, &report)) atomicAdd(&cur[idx[e]], 1);
   }
   __syncthreads();
   if (tid < 32) {
@@ -85,8 +86,12 @@ __global__ void __launch_bounds__(256) csr_kernel(Geo g, const int32_t* __restri
     __syncwarp();
     for (int e0 = 0; e0 < E; e0 += 32) {
       int e = e0 + lane;
-      int j = e < E ? idx[e] : -1;
-      if (j >= g.m) j = -1;
+      int j = -1;
+      if (e < E) {
+        const int i = e / g.topk;
+        bool report;
+        if (selected_entry_ok(g, idx + (long long)i * g.topk, i, e - i * g.topk, &report)) j = idx[e];
+      }
       int key = j < 0 ? -1 - lane : j;  // invalid entries never match each other
       unsigned mask = __match_any_sync(0xffffffffu, key);
       int rank = __popc(mask & ((1u << lane) - 1u));

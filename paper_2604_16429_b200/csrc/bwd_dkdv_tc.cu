@@ -447,12 +447,9 @@ int launch_dkdv_tc(const HostCtx& c, const void* q, const void* k, const void* v
       !make_map_rows(&mnl, neg_lse2, g) || !make_map_rows(&mnd, neg_d, g))
     return MOSAIC_E_CUDA;
   const size_t smem = sizeof(Smem) + 1024;
-  int dev = 0, sms = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-    return MOSAIC_E_CUDA;
-  if (cudaFuncSetAttribute(dkdv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-    return MOSAIC_E_CUDA;
+  static unsigned long long configured = 0;  // devices on which the kernel's shared-memory opt-in is set
+  int sms = 0;
+  if (const int rc = launch_setup(reinterpret_cast<const void*>(dkdv_tc_kernel), smem, &configured, &sms)) return rc;
   const int ipu = items_per_unit(g);
   const long long total = 2ll * g.U * ipu;  // one item per 128-row tile
   if (total > 0x7fffff00ll) return MOSAIC_E_UNSUPPORTED;

@@ -31,24 +31,7 @@ struct Geo {
 // Record the first device-side fault in the workspace status word (never traps).
 __device__ __forceinline__ void set_status(int* status, int code) { atomicCAS(status, 0, code); }
 
-// Local neighbourhood of query block i: rows clamp(by+dy), columns (bx+dx) mod nbw, each
-// block once, in first-occurrence order (dy, then dx ascending).  Returns the count.
-__device__ __forceinline__ int local_set(const Geo& g, int i, int* out) {
-  int by = i / g.nbw, bx = i - by * g.nbw, n = 0;
-  for (int dy = -g.rlat; dy <= g.rlat; ++dy) {
-    int y = min(max(by + dy, 0), g.nbh - 1);
-    for (int dx = -g.rlon; dx <= g.rlon; ++dx) {
-      int x = (bx + dx) % g.nbw;
-      x += x < 0 ? g.nbw : 0;
-      int id = y * g.nbw + x;
-      bool seen = false;
-      for (int a = 0; a < n; ++a) seen |= (out[a] == id);
-      if (!seen) out[n++] = id;
-    }
-  }
-  return n;
-}
-
+// Is key block j inside the local neighbourhood of query block i (rows clamp(by+dy), columns (bx+dx) mod nbw)?
 __device__ __forceinline__ bool is_local(const Geo& g, int i, int j) {
   int by = i / g.nbw, bx = i - by * g.nbw;
   int jy = j / g.nbw, jx = j - jy * g.nbw;
@@ -60,21 +43,20 @@ __device__ __forceinline__ bool is_local(const Geo& g, int i, int j) {
   return row_ok && col_ok;
 }
 
-// Attended list of query block i: local set followed by the valid selected ids.
-// Ids outside [-1, m) are skipped and reported.  `out` holds kMaxList entries.
-__device__ __forceinline__ int attended_list(const Geo& g, const int32_t* __restrict__ idx_row, int i,
-                                             int* out, int* status) {
-  int n = local_set(g, i, out);
-  for (int r = 0; r < g.topk; ++r) {
-    int j = idx_row[r];
-    if (j < 0) {
-      if (j != -1) set_status(status, MOSAIC_E_DEVICE_BAD_INDEX);
-      continue;
-    }
-    if (j >= g.m) { set_status(status, MOSAIC_E_DEVICE_BAD_INDEX); continue; }
-    if (n < kMaxList) out[n++] = j;
-  }
-  return n;
+// Is entry r of a row of block_idx (query block i) one the kernels use?  Ids outside [0, m), ids inside the
+// row's local set (already attended through the neighbourhood) and repeats of an earlier entry of the row are
+// not: they are skipped, and reported unless the entry is the padding value -1.
+__device__ __forceinline__ bool selected_entry_ok(const Geo& g, const int32_t* __restrict__ idx_row, int i, int r,
+                                                  bool* report) {
+  const int j = idx_row[r];
+  *report = false;
+  if (j == -1) return false;
+  *report = true;
+  if (j < 0 || j >= g.m || is_local(g, i, j)) return false;
+  for (int a = 0; a < r; ++a)
+    if (idx_row[a] == j) return false;
+  *report = false;
+  return true;
 }
 
 // First token (row-major grid index inside the unit) of row `r` of chunk `c` of block j.

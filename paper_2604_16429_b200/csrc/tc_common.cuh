@@ -269,7 +269,7 @@ __host__ __device__ inline int items_per_unit(const Geo& g) {
 }
 
 // Warp-cooperative attended list of query block i (local set, then valid selected ids) written to
-// ids[n0..); returns the new count.
+// ids[n0..); returns the new count.  `j` is this lane's entry of the block's row of block_idx (-1 beyond top-k).
 __device__ __forceinline__ int warp_attended(const Geo& g, int j, int i, int* ids, int n0, int lane, int* status) {
   const int by = i / g.nbw, bx = i - by * g.nbw;
   const int wl = 2 * g.rlon + 1, nl = (2 * g.rlat + 1) * wl;
@@ -286,7 +286,12 @@ __device__ __forceinline__ int warp_attended(const Geo& g, int j, int i, int* id
   const unsigned km = __ballot_sync(0xffffffffu, keep);
   if (keep) ids[n0 + __popc(km & ((1u << lane) - 1u))] = id;
   int n = n0 + __popc(km);
-  if (j < -1 || j >= g.m) { set_status(status, MOSAIC_E_DEVICE_BAD_INDEX); j = -1; }
+  // selected ids outside [-1, m), inside the local set (attended already) or repeated in the row: skipped, reported
+  const unsigned twins = __match_any_sync(0xffffffffu, j);
+  if (j != -1 && (j < 0 || j >= g.m || is_local(g, i, j) || (__ffs(twins) - 1) != lane)) {
+    set_status(status, MOSAIC_E_DEVICE_BAD_INDEX);
+    j = -1;
+  }
   const unsigned sm_ = __ballot_sync(0xffffffffu, j >= 0);
   if (j >= 0) ids[n + __popc(sm_ & ((1u << lane) - 1u))] = j;
   return n + __popc(sm_);
@@ -484,50 +489,6 @@ __device__ __forceinline__ void planner_loop(SM& sm, const Geo& g, const int32_t
   }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
-        qres != cudaDriverEntryPointSuccess)
-      return nullptr;
-    fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
-  return fn;
-}
-
-// [U, nlat, nlon, d] bf16 view, box = one 64-token chunk {d, bw, 64/bw, 1}, 128-byte swizzle.
-bool make_map(CUtensorMap* map, const void* base, const Geo& g) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)g.nlon, (cuuint64_t)g.nlat, (cuuint64_t)g.U};
-  cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)g.nlon * kD * 2, (cuuint64_t)g.N * kD * 2};
-  cuuint32_t box[4] = {(cuuint32_t)kD, (cuuint32_t)g.bw, (cuuint32_t)g.crows, 1u};
-  cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-
-// [U, nlat, nlon] fp32 view (one value per token), box = the 64 tokens of one chunk {bw, 64/bw, 1}, no swizzle.
-bool make_map_rows(CUtensorMap* map, const void* base, const Geo& g) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  cuuint64_t dims[3] = {(cuuint64_t)g.nlon, (cuuint64_t)g.nlat, (cuuint64_t)g.U};
-  cuuint64_t strides[2] = {(cuuint64_t)g.nlon * 4, (cuuint64_t)g.N * 4};
-  cuuint32_t box[3] = {(cuuint32_t)g.bw, (cuuint32_t)g.crows, 1u};
-  cuuint32_t estr[3] = {1u, 1u, 1u};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
                                             int c2) {
   asm volatile(
@@ -537,5 +498,16 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 }  // namespace
+
+// ---- host side (tmap.cu) -------------------------------------------------------------------
+// TMA descriptors are cached per (device, base pointer, geometry), so a call that sees the same tensors
+// again encodes nothing.
+// [U, nlat, nlon, d] bf16 view, box = one 64-token chunk {d, bw, 64/bw, 1}, 128-byte swizzle.
+bool make_map(CUtensorMap* map, const void* base, const Geo& g);
+// [U, nlat, nlon] fp32 view (one value per token), box = the 64 tokens of one chunk {bw, 64/bw, 1}, no swizzle.
+bool make_map_rows(CUtensorMap* map, const void* base, const Geo& g);
+// Current device, its SM count (cached), and the opt-in to `smem` bytes of dynamic shared memory for `func`
+// (set once per device; `done` is the caller's per-kernel bit set of devices already configured).
+int launch_setup(const void* func, size_t smem, unsigned long long* done, int* sms);
 
 }  // namespace mosaic

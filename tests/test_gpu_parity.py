@@ -115,6 +115,76 @@ def test_forward_is_deterministic_and_writes_everything():
     assert torch.equal(o1.view(torch.int16), o2.view(torch.int16)) and torch.equal(l1, l2)
 
 
+def test_select_nan_and_infinite_scores():
+    """A NaN pooled sum gives NaN scores: that block ranks after every number (also after -inf), and is
+    chosen only where fewer than top-k other candidates exist.  Same ids as the oracle, bit for bit."""
+    w = synth.small_case(32, 64, 8, 8, 4, B=1, H=2, seed=39)
+    x = synth.make_inputs(w)
+    k = x["k"].copy()
+    k[0, 0, 5 * 64 + 17, 3] = 0x7FC0                      # NaN inside key block (0, 2) of unit 0
+    k[0, 0, 20 * 64 + 40, 9] = 0xFF80                     # -inf inside key block (2, 5) of unit 0
+    k[0, 1, 9 * 64 + 3, 0] = 0x7F80                       # +inf inside key block (1, 0) of unit 1
+    x["k"] = k
+    want = G.oracle_select_all(w, x)
+    got = G.gpu_select(w, G.device_inputs(x)).cpu().numpy()
+    assert np.array_equal(got, want), f"{(got != want).sum()} of {want.size} ids differ"
+    wn = synth.small_case(16, 40, 8, 8, 4, B=1, H=1, seed=40)          # 4 candidates per row: NaN blocks must be listed last
+    xn = synth.make_inputs(wn)
+    kn = xn["k"].copy()
+    kn[0, 0, 3 * 40 + 20, 1] = 0x7FC0                     # block (0, 2)
+    kn[0, 0, 12 * 40 + 30, 1] = 0x7FC0                    # block (1, 3)
+    xn["k"] = kn
+    want = G.oracle_select_all(wn, xn)
+    got = G.gpu_select(wn, G.device_inputs(xn)).cpu().numpy()
+    assert np.array_equal(got, want)
+    assert (want[0, 0, 0] >= 0).all() and set(want[0, 0, 0][2:].tolist()) == {2, 8}
+
+
+def test_repeated_and_local_ids_are_skipped_and_reported():
+    """A caller's block_idx row that repeats an id or names a block of the row's own neighbourhood: the extra
+    entries are ignored (no block is attended twice) in forward and backward, and the status word says so."""
+    w = synth.small_case(32, 64, 8, 8, 4, B=1, H=1, seed=60, backward=True)
+    x = synth.make_inputs(w)
+    dx = G.device_inputs(x)
+    idx = G.gpu_select(w, dx)
+    clean = idx.clone()
+    clean[0, 0, 10, 2:] = -1
+    dirty = clean.clone()
+    dirty[0, 0, 10, 2] = clean[0, 0, 10, 0]                # repeat of entry 0
+    dirty[0, 0, 10, 3] = 11                                # right-hand neighbour of block 10: local
+    p = mb.Params.from_workload(w)
+    ws = mb.alloc_workspace(p, mb.OP_BWD)
+    o1, l1 = mb.mosaic_bsa_fwd(p, dx["q"], dx["k"], dx["v"], clean, ws=ws)
+    assert mb.mosaic_bsa_last_status(ws) == 0
+    o2, l2 = mb.mosaic_bsa_fwd(p, dx["q"], dx["k"], dx["v"], dirty, ws=ws)
+    assert mb.mosaic_bsa_last_status(ws) == -17
+    assert torch.equal(o1.view(torch.int16), o2.view(torch.int16)) and torch.equal(l1, l2)
+    G.compare_fwd_unit(w, x, 0, 0, clean.cpu().numpy()[0, 0], o2, l2)
+    g1 = mb.mosaic_bsa_bwd(p, dx["q"], dx["k"], dx["v"], o1, l1, dx["do"], clean, ws=ws)
+    assert mb.mosaic_bsa_last_status(ws) == 0
+    g2 = mb.mosaic_bsa_bwd(p, dx["q"], dx["k"], dx["v"], o1, l1, dx["do"], dirty, ws=ws)
+    assert mb.mosaic_bsa_last_status(ws) == -17
+    for a, b in zip(g1, g2):
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+
+
+def test_descriptor_cache_encodes_once_per_tensor():
+    w = synth.small_case(32, 64, 8, 8, 4, B=1, H=1, seed=59)
+    dx = G.device_inputs(synth.make_inputs(w))
+    p = mb.Params.from_workload(w)
+    ws = mb.alloc_workspace(p, mb.OP_FWD)
+    idx = mb.mosaic_bsa_select(p, dx["q"], dx["k"], ws=mb.alloc_workspace(p, mb.OP_SELECT))
+    o = torch.empty_like(dx["q"])
+    lse = torch.empty((w.B, w.H, w.N), dtype=torch.float32, device="cuda")
+    n0 = mb.descriptor_encodes()
+    mb.mosaic_bsa_fwd(p, dx["q"], dx["k"], dx["v"], idx, o=o, lse=lse, ws=ws)
+    n1 = mb.descriptor_encodes()
+    mb.mosaic_bsa_fwd(p, dx["q"], dx["k"], dx["v"], idx, o=o, lse=lse, ws=ws)
+    n2 = mb.descriptor_encodes()
+    assert 1 <= n1 - n0 <= 4 and n2 == n1                  # Q, K, V (and O) once; nothing on the second call
+    mb.check_status(ws, "fwd")
+
+
 def test_bad_block_id_is_reported_not_dereferenced():
     w = synth.small_case(32, 64, 8, 8, 4, B=1, H=1, seed=38)
     dx = G.device_inputs(synth.make_inputs(w))
@@ -150,10 +220,8 @@ def test_backward_matches_oracle(w):
         for h in range(w.H):
             dQ, dK, dV, _, _ = oracle.bwd(g, x["q"][b, h], x["k"][b, h], x["v"][b, h], x["do"][b, h], idx_h[b, h])
             for name, got, want in (("dQ", dq, dQ), ("dK", dk, dK), ("dV", dv, dV)):
+                G.assert_bwd_close(name, got[b, h], want)
                 gh = got[b, h].float().cpu().numpy().astype(np.float64)
-                assert np.isfinite(gh).all(), name
-                err = np.abs(gh - want).max()
-                assert err <= G.BWD_MAX_ABS, f"{name} max-abs {err:.4g}"
                 assert np.abs(gh - want).mean() <= 0.1 * max(np.abs(want).mean(), 1e-3), name
 
 
@@ -176,12 +244,40 @@ def test_backward_popular_key_blocks_lists_span_several_buffers():
     o, lse = G.gpu_fwd(w, dx, idx)
     dq, dk, dv = G.gpu_bwd(w, dx, o, lse, idx)
     dQ, dK, dV, _, _ = oracle.bwd(G.geom_of(w), x["q"][0, 0], x["k"][0, 0], x["v"][0, 0], x["do"][0, 0], idx_h)
+    assert np.abs(dV).max() > 20                                  # gradients large enough that bf16 storage sets the error
     for name, got, want in (("dQ", dq, dQ), ("dK", dk, dK), ("dV", dv, dV)):
-        gh = got[0, 0].float().cpu().numpy().astype(np.float64)
-        assert np.isfinite(gh).all(), name
-        # dK and dV of the popular blocks sum several hundred bf16-rounded terms: compare relative to the scale
-        err = np.abs(gh - want)
-        assert (err <= G.BWD_MAX_ABS + 1e-2 * np.abs(want)).all(), f"{name} max-abs {err.max():.4g}"
+        G.assert_bwd_close(name, got[0, 0], want)
+
+
+def test_backward_popular_key_block_with_four_chunks_per_block():
+    """The same continuation of a long list over several list buffers, with 16x16 blocks (four 64-token chunks
+    per block, the 0.25-degree shape): one key block that nearly every query block selects."""
+    w = synth.small_case(240, 320, 16, 16, 4, B=1, H=1, seed=50, backward=True)    # 15 x 20 blocks, m = 300
+    x = synth.make_inputs(w)
+    kf = synth.bf16_bits_to_f32(x["k"]).reshape(1, 1, 240, 320, 64).copy()
+    qf = synth.bf16_bits_to_f32(x["q"]).reshape(1, 1, 240, 320, 64).copy()
+    qf[..., 0] = np.abs(qf[..., 0]) + 1.0
+    kf[:, :, 112:128, 144:160, 0] = 6.0                         # block (7, 9)
+    x["k"] = synth.to_bf16_bits(kf.reshape(1, 1, -1, 64))
+    x["q"] = synth.to_bf16_bits(qf.reshape(1, 1, -1, 64))
+    dx = G.device_inputs(x)
+    idx = G.gpu_select(w, dx)
+    idx_h = idx.cpu().numpy()[0, 0]
+    g = G.geom_of(w)
+    assert np.array_equal(idx_h, oracle.select(g, x["q"][0, 0], x["k"][0, 0]))
+    popular = 7 * 20 + 9
+    assert (idx_h == popular).any(axis=1).sum() > 260           # in-degree beyond one list buffer (256 entries)
+    o, lse = G.gpu_fwd(w, dx, idx)
+    dq, dk, dv = G.gpu_bwd(w, dx, o, lse, idx)
+    qb = np.array([0, popular, 299], np.int32)
+    kb = np.array([popular, popular + 1, 0], np.int32)
+    dQ, dK, dV = oracle.bwd_blocks(g, x["q"][0, 0], x["k"][0, 0], x["v"][0, 0], x["do"][0, 0], idx_h, qb, kb)
+    for n, i in enumerate(qb):
+        G.assert_bwd_close(f"dQ block {i}", dq[0, 0][oracle.block_tokens(g, int(i))], dQ[n])
+    for n, j in enumerate(kb):
+        tj = oracle.block_tokens(g, int(j))
+        G.assert_bwd_close(f"dK block {j}", dk[0, 0][tj], dK[n])
+        G.assert_bwd_close(f"dV block {j}", dv[0, 0][tj], dV[n])
 
 
 def test_backward_custom_scale_and_wide_neighbourhood():
@@ -198,8 +294,7 @@ def test_backward_custom_scale_and_wide_neighbourhood():
         G.compare_fwd_unit(w, x, 0, h, idx_h[0, h], o, lse, scale=scale)
         dQ, dK, dV, _, _ = oracle.bwd(g, x["q"][0, h], x["k"][0, h], x["v"][0, h], x["do"][0, h], idx_h[0, h])
         for name, got, want in (("dQ", dq, dQ), ("dK", dk, dK), ("dV", dv, dV)):
-            err = np.abs(got[0, h].float().cpu().numpy().astype(np.float64) - want).max()
-            assert err <= G.BWD_MAX_ABS, f"{name} max-abs {err:.4g}"
+            G.assert_bwd_close(name, got[0, h], want)
 
 
 def test_forward_largest_topk_and_16x16_radius_two():
@@ -229,8 +324,7 @@ def test_degenerate_grids_forward_and_backward(nlat, nlon):
         G.compare_fwd_unit(w, x, 0, h, want[0, h], o, lse)
         dQ, dK, dV, _, _ = oracle.bwd(g, x["q"][0, h], x["k"][0, h], x["v"][0, h], x["do"][0, h], want[0, h])
         for name, got, ref in (("dQ", dq, dQ), ("dK", dk, dK), ("dV", dv, dV)):
-            err = np.abs(got[0, h].float().cpu().numpy().astype(np.float64) - ref).max()
-            assert err <= G.BWD_MAX_ABS, f"{name} max-abs {err:.4g}"
+            G.assert_bwd_close(name, got[0, h], ref)
 
 
 def test_backward_is_deterministic():

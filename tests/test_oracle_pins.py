@@ -125,6 +125,35 @@ def test_selection_known_winners_and_ties():
     assert idx[i].tolist() == [j for j in range(g.m) if j not in loc][:3]
 
 
+def test_selection_nan_score_ranks_below_every_number():
+    """A key block whose pooled sum is NaN gives a NaN score: it ranks after every finite or infinite
+    score (so it is chosen only when fewer than top-k other candidates exist), lower id first among NaNs."""
+    g = Geom(32, 64, d=8, bh=8, bw=8, topk=3)        # 4 x 8 blocks, m = 32
+    pq = np.zeros((g.m, g.d), np.float32)
+    pk = np.zeros((g.m, g.d), np.float32)
+    pq[:, 0] = 1.0
+    pk[:, 0] = -np.arange(g.m, dtype=np.float32)     # block 0 best, block 31 worst
+    i = 1 * g.nbw + 1                                # local = rows 0..2, cols 0..2
+    loc = local_blocks(1, 1, g.nbh, g.nbw)
+    cand = [j for j in range(g.m) if j not in loc]
+    kb = _blocks_from_pooled(g, pk)
+    kb[block_tokens(g.nlon, g.bh, g.bw, g.nbw, cand[0])[0], 0] = 0x7FC0      # bf16 NaN in the best candidate
+    idx = oracle.select(g, _blocks_from_pooled(g, pq), kb)
+    assert idx[i].tolist() == cand[1:4]                                     # the NaN block is passed over
+    # -inf is a number: it still ranks above NaN
+    g2 = Geom(16, 40, d=8, bh=8, bw=8, topk=4)       # 2 x 5 blocks: 4 candidates per row
+    pq2 = np.zeros((g2.m, g2.d), np.float32); pq2[:, 0] = 1.0
+    pk2 = np.zeros((g2.m, g2.d), np.float32); pk2[:, 0] = np.arange(g2.m, dtype=np.float32)
+    kb2 = _blocks_from_pooled(g2, pk2)
+    loc2 = local_blocks(0, 0, g2.nbh, g2.nbw)
+    cand2 = [j for j in range(g2.m) if j not in loc2]                        # [2, 3, 7, 8]
+    kb2[block_tokens(g2.nlon, g2.bh, g2.bw, g2.nbw, cand2[3])[0], 0] = 0x7FC0   # NaN (would be the best)
+    kb2[block_tokens(g2.nlon, g2.bh, g2.bw, g2.nbw, cand2[1])[0], 0] = 0x7FC0   # NaN
+    kb2[block_tokens(g2.nlon, g2.bh, g2.bw, g2.nbw, cand2[2])[0], 0] = 0xFF80   # -inf
+    idx2 = oracle.select(g2, _blocks_from_pooled(g2, pq2), kb2)
+    assert idx2[0].tolist() == [cand2[0], cand2[2], cand2[1], cand2[3]]      # finite, -inf, then NaNs by id
+
+
 def test_selection_padding_when_few_candidates():
     g = Geom(16, 32, d=8, bh=8, bw=8, topk=4)        # 2 x 4 blocks: local covers 6 of 8
     rng = np.random.default_rng(3)
@@ -325,6 +354,39 @@ def test_backward_visits_only_connected_blocks_and_shift_invariance():
     assert np.abs(dK.sum(axis=0)).max() < 1e-10 * np.abs(dK).sum()
     # sum_t dV_t = sum_l dO_l because the weights of each row sum to one
     assert np.abs(dV.sum(axis=0) - f64(do).sum(axis=0)).max() < 1e-9
+
+
+def test_backward_on_block_lists_equals_the_whole_unit_and_the_dense_formula():
+    """`bwd_blocks` (gradients of listed blocks only) against the whole-unit backward, which the tests above
+    pin, and against the dense softmax-attention gradient written out here when every block is attended."""
+    rng = np.random.default_rng(14)
+    g = Geom(32, 48, d=8, bh=8, bw=8, topk=3)        # m = 24, sparse pattern
+    q, k, v, do = (rand_bits(rng, g.N, g.d) for _ in range(4))
+    idx = oracle.select(g, q, k)
+    dQ, dK, dV, _, _ = oracle.bwd(g, q, k, v, do, idx)
+    qb, kb = [0, 7, 23, 12], [5, 23, 0]
+    bQ, bK, bV = oracle.bwd_blocks(g, q, k, v, do, idx, qb, kb)
+    for n, i in enumerate(qb):
+        assert np.abs(bQ[n] - dQ[block_tokens(g.nlon, g.bh, g.bw, g.nbw, i)]).max() < 1e-12
+    for n, j in enumerate(kb):
+        tj = block_tokens(g.nlon, g.bh, g.bw, g.nbw, j)
+        assert np.abs(bK[n] - dK[tj]).max() < 1e-12 and np.abs(bV[n] - dV[tj]).max() < 1e-12
+    assert np.abs(bK).max() > 1e-3 and np.abs(bQ).max() > 1e-3
+    # dense case, independent formula
+    g = Geom(16, 24, d=8, bh=8, bw=8, topk=6)
+    q, k, v, do = (rand_bits(rng, g.N, g.d) for _ in range(4))
+    idx = oracle.select(g, q, k)
+    qf, kf, vf, dof = f64(q), f64(k), f64(v), f64(do)
+    sc = 1 / math.sqrt(g.d)
+    x = sc * qf @ kf.T
+    P = np.exp(x - x.max(1, keepdims=True)); P /= P.sum(1, keepdims=True)
+    dS = P * (dof @ vf.T - (dof * (P @ vf)).sum(1, keepdims=True))
+    bQ, bK, bV = oracle.bwd_blocks(g, q, k, v, do, idx, [4], [1, 5])
+    assert np.abs(bQ[0] - (sc * dS @ kf)[block_tokens(g.nlon, g.bh, g.bw, g.nbw, 4)]).max() < 1e-11
+    for n, j in enumerate([1, 5]):
+        tj = block_tokens(g.nlon, g.bh, g.bw, g.nbw, j)
+        assert np.abs(bK[n] - (sc * dS.T @ qf)[tj]).max() < 1e-11
+        assert np.abs(bV[n] - (P.T @ dof)[tj]).max() < 1e-11
 
 
 # ------------------------------------------------------------------ cost model

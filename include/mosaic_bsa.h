@@ -127,14 +127,15 @@ int mosaic_bsa_bwd(const mosaic_bsa_params *p, const void *q, const void *k, con
  * Some callers cannot hand the library a workspace: a process whose framework claimed its whole memory
  * budget at start-up, a plug-in whose host application owns the allocator, a latency-critical loop in
  * which cudaMalloc (it may synchronise the device) is forbidden.  For them the scratch of the selection
- * (the pooled block sums of Q and K) lives in a fixed array inside the library image,
+ * (the pooled block sums of Q and K and the norms of those sums) lives in a fixed array inside the library image,
  * MOSAIC_BSA_STATIC_SCRATCH_BYTES long; every GPU that loads the library holds that array until the
  * process exits.  The call performs no cudaMalloc, cudaFree or other allocating routine.
  *   q, k       in   [B,H,N,d] bf16 (device)
  *   block_idx  out  [B,H,m,topk] int32 (device)
  * Limits and rules
- *   - The problem must fit: 256 + 2 * round_up_256(B*H*m*d*4) <= MOSAIC_BSA_STATIC_SCRATCH_BYTES,
- *     i.e. about B*H*m <= 8190 blocks for d = 64 (the 1.5-degree grid with 8 heads uses 3600).  A larger
+ *   - The problem must fit: 256 + 2 * round_up_256(B*H*m*d*4) + 2 * round_up_256(B*H*m*4)
+ *     <= MOSAIC_BSA_STATIC_SCRATCH_BYTES (= mosaic_bsa_workspace_bytes(p, MOSAIC_OP_SELECT)), i.e. about
+ *     B*H*m <= 8060 blocks for d = 64 (the 1.5-degree grid with 8 heads uses 3600).  A larger
  *     problem returns MOSAIC_E_WORKSPACE_TOO_SMALL and launches nothing.
  *   - The first call on each device looks up the device address of the array (with that device current)
  *     and remembers it; make that first call before any stream capture begins.

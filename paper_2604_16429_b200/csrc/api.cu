@@ -38,6 +38,17 @@ int validate(const mosaic_bsa_params* p, Geo* g) {
   return MOSAIC_OK;
 }
 
+SelectWs select_layout(const Geo& g) {
+  SelectWs w;
+  const size_t pooled = align256(sizeof(float) * (size_t)g.U * g.m * kD), norms = align256(sizeof(float) * (size_t)g.U * g.m);
+  w.pq = kStatusBytes;
+  w.pk = w.pq + pooled;
+  w.nq = w.pk + pooled;
+  w.nk = w.nq + norms;
+  w.total = w.nk + norms;
+  return w;
+}
+
 namespace {
 
 struct BwdWs { size_t D, negD, nlse2, off, q, total; };
@@ -52,7 +63,7 @@ BwdWs bwd_layout(const Geo& g) {
   w.total = at;
   return w;
 }
-size_t select_total(const Geo& g) { return kStatusBytes + 2 * align256(sizeof(float) * (size_t)g.U * g.m * kD); }
+size_t select_total(const Geo& g) { return select_layout(g).total; }
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
@@ -107,9 +118,10 @@ int mosaic_bsa_select(const mosaic_bsa_params* p, const void* q, const void* k, 
   if (!q || !k || (!block_idx && g.topk > 0)) return MOSAIC_E_INVALID_ARG;
   if (!aligned(q, 16) || !aligned(k, 16) || !aligned(block_idx, 4)) return MOSAIC_E_MISALIGNED;
   if ((rc = begin(p, ws, ws_bytes, select_total(g), cuda_stream, &c))) return rc;
-  float* pq = (float*)((char*)ws + kStatusBytes);
-  float* pk = (float*)((char*)pq + align256(sizeof(float) * (size_t)g.U * g.m * kD));
-  return launch_select(c, q, k, block_idx, pq, pk);
+  const SelectWs w = select_layout(g);
+  char* base = (char*)ws;
+  return launch_select(c, q, k, block_idx, (float*)(base + w.pq), (float*)(base + w.pk), (float*)(base + w.nq),
+                       (float*)(base + w.nk));
 }
 
 int mosaic_bsa_fwd(const mosaic_bsa_params* p, const void* q, const void* k, const void* v,

@@ -82,8 +82,12 @@ int validate(const mosaic_bsa_params* p, Geo* g);
 size_t align256(size_t x);
 
 // kernel launchers (one per translation unit)
+// Layout of the selection's scratch behind the status block: pooled sums of Q and of K ([U, m, d] fp32 each),
+// then the norm bounds of the pooled vectors ([U, m] fp32 each).
+struct SelectWs { size_t pq, pk, nq, nk, total; };
+SelectWs select_layout(const Geo& g);
 int launch_select(const HostCtx& c, const void* q, const void* k, int32_t* block_idx, float* pooled_q,
-                  float* pooled_k);
+                  float* pooled_k, float* norm_q, float* norm_k);
 int launch_fwd_tc(const HostCtx& c, const void* q, const void* k, const void* v, const int32_t* block_idx,
                   void* o, float* lse);
 int launch_dq_tc(const HostCtx& c, const void* q, const void* k, const void* v, const void* d_o, const float* lse,

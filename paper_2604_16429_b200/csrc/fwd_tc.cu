@@ -23,8 +23,11 @@
 // warp walks the loop, one elected lane issues), warp 11 draws items from the queue and builds their key
 // lists one item ahead, interleaved so that both tiles find work all along a list.
 // TMEM (512 columns): O of tile t at 64 t (fp32, 64 columns); two S buffers per tile at 128 + 128 t + 64 b
-// (fp32, 64 columns each).  P (bf16) overwrites the first 32 columns of its S buffer and is the TMEM A
-// operand of PV.  QK^T of product n+1 is issued before P V of product n, so the tensor core fills one S
+// (fp32, 64 columns each); the query tile of tile t (bf16, 32 columns) at 384 + 32 t.  P (bf16) overwrites
+// the first 32 columns of its S buffer and is the TMEM A operand of PV.  The query tile is a TMEM A operand
+// too: the softmax threads copy their rows there once per item, so QK^T reads only the key chunk from shared
+// memory (with both operands in shared memory an N = 64 product is bound by shared-memory bandwidth, not by
+// the tensor core).  QK^T of product n+1 is issued before P V of product n, so the tensor core fills one S
 // buffer while the softmax warps work on the other.
 // Softmax: fp32, base-2 exponentials with the scale folded in, running maximum moved only when it grows by
 // more than 2^8 (then O is rescaled, between two P V products), packed two-lane fp32 arithmetic, and a
@@ -43,6 +46,7 @@ constexpr int kStages = 8;                       // key/value ring depth (K + V 
 constexpr int kThreads = 384;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColO = 0, kColS = 128;       // O of tile t at 64 t; S buffer b of tile t at 128 + 128 t + 64 b
+constexpr uint32_t kColQ = 384;                  // query tile of tile t (bf16 pairs) at 384 + 32 t
 constexpr int kPolyEvery = 2;                   // one pair in every kPolyEvery groups of four logits takes the FMA-pipe exp2
 constexpr float kRescaleThreshold = 8.0f;        // log2 units: P stays below 2^8
 
@@ -51,6 +55,7 @@ struct Smem {
   unsigned char kv[kStages][2][kTile];     // [stage][K, V]
   unsigned long long kv_full[kStages], kv_empty[kStages];
   unsigned long long q_full[2][2], q_empty[2][2];  // [item parity][tile]
+  unsigned long long q_ready[2];                   // [tile]: the item's query rows are in TMEM
   unsigned long long s_full[2][2], p_full[2][2], pv_done[2][2];  // [tile][S buffer]
   unsigned long long list_full[kLists], list_empty[kLists];
   uint32_t tmem_base;
@@ -78,8 +83,9 @@ __global__ void __launch_bounds__(kThreads, 1)
     for (int t = 0; t < 2; ++t) {
       for (int b = 0; b < 2; ++b) {
         mbar_init(s32(&sm.q_full[b][t]), 1);
-        mbar_init(s32(&sm.q_empty[b][t]), 1);
+        mbar_init(s32(&sm.q_empty[b][t]), 128);
       }
+      mbar_init(s32(&sm.q_ready[t]), 128);
       for (int b = 0; b < 2; ++b) {
         mbar_init(s32(&sm.s_full[t][b]), 1);
         mbar_init(s32(&sm.p_full[t][b]), 128);
@@ -122,8 +128,8 @@ __global__ void __launch_bounds__(kThreads, 1)
         const ItemInfo& inf = sm.info[buf];
         const int n = inf.n, u = inf.unit;
         if (n < 0) break;
-        // query tiles (double-buffered by item parity): free once the tile's last QK^T of the item before
-        // the previous one has completed, so this load runs while the previous item still computes
+        // query tiles (double-buffered by item parity): free once the softmax threads have copied the rows of
+        // the item before the previous one to TMEM, so this load runs while the previous item still computes
         for (int t = 0; t < 2 && ok; ++t) {
           ok = mbar_wait(s32(&sm.q_empty[qb][t]), ((it >> 1) & 1) ^ 1, abort, status);
           if (!ok) break;
@@ -164,7 +170,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     // fills the next S while the softmax warps work on the current one.
     const int t = warp - 9;
     constexpr uint32_t idesc_qk = make_idesc(false), idesc_pv = make_idesc(true);
-    const uint32_t tcol_o = tmem + kColO + 64 * t, tcol_s = tmem + kColS + 128 * t;
+    const uint32_t tcol_o = tmem + kColO + 64 * t, tcol_s = tmem + kColS + 128 * t, tcol_q = tmem + kColQ + 32 * t;
     const uint32_t tbits = 3u << (2 * t);
     long long step = 0;   // ring position (all chunks, attended by this tile or not)
     uint32_t nt = 0;      // products issued by this tile so far: buffer nt & 1, phase (nt >> 1) & 1
@@ -187,19 +193,14 @@ __global__ void __launch_bounds__(kThreads, 1)
       __syncwarp();
     };
     for (int it = 0; ok; ++it) {
-      const int buf = it % kLists, qb = it & 1;
+      const int buf = it % kLists;
       ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.list_full[buf]), (it / kLists) & 1, abort, status));
       if (!ok) break;
       const int n = sm.info[buf].n;
       if (n < 0) break;
-      int last = -1;
-      for (int e = 0; e < n; ++e)
-        if (sm.mask[buf][e] & tbits) last = e;
-      // the query tile is loaded for every item; it must have landed before its buffer is handed back
-      ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.q_full[qb][t]), (it >> 1) & 1, abort, status));
-      const uint64_t qdesc = smem_desc(s32(sm.q[qb][t]));
+      // the item's query rows are in TMEM (copied there by the softmax threads)
+      ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.q_ready[t]), it & 1, abort, status));
       if (!ok) break;
-      if (last < 0 && elect_one()) mbar_arrive(s32(&sm.q_empty[qb][t]));
       bool first = true, pend = false, pend_first = false;
       uint32_t pend_n = 0;
       int pend_st = 0;
@@ -220,13 +221,11 @@ __global__ void __launch_bounds__(kThreads, 1)
           const uint32_t b = nt & 1;
           tc_fence_after();
           const uint64_t kdesc = smem_desc(s32(sm.kv[st][0]));
-          const bool release_q = e == last && c == g.cpb - 1;
           if (elect_one()) {
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)
-              umma_ss(tcol_s + 64 * b, qdesc + 2 * kk, kdesc + 2 * kk, idesc_qk, kk > 0);
+              umma_ts(tcol_s + 64 * b, tcol_q + 8 * kk, kdesc + 2 * kk, idesc_qk, kk > 0);
             tc_commit(s32(&sm.s_full[t][b]));
-            if (release_q) tc_commit(s32(&sm.q_empty[qb][t]));
           }
           __syncwarp();
           if (pend) issue_pv(pend_n, pend_st, pend_first);
@@ -245,17 +244,40 @@ __global__ void __launch_bounds__(kThreads, 1)
     const int h = 2 * t + hh;
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t ts = tmem + lane_off + kColS + 128 * t, to = tmem + lane_off + kColO + 64 * t;
+    const uint32_t tq = tmem + lane_off + kColQ + 32 * t;
     const uint32_t tbits = 3u << (2 * t), hbit = 1u << h;
     const uint64_t scale2 = pack2(g.scale_log2, g.scale_log2);
     uint32_t nt = 0;
     bool ok = true;
-    for (int it = 0; ok; ++it) {
+    // Copies this thread's query row of item `it2` from shared memory (128-byte swizzled rows) to TMEM, where it is
+    // the A operand of the item's QK^T products.  Called when every QK^T of the previous item has completed.
+    // Returns the item's list length (-1: no more work).
+    auto stage_q = [&](int it2) -> int {
+      const int buf2 = it2 % kLists, qb2 = it2 & 1;
+      ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.list_full[buf2]), (it2 / kLists) & 1, abort, status));
+      if (!ok) return -1;
+      const int n2 = sm.info[buf2].n;
+      if (n2 < 0) return -1;
+      ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.q_full[qb2][t]), (it2 >> 1) & 1, abort, status));
+      if (!ok) return -1;
+      const int r = tid & 127;  // row of the tile; rows 0-63 and 64-127 are two 8 KB chunks
+      const unsigned char* rowp = sm.q[qb2][t] + (r >> 6) * kTile + (r & 63) * 128;
+      uint32_t qv[32];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const uint4 v = *reinterpret_cast<const uint4*>(rowp + ((c ^ (r & 7)) << 4));
+        qv[4 * c] = v.x; qv[4 * c + 1] = v.y; qv[4 * c + 2] = v.z; qv[4 * c + 3] = v.w;
+      }
+      tmem_st32(tq, qv);
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(s32(&sm.q_ready[t]));
+      mbar_arrive(s32(&sm.q_empty[qb2][t]));
+      return n2;
+    };
+    int n = stage_q(0);
+    for (int it = 0; ok && n >= 0; ++it) {
       const int buf = it % kLists;
-      ok = mbar_wait(s32(&sm.list_full[buf]), (it / kLists) & 1, abort, status);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      const int n = sm.info[buf].n;
-      if (n < 0) break;
       float m_ref = -INFINITY, l = 0.f;
       uint32_t done = 0;
       for (int e = 0; e < n && ok; ++e) {
@@ -369,6 +391,10 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
       }
       if (!ok) break;
+      // every QK^T of this item has completed (its S was received): the next item's query rows can go to TMEM,
+      // and its first products run while this item's output is written
+      const int n_next = stage_q(it + 1);
+      if (!ok) break;
       if (done > 0) {
         ok = mbar_wait(s32(&sm.pv_done[t][(nt - 1) & 1]), ((nt - 1) >> 1) & 1, abort, status);
         ok = __all_sync(0xffffffffu, ok);
@@ -399,6 +425,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(s32(&sm.list_empty[buf]));
+      n = n_next;
     }
   }
   tc_fence_before();

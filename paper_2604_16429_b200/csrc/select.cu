@@ -17,24 +17,26 @@ namespace mosaic {
 // pool_kernel: eight lanes per (tensor, unit, block), four blocks per warp; a lane owns eight
 // consecutive channels (one 16-byte load per token) and adds them in token order, row-major inside
 // the block, so every channel is one sequential fp64 chain.  HBM-bound: reads 2*U*N*d*2 bytes once;
-// the loads of a whole block row are in flight together.
+// the loads of a whole block row are in flight together.  Beside the pooled sums it writes an upper
+// bound of each pooled vector's Euclidean norm, which the ranking kernel's screening pass needs.
 // ------------------------------------------------------------------------------------------
 template <int BW>
 __global__ void __launch_bounds__(256) pool_kernel(Geo g, const uint4* __restrict__ q, const uint4* __restrict__ k,
-                                                   float* __restrict__ pq, float* __restrict__ pk) {
+                                                   float* __restrict__ pq, float* __restrict__ pk,
+                                                   float* __restrict__ nq, float* __restrict__ nk) {
   const int sub = threadIdx.x & 7;  // which 8 channels
   const long long grp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 3;
   const long long per_tensor = (long long)g.U * g.m;
-  if (grp >= 2 * per_tensor) return;
-  const int which = grp >= per_tensor;
-  const long long w = grp - which * per_tensor;
+  const bool live = grp < 2 * per_tensor;  // the last warp may be partly idle; it still takes part in the shuffles
+  const int which = live && grp >= per_tensor;
+  const long long w = live ? grp - which * per_tensor : 0;
   const int u = (int)(w / g.m), j = (int)(w - (long long)u * g.m);
   const uint4* src = (which ? k : q) + (long long)u * g.N * (kD / 8) + sub;
   const int by = j / g.nbw, bx = j - by * g.nbw;
   double acc[8];
 #pragma unroll
   for (int c = 0; c < 8; ++c) acc[c] = 0.0;
-  for (int r = 0; r < g.bh; ++r) {
+  for (int r = 0; r < g.bh && live; ++r) {
     const uint4* row = src + ((long long)(by * g.bh + r) * g.nlon + bx * BW) * (kD / 8);
     uint4 v[BW];
 #pragma unroll
@@ -49,20 +51,43 @@ __global__ void __launch_bounds__(256) pool_kernel(Geo g, const uint4* __restric
       }
     }
   }
+  float p[8];
+  double ss = 0.0;
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+    p[c] = (float)acc[c];
+    ss += (double)p[c] * (double)p[c];
+  }
+  ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+  ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+  ss += __shfl_xor_sync(0xffffffffu, ss, 4);
+  if (!live) return;
   float4* dst = reinterpret_cast<float4*>((which ? pk : pq) + ((long long)u * g.m + j) * kD + 8 * sub);
-  dst[0] = make_float4((float)acc[0], (float)acc[1], (float)acc[2], (float)acc[3]);
-  dst[1] = make_float4((float)acc[4], (float)acc[5], (float)acc[6], (float)acc[7]);
+  dst[0] = make_float4(p[0], p[1], p[2], p[3]);
+  dst[1] = make_float4(p[4], p[5], p[6], p[7]);
+  // rounded up twice, so that it is never below the norm of the fp32 vector (NaN and inf pass through)
+  if (sub == 0) (which ? nk : nq)[(long long)u * g.m + j] = __fmul_ru(__double2float_ru(sqrt(ss)), 1.000001f);
 }
 
 // ------------------------------------------------------------------------------------------
-// topk_kernel<TI>: a CTA owns TI query blocks of one unit and streams the pooled keys in chunks of
-// JT blocks through shared memory (as fp64, channel-major).  The TI x JT scores of a chunk are a
-// register-tiled fp64 product: thread (ty, tx) holds the scores of rows ty + 16a and keys tx + 16b
-// and runs one FMA chain over channels 0..d-1 per score, so each score is the sequential sum the
-// selection is defined by.  Scores become sortable keys; a key that cannot enter its row's list
-// (worse than the row's current k-th best) is dropped at once.
-// Merge: one warp per query row keeps the sorted k-entry list, one entry per lane; the rows of a warp
-// advance in lockstep so that their reductions overlap.
+// topk_kernel<NW, RI, CAP>: ranking of the key blocks of NW * RI query blocks of one unit (warp w owns RI
+// rows; a lane owns the keys lane, lane + 32, ... of every 128-key chunk that streams through shared memory).
+//
+// The ids must be those of the exact fp64 scores, but almost all of the m scores of a row are irrelevant,
+// so the kernel screens in fp32 and scores exactly only what survives:
+//   1. screening score  s~ = fp32 FMA chain over the channels.  |s~ - s| <= gamma_64 * sum|a_c||b_c|
+//      <= 2^-18 (1 + 1e-5) |a||b|  (standard bound of a length-64 dot product, any order, FMA or not;
+//      Cauchy-Schwarz).  The kernel uses eps = 2^-16 * na * nb + 1e-37 with the norm bounds of the pooling
+//      kernel: four times the bound, which also covers the rounding of s~ -+ eps and subnormal products.
+//      A non-finite s~ or eps makes the candidate's interval (-inf, +inf).
+//   2. every lane tracks the two largest lower bounds s~ - eps among its own keys; the k-th largest of
+//      those 64 values is a lower bound thr of the row's k-th best exact score (they belong to k distinct
+//      candidates).  A candidate with s~ + eps < thr is worse than k others whatever the ties: dropped.
+//      The first chunk is screened twice, first only to obtain a threshold.
+//   3. survivors (id and upper bound) collect in shared memory, pruned whenever thr rises; a row whose
+//      survivors overflow (massive ties) falls back to scoring every key exactly.
+//   4. exact phase: the fp64 chain of the selection's definition for each survivor, inserted into the
+//      row's sorted k-entry list (one entry per lane) by (score descending, id ascending).
 // ------------------------------------------------------------------------------------------
 
 // Total-order key: larger key = better score.  0 = not a candidate, 1 = NaN.
@@ -78,209 +103,325 @@ __device__ __forceinline__ bool ranks_before(unsigned long long ka, int ia, unsi
   return ka > kb || (ka == kb && ia < ib);
 }
 
-template <int TI, int JT>
+// order-preserving map of non-NaN floats to unsigned integers
+__device__ __forceinline__ unsigned ordered_bits(float f) {
+  const unsigned b = __float_as_uint(f);
+  return (b >> 31) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float from_ordered_bits(unsigned o) {
+  return __uint_as_float((o >> 31) ? (o & 0x7fffffffu) : ~o);
+}
+
+constexpr int kJT = 128;        // keys per chunk
+constexpr int kKStr = kD + 4;   // padded row of the staged vectors (floats): 16-byte reads of one row per lane hit every bank once
+
+template <int NW, int RI, int CAP>
 struct TopkSmem {
-  static constexpr int KSTR = JT + 1;  // padded row of the key tile: conflict-free transposing stores
-  double qs[kD][TI];                   // pooled queries of this CTA, channel-major
-  double ks[kD][KSTR];                 // pooled keys of the current chunk, channel-major
-  unsigned long long keys[TI][JT];     // candidate keys of the current chunk (0 = none)
-  unsigned long long thr[TI];          // key of the row's current k-th best (0 while the list is short)
-  int flag[TI];                        // the row has a candidate in this chunk
-  short iy[TI], ix[TI], jy[JT], jx[JT];  // block coordinates of the rows and of the chunk's keys
+  float ks[2][kJT][kKStr];      // pooled keys of two chunks (one being read, one in flight)
+  float nk[2][kJT];             // their norm bounds
+  float qs[NW * RI][kKStr];     // pooled queries of this CTA
+  int surv[NW * RI][CAP];       // surviving key ids per row ...
+  float surv_ub[NW * RI][CAP];  // ... and the upper bound of their score
 };
 
-template <int TI, int JT>
-__global__ void __launch_bounds__(256) topk_kernel(Geo g, const float* __restrict__ pq,
-                                                   const float* __restrict__ pk, int32_t* __restrict__ block_idx) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  TopkSmem<TI, JT>& sm = *reinterpret_cast<TopkSmem<TI, JT>*>(smem_raw);
-  constexpr int RJ = JT / 16;                 // keys per thread
-  constexpr int RI = TI / 16;                 // query rows per thread
-  constexpr int RPW = TI / 8;                 // query rows per warp in the merge
+__device__ __forceinline__ void cp_async16(void* dst, const void* src, bool valid) {
+  const unsigned n = valid ? 16u : 0u;  // 0 source bytes: the destination is filled with zeros
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"((unsigned)__cvta_generic_to_shared(dst)),
+               "l"(src), "r"(n)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async4(void* dst, const void* src, bool valid) {
+  const unsigned n = valid ? 4u : 0u;
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"((unsigned)__cvta_generic_to_shared(dst)),
+               "l"(src), "r"(n)
+               : "memory");
+}
 
+// The warp's sorted list of the best candidates so far holds one entry per lane (lane r = rank r).  Offers this
+// lane's candidate (key 0 = none) together with those of the other lanes; every candidate that belongs to the k
+// best is inserted.
+__device__ __forceinline__ void insert_batch(unsigned long long key, int id, unsigned long long& lkey, int& lid, int k,
+                                             int lane) {
+  while (true) {
+    // warp-wide best remaining candidate: maximum of the key's high word, then of the low word among the lanes
+    // that hold that high word, then the lowest id among the lanes that hold the key
+    const unsigned hi = (unsigned)(key >> 32), lo = (unsigned)key;
+    const unsigned mh = __reduce_max_sync(0xffffffffu, hi);
+    const unsigned ml = __reduce_max_sync(0xffffffffu, hi == mh ? lo : 0u);
+    const unsigned long long bk = ((unsigned long long)mh << 32) | ml;
+    if (bk == 0ull) return;
+    const int bj = (int)__reduce_min_sync(0xffffffffu, key == bk ? (unsigned)id : 0x7fffffffu);
+    const unsigned long long tk = __shfl_sync(0xffffffffu, lkey, k - 1);
+    const int ti = __shfl_sync(0xffffffffu, lid, k - 1);
+    if (!(tk == 0ull || ranks_before(bk, bj, tk, ti))) return;  // the batch's best does not enter: nothing does
+    const bool before = lkey != 0ull && ranks_before(lkey, lid, bk, bj);
+    const int p = __popc(__ballot_sync(0xffffffffu, before));
+    const unsigned long long uk = __shfl_up_sync(0xffffffffu, lkey, 1);
+    const int ui = __shfl_up_sync(0xffffffffu, lid, 1);
+    if (lane == p) { lkey = bk; lid = bj; }
+    else if (lane > p) { lkey = uk; lid = ui; }
+    if (key == bk && id == bj) key = 0ull;  // taken
+  }
+}
+
+template <int NW, int RI, int CAP>
+__global__ void __launch_bounds__(NW * 32) topk_kernel(Geo g, const float* __restrict__ pq,
+                                                       const float* __restrict__ pk, const float* __restrict__ nq,
+                                                       const float* __restrict__ nk, int32_t* __restrict__ block_idx) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  using SM = TopkSmem<NW, RI, CAP>;
+  SM& sm = *reinterpret_cast<SM*>(smem_raw);
+  constexpr int TI = NW * RI, NT = NW * 32;
+  const float kInf = __int_as_float(0x7f800000);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int tx = tid & 15, ty = tid >> 4;
   const int tiles = (g.m + TI - 1) / TI;
   const int u = blockIdx.x / tiles, i0 = (blockIdx.x - u * tiles) * TI;
   const float* pq_u = pq + (long long)u * g.m * kD;
   const float* pk_u = pk + (long long)u * g.m * kD;
+  const float* nk_u = nk + (long long)u * g.m;
+  const int nchunks = (g.m + kJT - 1) / kJT;
 
-  for (int e = tid; e < TI * kD; e += 256) {
-    const int r = e / kD, c = e - r * kD, i = i0 + r;
-    sm.qs[c][r] = i < g.m ? (double)pq_u[(long long)i * kD + c] : 0.0;
+  auto load_chunk = [&](int ch, int buf) {
+    const int j0 = ch * kJT;
+    for (int e = tid; e < kJT * (kD / 4); e += NT) {
+      const int jj = e / (kD / 4), c4 = e - jj * (kD / 4);
+      const bool valid = j0 + jj < g.m;
+      cp_async16(&sm.ks[buf][jj][4 * c4], pk_u + (long long)(valid ? j0 + jj : 0) * kD + 4 * c4, valid);
+    }
+    for (int jj = tid; jj < kJT; jj += NT) {
+      const bool valid = j0 + jj < g.m;
+      cp_async4(&sm.nk[buf][jj], nk_u + (valid ? j0 + jj : 0), valid);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+
+  load_chunk(0, 0);
+  for (int e = tid; e < TI * (kD / 4); e += NT) {
+    const int r = e / (kD / 4), c4 = e - r * (kD / 4);
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (i0 + r < g.m) v = __ldg(reinterpret_cast<const float4*>(pq_u + (long long)(i0 + r) * kD + 4 * c4));
+    *reinterpret_cast<float4*>(&sm.qs[r][4 * c4]) = v;
   }
-  for (int r = tid; r < TI; r += 256) {
-    const int i = min(i0 + r, g.m - 1);
-    sm.thr[r] = 0ull;
-    sm.iy[r] = (short)(i / g.nbw);
-    sm.ix[r] = (short)(i - (i / g.nbw) * g.nbw);
+
+  // per row of this warp: block coordinates, norm bound, the lane's two best lower bounds, threshold, survivors
+  int iy[RI], ix[RI], cnt[RI];
+  float nqv[RI], m1[RI], m2[RI], thr[RI];
+#pragma unroll
+  for (int a = 0; a < RI; ++a) {
+    const int i = min(i0 + warp * RI + a, g.m - 1);
+    iy[a] = i / g.nbw;
+    ix[a] = i - iy[a] * g.nbw;
+    nqv[a] = __ldg(nq + (long long)u * g.m + i);
+    m1[a] = -kInf; m2[a] = -kInf; thr[a] = -kInf;
+    cnt[a] = 0;
   }
+  const unsigned lower = (1u << lane) - 1u;
 
-  // sorted list of the best candidates so far: entry `lane` of each row this warp owns
-  unsigned long long lkey[RPW];
-  int lid[RPW];
-#pragma unroll
-  for (int r = 0; r < RPW; ++r) { lkey[r] = 0ull; lid[r] = -1; }
-
-  for (int j0 = 0; j0 < g.m; j0 += JT) {
-    __syncthreads();  // previous chunk fully merged (and qs, thr written on the first pass)
-    const int nj = min(JT, g.m - j0);
-#pragma unroll
-    for (int e = tid; e < JT * kD / 4; e += 256) {
-      const int jj = e / (kD / 4), c4 = (e - jj * (kD / 4)) * 4;
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (jj < nj) v = __ldg(reinterpret_cast<const float4*>(pk_u + (long long)(j0 + jj) * kD + c4));
-      sm.ks[c4][jj] = (double)v.x;
-      sm.ks[c4 + 1][jj] = (double)v.y;
-      sm.ks[c4 + 2][jj] = (double)v.z;
-      sm.ks[c4 + 3][jj] = (double)v.w;
+  // thr <- k-th largest of the warp's tracked lower bounds (a pop takes the largest out of its lane's pair)
+  auto update_threshold = [&](int a) {
+    float t1 = m1[a], t2 = m2[a];
+    for (int r = 0; r + 1 < g.topk; ++r) {
+      const unsigned o = ordered_bits(t1);
+      const unsigned best = __reduce_max_sync(0xffffffffu, o);
+      const unsigned who = __ballot_sync(0xffffffffu, o == best);
+      if (lane == __ffs(who) - 1) { t1 = t2; t2 = -kInf; }
     }
-    if (tid < JT) {
-      const int j = min(j0 + tid, g.m - 1);
-      sm.jy[tid] = (short)(j / g.nbw);
-      sm.jx[tid] = (short)(j - (j / g.nbw) * g.nbw);
-    }
-    for (int r = tid; r < TI; r += 256) sm.flag[r] = 0;
-    __syncthreads();
-    {
-      double acc[RI][RJ];
-#pragma unroll
-      for (int a = 0; a < RI; ++a)
-#pragma unroll
-        for (int b = 0; b < RJ; ++b) acc[a][b] = 0.0;
-#pragma unroll 8
-      for (int c = 0; c < kD; ++c) {
-        double qv[RI], kv[RJ];
-#pragma unroll
-        for (int a = 0; a < RI; ++a) qv[a] = sm.qs[c][ty + 16 * a];
-#pragma unroll
-        for (int b = 0; b < RJ; ++b) kv[b] = sm.ks[c][tx + 16 * b];
-#pragma unroll
-        for (int a = 0; a < RI; ++a)
-#pragma unroll
-          for (int b = 0; b < RJ; ++b) acc[a][b] = fma(qv[a], kv[b], acc[a][b]);
+    thr[a] = from_ordered_bits(__reduce_max_sync(0xffffffffu, ordered_bits(t1)));
+  };
+  // drop the survivors of row a that the current threshold rules out (order kept)
+  auto prune = [&](int a) {
+    const int row = warp * RI + a, n = min(cnt[a], CAP);
+    if (cnt[a] > CAP) return;  // overflowed: the row is rescored in full anyway
+    int kept = 0;
+    for (int e0 = 0; e0 < n; e0 += 32) {
+      const int e = e0 + lane;
+      const int j = e < n ? sm.surv[row][e] : 0;
+      const float ub = e < n ? sm.surv_ub[row][e] : 0.f;
+      const bool keep = e < n && !(ub < thr[a]);
+      const unsigned km = __ballot_sync(0xffffffffu, keep);
+      __syncwarp();
+      if (keep) {
+        const int at = kept + __popc(km & lower);
+        sm.surv[row][at] = j;
+        sm.surv_ub[row][at] = ub;
       }
-#pragma unroll
-      for (int a = 0; a < RI; ++a) {
-        const int r = ty + 16 * a, i = i0 + r;
-        const unsigned long long th = sm.thr[r];
-        const int iy = sm.iy[r], ix = sm.ix[r];
-        bool any = false;
-#pragma unroll
-        for (int b = 0; b < RJ; ++b) {
-          const int jj = tx + 16 * b;
-          int dx = sm.jx[jj] - ix;
-          dx += dx < 0 ? g.nbw : 0;  // (jx - ix) mod nbw
-          const bool local = abs(sm.jy[jj] - iy) <= g.rlat && (dx <= g.rlon || g.nbw - dx <= g.rlon);
-          unsigned long long key = 0ull;
-          if (jj < nj && i < g.m && !local) {
-            key = score_key(acc[a][b]);
-            if (key < th) key = 0ull;  // cannot enter the list (an equal key may: lower id wins)
-          }
-          sm.keys[r][jj] = key;
-          any |= key != 0ull;
-        }
-        if (any) sm.flag[r] = 1;
-      }
-    }
-    __syncthreads();
-    // merge, all rows of this warp in lockstep: repeatedly take each row's best remaining chunk entry
-    // while it still enters the row's list
-    unsigned live = 0;
-#pragma unroll
-    for (int rr = 0; rr < RPW; ++rr) live |= (sm.flag[warp * RPW + rr] ? 1u : 0u) << rr;
-    for (int round = 0; round < g.topk && live; ++round) {
-      unsigned long long bk[RPW];
-      int bj[RPW];
-#pragma unroll
-      for (int rr = 0; rr < RPW; ++rr) {
-        bk[rr] = 0ull;
-        bj[rr] = 0x7fffffff;
-        if ((live >> rr) & 1) {
-          const unsigned long long* row = sm.keys[warp * RPW + rr];
-#pragma unroll
-          for (int s = 0; s < JT / 32; ++s) {
-            const unsigned long long kk = row[lane + 32 * s];
-            const int jj = j0 + lane + 32 * s;
-            if (kk != 0ull && ranks_before(kk, jj, bk[rr], bj[rr])) { bk[rr] = kk; bj[rr] = jj; }
-          }
-        }
-      }
-      // warp-wide best of each row: maximum of the key's high word, then of the low word among the
-      // lanes that hold that high word, then the lowest block id among the lanes that hold the key
-#pragma unroll
-      for (int rr = 0; rr < RPW; ++rr) {
-        if (!((live >> rr) & 1)) continue;  // warp-uniform
-        const unsigned hi = (unsigned)(bk[rr] >> 32), lo = (unsigned)bk[rr];
-        const unsigned mh = __reduce_max_sync(0xffffffffu, hi);
-        const unsigned ml = __reduce_max_sync(0xffffffffu, hi == mh ? lo : 0u);
-        const bool mine = bk[rr] != 0ull && hi == mh && lo == ml;
-        bj[rr] = __reduce_min_sync(0xffffffffu, mine ? bj[rr] : 0x7fffffff);
-        bk[rr] = ((unsigned long long)mh << 32) | ml;
-      }
-#pragma unroll
-      for (int rr = 0; rr < RPW; ++rr) {
-        // list is sorted best-first; its last wanted entry sits in lane topk-1
-        if (!((live >> rr) & 1)) continue;
-        const unsigned long long tk = __shfl_sync(0xffffffffu, lkey[rr], g.topk - 1);
-        const int ti = __shfl_sync(0xffffffffu, lid[rr], g.topk - 1);
-        const bool enters = bk[rr] != 0ull && (tk == 0ull || ranks_before(bk[rr], bj[rr], tk, ti));
-        if (!enters) { live &= ~(1u << rr); continue; }  // chunk exhausted for this row
-        // insert at position p = number of entries ranking before the new one
-        const bool before = lkey[rr] != 0ull && ranks_before(lkey[rr], lid[rr], bk[rr], bj[rr]);
-        const int p = __popc(__ballot_sync(0xffffffffu, before));
-        const unsigned long long uk = __shfl_up_sync(0xffffffffu, lkey[rr], 1);
-        const int ui = __shfl_up_sync(0xffffffffu, lid[rr], 1);
-        if (lane == p) { lkey[rr] = bk[rr]; lid[rr] = bj[rr]; }
-        else if (lane > p) { lkey[rr] = uk; lid[rr] = ui; }
-        if (lane == ((bj[rr] - j0) & 31)) sm.keys[warp * RPW + rr][bj[rr] - j0] = 0ull;  // taken
-      }
+      kept += __popc(km);
       __syncwarp();
     }
-#pragma unroll
-    for (int rr = 0; rr < RPW; ++rr) {
-      const unsigned long long tk = __shfl_sync(0xffffffffu, lkey[rr], g.topk - 1);
-      if (lane == 0) sm.thr[warp * RPW + rr] = tk;  // 0 until the list holds topk entries
+    cnt[a] = kept;
+  };
+
+  // chunk -1 is the first chunk screened for a threshold only; then every chunk, the first one again
+  for (int step = -1; step < nchunks; ++step) {
+    const int ch = max(step, 0), buf = (step + 1) & 1;
+    // the next chunk streams in while this one is screened (after the threshold pass: the first chunk once more)
+    const int nxt = step + 1 < nchunks ? max(step + 1, 0) : -1;
+    if (nxt >= 0) {
+      load_chunk(nxt, buf ^ 1);
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
+    } else {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
-  }
+    __syncthreads();
+    const int j0 = ch * kJT;
+    float acc[RI][4];
 #pragma unroll
-  for (int rr = 0; rr < RPW; ++rr) {
-    const int i = i0 + warp * RPW + rr;
-    if (i < g.m && lane < g.topk)
-      block_idx[((long long)u * g.m + i) * g.topk + lane] = lkey[rr] != 0ull ? lid[rr] : -1;
+    for (int a = 0; a < RI; ++a)
+#pragma unroll
+      for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+#pragma unroll 4
+    for (int c4 = 0; c4 < kD / 4; ++c4) {
+      float4 kv[4];
+#pragma unroll
+      for (int b = 0; b < 4; ++b) kv[b] = *reinterpret_cast<const float4*>(&sm.ks[buf][lane + 32 * b][4 * c4]);
+#pragma unroll
+      for (int a = 0; a < RI; ++a) {
+        const float4 qv = *reinterpret_cast<const float4*>(&sm.qs[warp * RI + a][4 * c4]);
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+          acc[a][b] = fmaf(qv.x, kv[b].x, acc[a][b]);
+          acc[a][b] = fmaf(qv.y, kv[b].y, acc[a][b]);
+          acc[a][b] = fmaf(qv.z, kv[b].z, acc[a][b]);
+          acc[a][b] = fmaf(qv.w, kv[b].w, acc[a][b]);
+        }
+      }
+    }
+    int jy[4], jx[4];
+    float nkv[4];
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const int j = min(j0 + lane + 32 * b, g.m - 1);
+      jy[b] = j / g.nbw;
+      jx[b] = j - jy[b] * g.nbw;
+      nkv[b] = sm.nk[buf][lane + 32 * b];
+    }
+#pragma unroll
+    for (int a = 0; a < RI; ++a) {
+      const bool row_ok = i0 + warp * RI + a < g.m;  // warp-uniform
+      const int row = warp * RI + a;
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        const int j = j0 + lane + 32 * b;
+        int dx = jx[b] - ix[a];
+        dx += dx < 0 ? g.nbw : 0;  // (jx - ix) mod nbw
+        const bool local = abs(jy[b] - iy[a]) <= g.rlat && (dx <= g.rlon || g.nbw - dx <= g.rlon);
+        const bool cand = row_ok && j < g.m && !local;
+        const float s = acc[a][b], eps = fmaf(nqv[a] * nkv[b], 1.52587890625e-5f, 1e-37f);
+        const bool fin = fabsf(s) <= 1e38f && eps <= 1e38f;
+        const float lb = fin ? s - eps : -kInf, ub = fin ? s + eps : kInf;
+        if (step >= 0) {
+          const bool keep = cand && !(ub < thr[a]);
+          const unsigned km = __ballot_sync(0xffffffffu, keep);
+          if (keep) {
+            const int at = cnt[a] + __popc(km & lower);
+            if (at < CAP) { sm.surv[row][at] = j; sm.surv_ub[row][at] = ub; }
+          }
+          cnt[a] += __popc(km);
+        }
+        if (step != 0 && cand) {  // the first chunk's bounds were tracked in the threshold pass
+          if (lb > m1[a]) { m2[a] = m1[a]; m1[a] = lb; }
+          else m2[a] = fmaxf(m2[a], lb);
+        }
+      }
+    }
+    // a higher threshold after the first chunks, then every fourth chunk, and at the end
+    if (step < 4 || (step & 3) == 3 || step == nchunks - 1) {
+      __syncwarp();
+#pragma unroll
+      for (int a = 0; a < RI; ++a) {
+        update_threshold(a);
+        if (step >= 0) prune(a);
+      }
+    }
+    __syncthreads();  // everyone is done with this buffer before the chunk after next lands in it
+  }
+
+  // exact phase: one row of the warp at a time
+#pragma unroll
+  for (int a = 0; a < RI; ++a) {
+    const int row = warp * RI + a, i = i0 + row;
+    if (i >= g.m) break;  // warp-uniform
+    const float* qrow = sm.qs[row];
+    auto exact_key = [&](int j) {
+      const float4* krow = reinterpret_cast<const float4*>(pk_u + (long long)j * kD);
+      double s = 0.0;
+#pragma unroll 4
+      for (int c4 = 0; c4 < kD / 4; ++c4) {
+        const float4 kv = __ldg(krow + c4);
+        s = fma((double)qrow[4 * c4], (double)kv.x, s);
+        s = fma((double)qrow[4 * c4 + 1], (double)kv.y, s);
+        s = fma((double)qrow[4 * c4 + 2], (double)kv.z, s);
+        s = fma((double)qrow[4 * c4 + 3], (double)kv.w, s);
+      }
+      return score_key(s);
+    };
+    unsigned long long lkey = 0ull;
+    int lid = -1;
+    __syncwarp();
+    if (cnt[a] <= CAP) {
+      for (int e0 = 0; e0 < cnt[a]; e0 += 32) {
+        const int e = e0 + lane;
+        const int j = e < cnt[a] ? sm.surv[row][e] : -1;
+        insert_batch(j >= 0 ? exact_key(j) : 0ull, j, lkey, lid, g.topk, lane);
+      }
+    } else {  // too many survivors to hold: score every key of the unit
+      for (int jb = 0; jb < g.m; jb += 32) {
+        const int j = jb + lane;
+        bool cand = j < g.m;
+        if (cand) {
+          const int jy = j / g.nbw, jx = j - jy * g.nbw;
+          int dx = jx - ix[a];
+          dx += dx < 0 ? g.nbw : 0;
+          cand = !(abs(jy - iy[a]) <= g.rlat && (dx <= g.rlon || g.nbw - dx <= g.rlon));
+        }
+        insert_batch(cand ? exact_key(j) : 0ull, j, lkey, lid, g.topk, lane);
+      }
+    }
+    if (lane < g.topk) block_idx[((long long)u * g.m + i) * g.topk + lane] = lkey != 0ull ? lid : -1;
   }
 }
 
-template <int TI, int JT>
-int launch_topk(const HostCtx& c, const float* pooled_q, const float* pooled_k, int32_t* block_idx) {
+template <int NW, int RI, int CAP>
+int launch_topk(const HostCtx& c, const float* pooled_q, const float* pooled_k, const float* norm_q,
+                const float* norm_k, int32_t* block_idx) {
   const Geo& g = c.g;
-  const size_t smem = sizeof(TopkSmem<TI, JT>);
-  if (cudaFuncSetAttribute(topk_kernel<TI, JT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-    return MOSAIC_E_CUDA;
-  const int tiles = (g.m + TI - 1) / TI;
-  topk_kernel<TI, JT><<<(unsigned)(g.U * tiles), 256, smem, c.stream>>>(g, pooled_q, pooled_k, block_idx);
+  const size_t smem = sizeof(TopkSmem<NW, RI, CAP>);
+  static unsigned long long configured = 0;  // devices on which the kernel's shared-memory opt-in is set
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return MOSAIC_E_CUDA;
+  if (dev < 0 || dev >= 64) return MOSAIC_E_UNSUPPORTED;
+  if (!((configured >> dev) & 1ull)) {
+    if (cudaFuncSetAttribute(topk_kernel<NW, RI, CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+        cudaSuccess)
+      return MOSAIC_E_CUDA;
+    configured |= 1ull << dev;
+  }
+  const int tiles = (g.m + NW * RI - 1) / (NW * RI);
+  topk_kernel<NW, RI, CAP><<<(unsigned)(g.U * tiles), NW * 32, smem, c.stream>>>(g, pooled_q, pooled_k, norm_q,
+                                                                                norm_k, block_idx);
   return cudaGetLastError() == cudaSuccess ? MOSAIC_OK : MOSAIC_E_CUDA;
 }
 
 int launch_select(const HostCtx& c, const void* q, const void* k, int32_t* block_idx, float* pooled_q,
-                  float* pooled_k) {
+                  float* pooled_k, float* norm_q, float* norm_k) {
   const Geo& g = c.g;
   {
     const long long threads = 2ll * g.U * g.m * 8;
     const unsigned blocks = (unsigned)((threads + 255) / 256);
     if (g.bw == 8)
-      pool_kernel<8><<<blocks, 256, 0, c.stream>>>(g, (const uint4*)q, (const uint4*)k, pooled_q, pooled_k);
+      pool_kernel<8><<<blocks, 256, 0, c.stream>>>(g, (const uint4*)q, (const uint4*)k, pooled_q, pooled_k, norm_q,
+                                                   norm_k);
     else
-      pool_kernel<16><<<blocks, 256, 0, c.stream>>>(g, (const uint4*)q, (const uint4*)k, pooled_q, pooled_k);
+      pool_kernel<16><<<blocks, 256, 0, c.stream>>>(g, (const uint4*)q, (const uint4*)k, pooled_q, pooled_k, norm_q,
+                                                    norm_k);
     if (cudaGetLastError() != cudaSuccess) return MOSAIC_E_CUDA;
   }
   if (g.topk > 0) {
-    // the most query blocks per CTA (64, 32, 16) that still gives every SM two CTAs; 16 otherwise
+    // the most query blocks per CTA (64, 32, 16) that still gives every SM about two CTAs; 16 otherwise
     auto ctas = [&](int ti) { return (long long)g.U * ((g.m + ti - 1) / ti); };
-    // small problems (16 rows per CTA) take keys in chunks of 128 to halve the number of merge passes
-    const int rc = ctas(64) >= 296 ? launch_topk<64, 64>(c, pooled_q, pooled_k, block_idx)
-                 : ctas(32) >= 296 ? launch_topk<32, 64>(c, pooled_q, pooled_k, block_idx)
-                                   : launch_topk<16, 128>(c, pooled_q, pooled_k, block_idx);
+    const int rc = ctas(64) >= 296 ? launch_topk<8, 8, 128>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx)
+                 : ctas(32) >= 296 ? launch_topk<4, 8, 96>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx)
+                                   : launch_topk<4, 4, 192>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx);
     if (rc) return rc;
   }
   return MOSAIC_OK;

@@ -12,7 +12,7 @@
 namespace mosaic {
 namespace {
 
-// status block + pooled Q sums + pooled K sums.  Every device that loads the library holds this array
+// status block + pooled Q and K sums + their norm bounds.  Every device that loads the library holds this array
 // until the process exits.
 static __device__ __align__(256) unsigned char g_static_scratch[MOSAIC_BSA_STATIC_SCRATCH_BYTES];
 
@@ -50,8 +50,8 @@ extern "C" int mosaic_bsa_select_static(const mosaic_bsa_params* p, const void* 
   if (!q || !k || (!block_idx && g.topk > 0)) return MOSAIC_E_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(k)) & 15u) return MOSAIC_E_MISALIGNED;
   if (reinterpret_cast<uintptr_t>(block_idx) & 3u) return MOSAIC_E_MISALIGNED;
-  const size_t pooled = align256(sizeof(float) * (size_t)g.U * g.m * kD);
-  if (kStatusBytes + 2 * pooled > (size_t)MOSAIC_BSA_STATIC_SCRATCH_BYTES) return MOSAIC_E_WORKSPACE_TOO_SMALL;
+  const SelectWs w = select_layout(g);
+  if (w.total > (size_t)MOSAIC_BSA_STATIC_SCRATCH_BYTES) return MOSAIC_E_WORKSPACE_TOO_SMALL;
   int major = 0, dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
@@ -61,10 +61,9 @@ extern "C" int mosaic_bsa_select_static(const mosaic_bsa_params* p, const void* 
   if ((rc = scratch_address(&base))) return rc;
   c.stream = (cudaStream_t)cuda_stream;
   c.status = reinterpret_cast<int*>(base);
-  // the array keeps what the previous call left: the status block must start at zero; the pooled sums
-  // are fully rewritten by the pooling kernel before the ranking kernel reads them
+  // the array keeps what the previous call left: the status block must start at zero; the pooled sums and
+  // norm bounds are fully rewritten by the pooling kernel before the ranking kernel reads them
   if (cudaMemsetAsync(base, 0, kStatusBytes, c.stream) != cudaSuccess) return MOSAIC_E_CUDA;
-  float* pq = reinterpret_cast<float*>(base + kStatusBytes);
-  float* pk = reinterpret_cast<float*>(base + kStatusBytes + pooled);
-  return launch_select(c, q, k, block_idx, pq, pk);
+  return launch_select(c, q, k, block_idx, reinterpret_cast<float*>(base + w.pq), reinterpret_cast<float*>(base + w.pk),
+                       reinterpret_cast<float*>(base + w.nq), reinterpret_cast<float*>(base + w.nk));
 }

@@ -11,24 +11,16 @@ from paper_2604_16429_b200 import binding as mb
 from paper_2604_16429_b200 import synth
 
 FWD_MAX_ABS, FWD_MEAN_ABS = 2e-2, 2e-3      # forward tolerances (bf16 inputs, fp64 oracle)
-BWD_MAX_ABS = 5e-2                          # backward tolerance for gradients of ordinary magnitude
-BWD_REL = 2.0 ** -7                         # ... plus this much of |reference|: gradients are stored as bf16
+BWD_MAX_ABS = 5e-2                          # backward tolerance (max-abs, every element)
 LSE_ABS = 2e-3                              # fp32 log-sum-exp of fp32-accumulated logits
 GUARD = 4096                                # bytes of canary before and after every output and workspace
-
-
-def bwd_tol(ref: np.ndarray) -> np.ndarray:
-    """Element-wise backward bound: 5e-2, widened for large gradients because the result is rounded to
-    bf16 (half an ulp is up to 2^-8 of the value) after summing bf16-rounded P and dS terms."""
-    return BWD_MAX_ABS + BWD_REL * np.abs(ref)
 
 
 def assert_bwd_close(name, got, ref):
     gh = got.float().cpu().numpy().astype(np.float64) if torch.is_tensor(got) else np.asarray(got, np.float64)
     assert np.isfinite(gh).all(), f"{name}: unwritten or non-finite gradient"
     err = np.abs(gh - ref)
-    bad = err > bwd_tol(ref)
-    assert not bad.any(), f"{name}: {int(bad.sum())} elements beyond the bound, max-abs {err.max():.4g} at |ref| {np.abs(ref)[np.unravel_index(err.argmax(), err.shape)]:.4g}"
+    assert err.max() <= BWD_MAX_ABS, f"{name}: max-abs {err.max():.4g} at |ref| {np.abs(ref)[np.unravel_index(err.argmax(), err.shape)]:.4g}"
     return float(err.max())
 
 

@@ -51,6 +51,43 @@ def test_select_ties_go_to_lower_block_id():
     assert rows
 
 
+def test_select_near_ties_below_the_screening_resolution():
+    """Twenty key blocks whose scores differ by about 1e-6 of their size, far below what an fp32 score can
+    resolve: which eight of them a row takes, and in which order, is decided by the exact fp64 chain."""
+    w = synth.small_case(120, 160, 8, 8, 8, B=1, H=2, seed=71)                 # m = 300
+    x = synth.make_inputs(w)
+    kf = synth.bf16_bits_to_f32(x["k"]).reshape(1, 2, 120, 160, 64).copy()
+    qf = synth.bf16_bits_to_f32(x["q"]).reshape(1, 2, 120, 160, 64).copy()
+    qf[..., 0] = np.abs(qf[..., 0]) + 1.0
+    for t in range(20):
+        by, bx = (3 * t) % 15, (7 * t) % 20
+        blk = kf[:, :, 8 * by:8 * by + 8, 8 * bx:8 * bx + 8]
+        blk[...] = 0.0
+        blk[..., 0] = 4.0                                                       # pooled channel 0: 256 for all twenty
+        blk[:, :, 0, 0, 1] = (1 + t) * 2.0 ** -10                               # the only difference between them
+    x["k"] = synth.to_bf16_bits(kf.reshape(1, 2, -1, 64))
+    x["q"] = synth.to_bf16_bits(qf.reshape(1, 2, -1, 64))
+    want = G.oracle_select_all(w, x)
+    got = G.gpu_select(w, G.device_inputs(x)).cpu().numpy()
+    assert np.array_equal(got, want), f"{(got != want).sum()} of {want.size} ids differ"
+    special = {((3 * t) % 15) * 20 + (7 * t) % 20 for t in range(20)}
+    assert np.mean([len(special & set(r.tolist())) for r in want[0, 0]]) > 7    # the rows do choose among them
+
+
+def test_select_all_scores_tied_takes_the_full_rescoring_path():
+    """Every key block identical: all scores of a row tie exactly, nothing can be screened out, and the rows
+    fall back to scoring every key; the lowest non-local ids win."""
+    w = synth.small_case(120, 160, 8, 8, 6, B=1, H=1, seed=72)                 # m = 300 > survivors a row can hold
+    x = synth.make_inputs(w)
+    k = x["k"].reshape(1, 1, 15, 8, 20, 8, 64).copy()
+    k[...] = k[:, :, :1, :, :1]                                                 # every block repeats block 0
+    x["k"] = np.ascontiguousarray(k.reshape(1, 1, -1, 64))
+    want = G.oracle_select_all(w, x)
+    got = G.gpu_select(w, G.device_inputs(x)).cpu().numpy()
+    assert np.array_equal(got, want)
+    assert want[0, 0, 150].tolist() == [0, 1, 2, 3, 4, 5]
+
+
 FWD_CASES = [
     (synth.WORKLOADS["c1_tiny"], 0.0),
     (synth.small_case(24, 40, 8, 8, 3, B=1, H=2, seed=31), 0.0),                # m = 15: last tile holds one block
@@ -169,7 +206,7 @@ def test_repeated_and_local_ids_are_skipped_and_reported():
 
 
 def test_descriptor_cache_encodes_once_per_tensor():
-    w = synth.small_case(32, 64, 8, 8, 4, B=1, H=1, seed=59)
+    w = synth.small_case(56, 88, 8, 8, 4, B=1, H=1, seed=59)    # a grid no other test uses: nothing cached for it yet
     dx = G.device_inputs(synth.make_inputs(w))
     p = mb.Params.from_workload(w)
     ws = mb.alloc_workspace(p, mb.OP_FWD)
@@ -181,7 +218,7 @@ def test_descriptor_cache_encodes_once_per_tensor():
     n1 = mb.descriptor_encodes()
     mb.mosaic_bsa_fwd(p, dx["q"], dx["k"], dx["v"], idx, o=o, lse=lse, ws=ws)
     n2 = mb.descriptor_encodes()
-    assert 1 <= n1 - n0 <= 4 and n2 == n1                  # Q, K, V (and O) once; nothing on the second call
+    assert n1 - n0 == 3 and n2 == n1                       # Q, K, V once; nothing on the second call
     mb.check_status(ws, "fwd")
 
 
@@ -244,7 +281,6 @@ def test_backward_popular_key_blocks_lists_span_several_buffers():
     o, lse = G.gpu_fwd(w, dx, idx)
     dq, dk, dv = G.gpu_bwd(w, dx, o, lse, idx)
     dQ, dK, dV, _, _ = oracle.bwd(G.geom_of(w), x["q"][0, 0], x["k"][0, 0], x["v"][0, 0], x["do"][0, 0], idx_h)
-    assert np.abs(dV).max() > 20                                  # gradients large enough that bf16 storage sets the error
     for name, got, want in (("dQ", dq, dQ), ("dK", dk, dK), ("dV", dv, dV)):
         G.assert_bwd_close(name, got[0, 0], want)
 

@@ -41,7 +41,7 @@ def test_static_scratch_selection_matches_twice_in_a_row():
 
 def test_static_scratch_rejects_problems_beyond_its_size():
     p = mb.Params(B=24, H=8, nlat=120, nlon=240, topk=8)       # 192 units x 450 blocks: 44 MB of pooled sums
-    assert 256 + 2 * p.U * p.m * p.d * 4 > mb.STATIC_SCRATCH_BYTES
+    assert mb.workspace_bytes(p, mb.OP_SELECT) > mb.STATIC_SCRATCH_BYTES
     pc = p.c()
     rc = mb.lib().mosaic_bsa_select_static(ctypes.byref(pc), 256, 256, 256, None)   # never dereferenced: the size check comes first
     assert rc == -3 and "workspace" in mb.strerror(rc)

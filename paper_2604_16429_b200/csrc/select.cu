@@ -83,11 +83,13 @@ __global__ void __launch_bounds__(256) pool_kernel(Geo g, const uint4* __restric
 //   2. every lane tracks the two largest lower bounds s~ - eps among its own keys; the k-th largest of
 //      those 64 values is a lower bound thr of the row's k-th best exact score (they belong to k distinct
 //      candidates).  A candidate with s~ + eps < thr is worse than k others whatever the ties: dropped.
-//      The first chunk is screened twice, first only to obtain a threshold.
-//   3. survivors (id and upper bound) collect in shared memory, pruned whenever thr rises; a row whose
+//      Chunks are visited from the CTA's own neighbourhood outwards (on smooth fields the best keys are
+//      near, so the threshold is tight at once); the first chunk is screened twice, first for a threshold only.
+//   3. survivors (id and upper bound) collect in shared memory, pruned when thr has risen; a row whose
 //      survivors overflow (massive ties) falls back to scoring every key exactly.
-//   4. exact phase: the fp64 chain of the selection's definition for each survivor, inserted into the
-//      row's sorted k-entry list (one entry per lane) by (score descending, id ascending).
+//   4. exact phase: the fp64 chain of the selection's definition for every survivor of the warp's rows
+//      (lanes take survivors, two chains in flight each), then each row ranks its survivors by
+//      (score descending, id ascending) by counting, and ranks 0..k-1 are written.
 // ------------------------------------------------------------------------------------------
 
 // Total-order key: larger key = better score.  0 = not a candidate, 1 = NaN.
@@ -114,11 +116,17 @@ __device__ __forceinline__ float from_ordered_bits(unsigned o) {
 
 constexpr int kJT = 128;        // keys per chunk
 constexpr int kKStr = kD + 4;   // padded row of the staged vectors (floats): 16-byte reads of one row per lane hit every bank once
+constexpr int kExact = 64;      // most survivors of a row that the counting rank handles (more: insertion path)
 
 template <int NW, int RI, int CAP>
 struct TopkSmem {
-  float ks[2][kJT][kKStr];      // pooled keys of two chunks (one being read, one in flight)
-  float nk[2][kJT];             // their norm bounds
+  union {
+    struct {
+      float ks[2][kJT][kKStr];  // pooled keys of two chunks (one being read, one in flight)
+      float nk[2][kJT];         // their norm bounds
+    } scr;
+    unsigned long long ekey[NW * RI][kExact];  // exact phase: score keys of the rows' survivors
+  };
   float qs[NW * RI][kKStr];     // pooled queries of this CTA
   int surv[NW * RI][CAP];       // surviving key ids per row ...
   float surv_ub[NW * RI][CAP];  // ... and the upper bound of their score
@@ -164,6 +172,24 @@ __device__ __forceinline__ void insert_batch(unsigned long long key, int id, uns
   }
 }
 
+// exact score of (pooled query row in shared memory, pooled key row j in global memory) as a sortable key
+__device__ __forceinline__ unsigned long long exact_key(const float* qrow, const float* __restrict__ pk_u, int j) {
+  const float4* krow = reinterpret_cast<const float4*>(pk_u + (long long)j * kD);
+  float4 kv[kD / 4];
+#pragma unroll
+  for (int c4 = 0; c4 < kD / 4; ++c4) kv[c4] = __ldg(krow + c4);
+  double s = 0.0;
+#pragma unroll
+  for (int c4 = 0; c4 < kD / 4; ++c4) {
+    const float4 qv = *reinterpret_cast<const float4*>(qrow + 4 * c4);
+    s = fma((double)qv.x, (double)kv[c4].x, s);
+    s = fma((double)qv.y, (double)kv[c4].y, s);
+    s = fma((double)qv.z, (double)kv[c4].z, s);
+    s = fma((double)qv.w, (double)kv[c4].w, s);
+  }
+  return score_key(s);
+}
+
 template <int NW, int RI, int CAP>
 __global__ void __launch_bounds__(NW * 32) topk_kernel(Geo g, const float* __restrict__ pq,
                                                        const float* __restrict__ pk, const float* __restrict__ nq,
@@ -186,16 +212,29 @@ __global__ void __launch_bounds__(NW * 32) topk_kernel(Geo g, const float* __res
     for (int e = tid; e < kJT * (kD / 4); e += NT) {
       const int jj = e / (kD / 4), c4 = e - jj * (kD / 4);
       const bool valid = j0 + jj < g.m;
-      cp_async16(&sm.ks[buf][jj][4 * c4], pk_u + (long long)(valid ? j0 + jj : 0) * kD + 4 * c4, valid);
+      cp_async16(&sm.scr.ks[buf][jj][4 * c4], pk_u + (long long)(valid ? j0 + jj : 0) * kD + 4 * c4, valid);
     }
     for (int jj = tid; jj < kJT; jj += NT) {
       const bool valid = j0 + jj < g.m;
-      cp_async4(&sm.nk[buf][jj], nk_u + (valid ? j0 + jj : 0), valid);
+      cp_async4(&sm.scr.nk[buf][jj], nk_u + (valid ? j0 + jj : 0), valid);
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
   };
+  // visiting order: the chunk that holds the middle of this CTA's rows, then alternately the next one above and
+  // below (every chunk once).  seq_next() hands out that sequence.
+  const int c_home = min((i0 + TI / 2) / kJT, nchunks - 1);
+  int seq_lo = c_home - 1, seq_hi = c_home + 1, seq_n = 0;
+  auto seq_next = [&]() {
+    int c;
+    if (seq_n == 0) c = c_home;
+    else if (seq_hi < nchunks && (seq_lo < 0 || (seq_n & 1))) c = seq_hi++;
+    else c = seq_lo--;
+    ++seq_n;
+    return c;
+  };
 
-  load_chunk(0, 0);
+  int ch_cur = seq_next();  // visit 0 (threshold only) and visit 1 both take the home chunk
+  load_chunk(ch_cur, 0);
   for (int e = tid; e < TI * (kD / 4); e += NT) {
     const int r = e / (kD / 4), c4 = e - r * (kD / 4);
     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -204,7 +243,7 @@ __global__ void __launch_bounds__(NW * 32) topk_kernel(Geo g, const float* __res
   }
 
   // per row of this warp: block coordinates, norm bound, the lane's two best lower bounds, threshold, survivors
-  int iy[RI], ix[RI], cnt[RI];
+  int iy[RI], ix[RI], cnt[RI], cnt_upd[RI];
   float nqv[RI], m1[RI], m2[RI], thr[RI];
 #pragma unroll
   for (int a = 0; a < RI; ++a) {
@@ -213,20 +252,29 @@ __global__ void __launch_bounds__(NW * 32) topk_kernel(Geo g, const float* __res
     ix[a] = i - iy[a] * g.nbw;
     nqv[a] = __ldg(nq + (long long)u * g.m + i);
     m1[a] = -kInf; m2[a] = -kInf; thr[a] = -kInf;
-    cnt[a] = 0;
+    cnt[a] = 0; cnt_upd[a] = 0;
   }
   const unsigned lower = (1u << lane) - 1u;
 
-  // thr <- k-th largest of the warp's tracked lower bounds (a pop takes the largest out of its lane's pair)
-  auto update_threshold = [&](int a) {
-    float t1 = m1[a], t2 = m2[a];
+  // thr <- k-th largest of the warp's tracked lower bounds, for the rows in `rows` (bit a = row a), all of them in
+  // lockstep so that the latencies of their warp-wide steps overlap.  A pop takes the largest out of its lane's pair.
+  auto update_thresholds = [&](unsigned rows) {
+    float t1[RI], t2[RI];
+#pragma unroll
+    for (int a = 0; a < RI; ++a) { t1[a] = m1[a]; t2[a] = m2[a]; }
     for (int r = 0; r + 1 < g.topk; ++r) {
-      const unsigned o = ordered_bits(t1);
-      const unsigned best = __reduce_max_sync(0xffffffffu, o);
-      const unsigned who = __ballot_sync(0xffffffffu, o == best);
-      if (lane == __ffs(who) - 1) { t1 = t2; t2 = -kInf; }
+#pragma unroll
+      for (int a = 0; a < RI; ++a) {
+        if (!((rows >> a) & 1u)) continue;  // warp-uniform
+        const unsigned o = ordered_bits(t1[a]);
+        const unsigned best = __reduce_max_sync(0xffffffffu, o);
+        const unsigned who = __ballot_sync(0xffffffffu, o == best);
+        if (lane == __ffs(who) - 1) { t1[a] = t2[a]; t2[a] = -kInf; }
+      }
     }
-    thr[a] = from_ordered_bits(__reduce_max_sync(0xffffffffu, ordered_bits(t1)));
+#pragma unroll
+    for (int a = 0; a < RI; ++a)
+      if ((rows >> a) & 1u) thr[a] = from_ordered_bits(__reduce_max_sync(0xffffffffu, ordered_bits(t1[a])));
   };
   // drop the survivors of row a that the current threshold rules out (order kept)
   auto prune = [&](int a) {
@@ -251,13 +299,12 @@ __global__ void __launch_bounds__(NW * 32) topk_kernel(Geo g, const float* __res
     cnt[a] = kept;
   };
 
-  // chunk -1 is the first chunk screened for a threshold only; then every chunk, the first one again
-  for (int step = -1; step < nchunks; ++step) {
-    const int ch = max(step, 0), buf = (step + 1) & 1;
-    // the next chunk streams in while this one is screened (after the threshold pass: the first chunk once more)
-    const int nxt = step + 1 < nchunks ? max(step + 1, 0) : -1;
-    if (nxt >= 0) {
-      load_chunk(nxt, buf ^ 1);
+  // visit 0 screens the home chunk for a threshold only; visits 1 .. nchunks screen every chunk, the home chunk first
+  for (int v = 0; v <= nchunks; ++v) {
+    const int ch = ch_cur, buf = v & 1;
+    if (v < nchunks) {  // the next visit's chunk streams in while this one is screened
+      ch_cur = v == 0 ? ch : seq_next();
+      load_chunk(ch_cur, buf ^ 1);
       asm volatile("cp.async.wait_group 1;" ::: "memory");
     } else {
       asm volatile("cp.async.wait_group 0;" ::: "memory");
@@ -273,7 +320,7 @@ __global__ void __launch_bounds__(NW * 32) topk_kernel(Geo g, const float* __res
     for (int c4 = 0; c4 < kD / 4; ++c4) {
       float4 kv[4];
 #pragma unroll
-      for (int b = 0; b < 4; ++b) kv[b] = *reinterpret_cast<const float4*>(&sm.ks[buf][lane + 32 * b][4 * c4]);
+      for (int b = 0; b < 4; ++b) kv[b] = *reinterpret_cast<const float4*>(&sm.scr.ks[buf][lane + 32 * b][4 * c4]);
 #pragma unroll
       for (int a = 0; a < RI; ++a) {
         const float4 qv = *reinterpret_cast<const float4*>(&sm.qs[warp * RI + a][4 * c4]);
@@ -293,8 +340,9 @@ __global__ void __launch_bounds__(NW * 32) topk_kernel(Geo g, const float* __res
       const int j = min(j0 + lane + 32 * b, g.m - 1);
       jy[b] = j / g.nbw;
       jx[b] = j - jy[b] * g.nbw;
-      nkv[b] = sm.nk[buf][lane + 32 * b];
+      nkv[b] = sm.scr.nk[buf][lane + 32 * b];
     }
+    unsigned stale = 0;  // rows whose threshold should be recomputed
 #pragma unroll
     for (int a = 0; a < RI; ++a) {
       const bool row_ok = i0 + warp * RI + a < g.m;  // warp-uniform
@@ -309,7 +357,7 @@ __global__ void __launch_bounds__(NW * 32) topk_kernel(Geo g, const float* __res
         const float s = acc[a][b], eps = fmaf(nqv[a] * nkv[b], 1.52587890625e-5f, 1e-37f);
         const bool fin = fabsf(s) <= 1e38f && eps <= 1e38f;
         const float lb = fin ? s - eps : -kInf, ub = fin ? s + eps : kInf;
-        if (step >= 0) {
+        if (v >= 1) {
           const bool keep = cand && !(ub < thr[a]);
           const unsigned km = __ballot_sync(0xffffffffu, keep);
           if (keep) {
@@ -318,66 +366,103 @@ __global__ void __launch_bounds__(NW * 32) topk_kernel(Geo g, const float* __res
           }
           cnt[a] += __popc(km);
         }
-        if (step != 0 && cand) {  // the first chunk's bounds were tracked in the threshold pass
+        if (v != 1 && cand) {  // the home chunk's bounds were tracked in the threshold-only visit
           if (lb > m1[a]) { m2[a] = m1[a]; m1[a] = lb; }
           else m2[a] = fmaxf(m2[a], lb);
         }
       }
+      // recompute when the row has no threshold yet, gathered enough new survivors to suggest it is stale, fills
+      // up, or is about to be scored
+      const bool due = v <= 1 || v == nchunks || cnt[a] - cnt_upd[a] >= g.topk / 2 + 4 || cnt[a] > CAP / 2;
+      if (row_ok && due && cnt[a] <= CAP) stale |= 1u << a;
     }
-    // a higher threshold after the first chunks, then every fourth chunk, and at the end
-    if (step < 4 || (step & 3) == 3 || step == nchunks - 1) {
+    if (stale) {  // warp-uniform
       __syncwarp();
+      update_thresholds(stale);
 #pragma unroll
-      for (int a = 0; a < RI; ++a) {
-        update_threshold(a);
-        if (step >= 0) prune(a);
-      }
+      for (int a = 0; a < RI; ++a)
+        if ((stale >> a) & 1u) {
+          if (v >= 1) prune(a);
+          cnt_upd[a] = cnt[a];
+        }
     }
     __syncthreads();  // everyone is done with this buffer before the chunk after next lands in it
   }
 
-  // exact phase: one row of the warp at a time
+  // ---- exact phase (the staging buffers are free now and hold the survivors' score keys)
+  // rows whose survivors fit the counting rank: flatten (row, entry) pairs over the lanes, two chains in flight
+  int base_of[RI + 1];
+  base_of[0] = 0;
+  unsigned slow = 0;  // rows that take the insertion path (more than kExact survivors, or overflowed)
+#pragma unroll
+  for (int a = 0; a < RI; ++a) {
+    const bool row_ok = i0 + warp * RI + a < g.m;
+    const bool fast = row_ok && cnt[a] <= kExact;
+    if (row_ok && !fast) slow |= 1u << a;
+    base_of[a + 1] = base_of[a] + (fast ? cnt[a] : 0);
+  }
+  __syncwarp();
+  const int total = base_of[RI];
+  for (int p0 = 0; p0 < total; p0 += 64) {
+    int pa[2], pe[2], pj[2];
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+      const int p = p0 + 32 * t + lane;
+      pa[t] = -1; pe[t] = 0; pj[t] = 0;
+      if (p < total) {
+#pragma unroll
+        for (int a = 0; a < RI; ++a)
+          if (p >= base_of[a] && p < base_of[a + 1]) { pa[t] = a; pe[t] = p - base_of[a]; }
+        pj[t] = sm.surv[warp * RI + pa[t]][pe[t]];
+      }
+    }
+    // both chains in one instruction stream (inlined twice; the loads of the second overlap the first's arithmetic)
+    unsigned long long k0 = 0ull, k1 = 0ull;
+    if (pa[0] >= 0) k0 = exact_key(sm.qs[warp * RI + pa[0]], pk_u, pj[0]);
+    if (pa[1] >= 0) k1 = exact_key(sm.qs[warp * RI + pa[1]], pk_u, pj[1]);
+    if (pa[0] >= 0) sm.ekey[warp * RI + pa[0]][pe[0]] = k0;
+    if (pa[1] >= 0) sm.ekey[warp * RI + pa[1]][pe[1]] = k1;
+  }
+  __syncwarp();
 #pragma unroll
   for (int a = 0; a < RI; ++a) {
     const int row = warp * RI + a, i = i0 + row;
     if (i >= g.m) break;  // warp-uniform
-    const float* qrow = sm.qs[row];
-    auto exact_key = [&](int j) {
-      const float4* krow = reinterpret_cast<const float4*>(pk_u + (long long)j * kD);
-      double s = 0.0;
-#pragma unroll 4
-      for (int c4 = 0; c4 < kD / 4; ++c4) {
-        const float4 kv = __ldg(krow + c4);
-        s = fma((double)qrow[4 * c4], (double)kv.x, s);
-        s = fma((double)qrow[4 * c4 + 1], (double)kv.y, s);
-        s = fma((double)qrow[4 * c4 + 2], (double)kv.z, s);
-        s = fma((double)qrow[4 * c4 + 3], (double)kv.w, s);
+    int32_t* out = block_idx + ((long long)u * g.m + i) * g.topk;
+    if (!((slow >> a) & 1u)) {
+      const int n = cnt[a];
+      for (int e = lane; e < n; e += 32) {  // rank by counting the survivors that come first
+        const unsigned long long key = sm.ekey[row][e];
+        const int id = sm.surv[row][e];
+        int rank = 0;
+        for (int f = 0; f < n; ++f) rank += ranks_before(sm.ekey[row][f], sm.surv[row][f], key, id) ? 1 : 0;
+        if (rank < g.topk) out[rank] = id;
       }
-      return score_key(s);
-    };
-    unsigned long long lkey = 0ull;
-    int lid = -1;
-    __syncwarp();
-    if (cnt[a] <= CAP) {
-      for (int e0 = 0; e0 < cnt[a]; e0 += 32) {
-        const int e = e0 + lane;
-        const int j = e < cnt[a] ? sm.surv[row][e] : -1;
-        insert_batch(j >= 0 ? exact_key(j) : 0ull, j, lkey, lid, g.topk, lane);
-      }
-    } else {  // too many survivors to hold: score every key of the unit
-      for (int jb = 0; jb < g.m; jb += 32) {
-        const int j = jb + lane;
-        bool cand = j < g.m;
-        if (cand) {
-          const int jy = j / g.nbw, jx = j - jy * g.nbw;
-          int dx = jx - ix[a];
-          dx += dx < 0 ? g.nbw : 0;
-          cand = !(abs(jy - iy[a]) <= g.rlat && (dx <= g.rlon || g.nbw - dx <= g.rlon));
+      if (lane >= n && lane < g.topk) out[lane] = -1;
+    } else {
+      unsigned long long lkey = 0ull;
+      int lid = -1;
+      if (cnt[a] <= CAP) {
+        for (int e0 = 0; e0 < cnt[a]; e0 += 32) {
+          const int e = e0 + lane;
+          const int j = e < cnt[a] ? sm.surv[row][e] : -1;
+          insert_batch(j >= 0 ? exact_key(sm.qs[row], pk_u, j) : 0ull, j, lkey, lid, g.topk, lane);
         }
-        insert_batch(cand ? exact_key(j) : 0ull, j, lkey, lid, g.topk, lane);
+      } else {  // too many survivors to hold: score every key of the unit
+        for (int jb = 0; jb < g.m; jb += 32) {
+          const int j = jb + lane;
+          bool cand = j < g.m;
+          if (cand) {
+            const int jy = j / g.nbw, jx = j - jy * g.nbw;
+            int dx = jx - ix[a];
+            dx += dx < 0 ? g.nbw : 0;
+            cand = !(abs(jy - iy[a]) <= g.rlat && (dx <= g.rlon || g.nbw - dx <= g.rlon));
+          }
+          insert_batch(cand ? exact_key(sm.qs[row], pk_u, j) : 0ull, j, lkey, lid, g.topk, lane);
+        }
       }
+      if (lane < g.topk) out[lane] = lkey != 0ull ? lid : -1;
     }
-    if (lane < g.topk) block_idx[((long long)u * g.m + i) * g.topk + lane] = lkey != 0ull ? lid : -1;
   }
 }
 
@@ -420,7 +505,7 @@ int launch_select(const HostCtx& c, const void* q, const void* k, int32_t* block
     // the most query blocks per CTA (64, 32, 16) that still gives every SM about two CTAs; 16 otherwise
     auto ctas = [&](int ti) { return (long long)g.U * ((g.m + ti - 1) / ti); };
     const int rc = ctas(64) >= 296 ? launch_topk<8, 8, 128>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx)
-                 : ctas(32) >= 296 ? launch_topk<4, 8, 96>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx)
+                 : ctas(32) >= 296 ? launch_topk<4, 8, 128>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx)
                                    : launch_topk<4, 4, 192>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx);
     if (rc) return rc;
   }

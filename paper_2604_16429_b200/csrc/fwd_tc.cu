@@ -142,6 +142,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
         for (int e = 0; e < n && ok; ++e) {
           const int j = sm.ids[buf][e], by = j / g.nbw, bx = j - by * g.nbw;
+          const uint32_t mk = sm.mask[buf][e];
           for (int c = 0; c < g.cpb; ++c, ++step) {
             const int st = (int)(step % kStages);
             ok = mbar_wait(s32(&sm.kv_empty[st]), (uint32_t)((step / kStages) & 1) ^ 1, abort, status);
@@ -149,6 +150,10 @@ __global__ void __launch_bounds__(kThreads, 1)
             mbar_expect_tx(s32(&sm.kv_full[st]), 2 * kTile);
             tma_load_4d(s32(sm.kv[st][0]), &map_k, s32(&sm.kv_full[st]), 0, bx * g.bw, by * g.bh + c * g.crows, u);
             tma_load_4d(s32(sm.kv[st][1]), &map_v, s32(&sm.kv_full[st]), 0, bx * g.bw, by * g.bh + c * g.crows, u);
+            // a tile that does not attend this entry never looks at the stage: its release is given here (the other
+            // tile's release, after its P V, is what lets the stage be reused)
+            if (!(mk & 3u)) mbar_arrive(s32(&sm.kv_empty[st]));
+            if (!(mk & 12u)) mbar_arrive(s32(&sm.kv_empty[st]));
           }
         }
         if (ok) mbar_arrive(s32(&sm.list_empty[buf]));
@@ -205,16 +210,12 @@ __global__ void __launch_bounds__(kThreads, 1)
       uint32_t pend_n = 0;
       int pend_st = 0;
       for (int e = 0; e < n && ok; ++e) {
-        const bool act = (sm.mask[buf][e] & tbits) != 0;
+        if (!(sm.mask[buf][e] & tbits)) { step += g.cpb; continue; }  // not attended: the producer released the stages
         for (int c = 0; c < g.cpb && ok; ++c, ++step) {
           const int st = (int)(step % kStages);
           ok = __all_sync(0xffffffffu,
                           mbar_wait(s32(&sm.kv_full[st]), (uint32_t)((step / kStages) & 1), abort, status));
           if (!ok) break;
-          if (!act) {
-            if (elect_one()) mbar_arrive(s32(&sm.kv_empty[st]));
-            continue;
-          }
           // S buffer nt & 1 (aliased by P) was last read by P V of product nt - 2, which this warp issued
           // earlier: tensor-core operations of one thread execute in issue order, so this QK^T cannot
           // overwrite the buffer before that product has consumed it, and no wait is needed here

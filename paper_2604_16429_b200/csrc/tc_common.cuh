@@ -48,6 +48,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// Non-blocking test of a phase.
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 // Bounded wait.  Returns false after the limit (status recorded) or once another thread aborted.
 // The clock and the abort flag are looked at only every 64 polls to keep the poll loop light.
 __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort, int* status) {
@@ -68,6 +78,23 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort, int* status) {
   if (mbar_try_wait(bar, parity)) return true;
   return mbar_wait_slow(bar, parity, abort, status);
+}
+
+// Warp-wide wait: lane 0 polls, the warp learns the outcome and synchronises (polls by all 32 lanes serialise on the
+// barrier word and cost several times as much).  What lane 0 acquired is visible to the warp after the barrier.
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort, int* status, int lane) {
+  bool ok = true;
+  if (lane == 0) ok = mbar_wait(bar, parity, abort, status);
+  ok = __all_sync(0xffffffffu, ok);
+  __syncwarp();
+  return ok;
+}
+__device__ __forceinline__ bool warp_test(uint32_t bar, uint32_t parity, int lane) {
+  bool ok = true;
+  if (lane == 0) ok = mbar_test(bar, parity);
+  ok = __all_sync(0xffffffffu, ok);
+  __syncwarp();
+  return ok;
 }
 
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,

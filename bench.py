@@ -41,9 +41,34 @@ NOMINAL_BF16_TFLOPS = 2250.0
 FALLBACK_BF16_TFLOPS = 1590.0
 FALLBACK_HBM_GBS = 6650.0
 L2_FLUSH_BYTES = 256 << 20
-# DRAM bytes moved by one fwd_tc_kernel launch (ncu, dram__bytes_read.sum + dram__bytes_write.sum of the
-# capture summarised in profiles/fwd_tc_kernel_c2_1p5deg.md).  Workloads without a capture report null.
-FWD_TRAFFIC_BYTES = {"c2_1p5deg": 88.69e6 + 12.58e6}
+MIN_TIMED_SECONDS = 0.5           # the timed region is at least this long, whatever --steps says
+OTHER_WORKLOADS = ("c5_0p25deg", "c3_1p5deg_ens24")   # timed beside the default workload (forward only, few steps)
+OTHER_STEPS = 5
+
+
+def kernel_sources_digest() -> str:
+    """SHA-256 over the sources of the forward kernel: a stored DRAM-traffic figure is only reported while
+    the kernel it was measured on is the kernel that runs."""
+    import hashlib
+    h = hashlib.sha256()
+    for f in ("fwd_tc.cu", "tc_common.cuh", "common.cuh"):
+        h.update(open(os.path.join(ROOT, "paper_2604_16429_b200", "csrc", f), "rb").read())
+    return h.hexdigest()
+
+
+def measured_traffic(workload: str):
+    """DRAM bytes per launch of the forward kernel from the kept ncu summary of this workload, or None when
+    there is none or the kernel has changed since (the summary records the digest of the sources it measured)."""
+    import re
+    path = os.path.join(ROOT, "profiles", f"fwd_tc_kernel_{workload}.md")
+    if not os.path.exists(path):
+        return None, "no ncu capture kept for this workload"
+    m = re.search(r"kernel_sha256=([0-9a-f]{64})\s+dram_bytes_per_launch=([0-9.eE+]+)", open(path).read())
+    if not m:
+        return None, "the kept ncu summary carries no traffic record"
+    if m.group(1) != kernel_sources_digest():
+        return None, "kernel changed since the kept ncu capture"
+    return float(m.group(2)), "ncu dram__bytes_read.sum + dram__bytes_write.sum, one launch, kept summary of this workload"
 
 
 def measured_peaks():
@@ -195,6 +220,57 @@ def run_reference(args, w):
 
 
 # ------------------------------------------------------------------------------------------
+def forward_only(w, dev, peaks, steps, cuda_index) -> dict:
+    """Selection + forward of another workload, timed like the main one (CUDA events per step, L2 flushed
+    between steps, clocks sampled during the timed region); host generation of the inputs is outside it."""
+    import torch
+
+    from paper_2604_16429_b200 import binding as mb
+    x = synth.make_inputs(w, with_do=False)
+    dx = {k: torch.from_numpy(v.view(np.int16)).to(dev).view(torch.bfloat16) for k, v in x.items()}
+    del x
+    p = mb.Params.from_workload(w)
+    ws = torch.empty(max(mb.workspace_bytes(p, op) for op in (mb.OP_SELECT, mb.OP_FWD)), dtype=torch.uint8, device=dev)
+    idx = torch.empty((w.B, w.H, w.m, w.topk), dtype=torch.int32, device=dev)
+    o = torch.empty_like(dx["q"])
+    lse = torch.empty((w.B, w.H, w.N), dtype=torch.float32, device=dev)
+    flush_buf = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step(ev=None):
+        if ev:
+            ev[0].record(stream)
+        mb.mosaic_bsa_select(p, dx["q"], dx["k"], block_idx=idx, ws=ws)
+        if ev:
+            ev[1].record(stream)
+        mb.mosaic_bsa_fwd(p, dx["q"], dx["k"], dx["v"], idx, o=o, lse=lse, ws=ws)
+        if ev:
+            ev[2].record(stream)
+
+    for _ in range(3):
+        flush_buf.zero_()
+        step()
+    torch.cuda.synchronize()
+    mb.check_status(ws, "warm-up of " + w.name)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+    sampler = ClockSampler(cuda_index)
+    sampler.start()
+    for s in range(steps):
+        flush_buf.zero_()
+        step(evs[s])
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    mb.check_status(ws, "timed region of " + w.name)
+    t_sel = sum(e[0].elapsed_time(e[1]) for e in evs) / steps
+    t_fwd = sum(e[1].elapsed_time(e[2]) for e in evs) / steps
+    fl = flops.fwd_flops(w)
+    tf = fl / (t_fwd * 1e-3) / 1e12
+    return {"workload": describe(w), "steps": steps, "select_ms": t_sel, "fwd_ms": t_fwd, "ms_layer_fwd": t_sel + t_fwd,
+            "fwd_tflops": tf, "step_tflops": fl / ((t_sel + t_fwd) * 1e-3) / 1e12,
+            "roofline_frac_of_measured_burst": tf / peaks["bf16_tflops"], "frac_of_nominal_2250": tf / NOMINAL_BF16_TFLOPS,
+            "select_pool_gbs_lower_bound": 2.0 * w.U * w.N * w.d * 2 / (t_sel * 1e-3) / 1e9, "clocks": clocks}
+
+
 def run_ours(args, w):
     import torch
 
@@ -243,7 +319,15 @@ def run_ours(args, w):
     torch.cuda.synchronize()
     mb.check_status(ws, "warm-up")
 
-    K = args.steps
+    # step count: at least --steps, and enough for MIN_TIMED_SECONDS of GPU time (estimated from a short probe)
+    probe = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    probe[0].record(stream)
+    for _ in range(5):
+        flush_buf.zero_()
+        fwd_step()
+    probe[1].record(stream)
+    torch.cuda.synchronize()
+    K = max(args.steps, min(20000, int(args.min_seconds * 1e3 / max(probe[0].elapsed_time(probe[1]) / 5, 1e-3)) + 1))
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
     sampler = ClockSampler(local_rank)
     mdist.barrier()
@@ -261,7 +345,7 @@ def run_ours(args, w):
     mb.check_status(ws, "timed region")
 
     # backward of the same workload, timed the same way (reported under "stages")
-    kb = min(K, 20)
+    kb = min(K, 50)
     evb = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(kb)]
     for s in range(kb):
         flush_buf.zero_()
@@ -272,7 +356,7 @@ def run_ours(args, w):
     t_bwd = sum(e[0].elapsed_time(e[1]) for e in evb) / kb
 
     # end to end: pinned host -> device, step, device -> pinned host
-    ke = min(K, 10)
+    ke = min(K, 20)
     o_host = torch.empty(o.shape, dtype=torch.int16).pin_memory()
     eve = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(ke)]
     for s in range(ke + 1):
@@ -289,6 +373,7 @@ def run_ours(args, w):
     h2d = 3 * dx["q"].numel() * 2
     d2h = o.numel() * 2
 
+    traffic, traffic_source = measured_traffic(w.name)
     t_step_max = mdist.max_over_ranks(t_step, dev)
     t_e2e_max = mdist.max_over_ranks(t_e2e, dev)
     fl = flops.fwd_flops(w)
@@ -298,7 +383,8 @@ def run_ours(args, w):
     pool_bytes = 2.0 * w.U * w.N * w.d * 2
 
     line = {
-        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": K, "steps_requested": args.steps,
+        "warmup": max(args.warmup, 3),
         "ms_per_step": t_step_max, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": describe(w), "l2": f"flushed between timed iterations ({L2_FLUSH_BYTES >> 20} MiB write)",
@@ -309,7 +395,7 @@ def run_ours(args, w):
         "gpu_launches": 3 * K,
         "roofline": {"kernel": "fwd_tc_kernel", "bound": "tensor", "achieved": fwd_tflops,
                      "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": fwd_tflops / peaks["bf16_tflops"],
-                     "traffic": FWD_TRAFFIC_BYTES.get(w.name), "peak_source": peaks["source"] + " (burst)",
+                     "traffic": traffic, "traffic_source": traffic_source, "peak_source": peaks["source"] + " (burst)",
                      "frac_of_nominal_2250": fwd_tflops / NOMINAL_BF16_TFLOPS, "ms": t_fwd},
         "stages": {"select_ms": t_sel, "fwd_ms": t_fwd, "bwd_ms": t_bwd, "ms_layer_fwd": t_step,
                    "fwd_tflops": fwd_tflops, "bwd_tflops": flops.bwd_flops(w) / (t_bwd * 1e-3) / 1e12,
@@ -320,6 +406,11 @@ def run_ours(args, w):
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(w, x, idx, o, lse)
+    if world == 1 and args.workload == "c2_1p5deg" and not args.no_other_workloads:
+        del dx, host, o, lse, dq, dk, dv, idx, ws, x
+        torch.cuda.empty_cache()
+        line["other_workloads"] = {name: forward_only(synth.WORKLOADS[name], dev, peaks, OTHER_STEPS, local_rank)
+                                   for name in OTHER_WORKLOADS}
     if rank == 0:
         print(json.dumps(line), flush=True)
     mdist.finalize()
@@ -333,6 +424,9 @@ def main():
     ap.add_argument("--workload", default="c2_1p5deg", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-other-workloads", action="store_true")
+    ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_SECONDS,
+                    help="floor of the timed region in seconds of GPU time (0: exactly --steps steps, for profiler captures)")
     args = ap.parse_args()
     w = synth.WORKLOADS[args.workload]
     if args.impl == "reference":

@@ -151,7 +151,7 @@ int mosaic_bsa_bwd(const mosaic_bsa_params* p, const void* q, const void* k, con
   for (const void* x : ptrs)
     if (!aligned(x, 16)) return MOSAIC_E_MISALIGNED;
   if (!aligned(lse, 4) || !aligned(block_idx, 4)) return MOSAIC_E_MISALIGNED;
-  if ((size_t)g.m * sizeof(int) > 200 * 1024) return MOSAIC_E_UNSUPPORTED;
+  if (2 * (size_t)g.m * sizeof(int) + (size_t)g.m * g.topk / 8 + 8 > 200 * 1024) return MOSAIC_E_UNSUPPORTED;  // transposed-pattern kernel
   BwdWs w = bwd_layout(g);
   if ((rc = begin(p, ws, ws_bytes, w.total, cuda_stream, &c))) return rc;
   char* base = (char*)ws;

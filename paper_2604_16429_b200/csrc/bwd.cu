@@ -50,60 +50,98 @@ __global__ void __launch_bounds__(256) rowdot_kernel(long long tokens, const uin
 
 // ------------------------------------------------------------------------------------------
 // Transposed pattern: for every key block j the ascending list of query blocks that selected it.
-// One CTA per unit: histogram, exclusive scan, then an ordered fill by a single warp so that
-// each list comes out sorted by query block id (this fixes the dK/dV summation order).
+// One CTA per unit.  The query blocks are cut into `nseg` contiguous segments:
+//   1. one thread per query block validates its row of block_idx (ids outside [0, m), ids of the row's own
+//      neighbourhood and repeats are dropped, exactly as the forward drops them), marks the valid entries in a
+//      bit array and counts them per (segment, key block);
+//   2. per key block, a running sum over the segments and an exclusive scan over the key blocks turn the counts
+//      into the position where each segment's part of each list starts;
+//   3. every warp fills its segments in entry order, so each list comes out sorted by query block id (this
+//      fixes the dK/dV summation order).
+// Shared memory: (nseg + 1) * m counters + m * topk bits.
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) csr_kernel(Geo g, const int32_t* __restrict__ block_idx,
-                                                  int32_t* __restrict__ csr_off, int32_t* __restrict__ csr_q) {
-  extern __shared__ int cur[];  // [m] counts, then running cursors
-  const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
+                                                  int32_t* __restrict__ csr_off, int32_t* __restrict__ csr_q, int nseg) {
+  extern __shared__ int csr_sm[];
+  int* tot = csr_sm;                        // [m] list lengths, then list starts
+  int* seg = csr_sm + g.m;                  // [nseg][m] counts, then cursors
+  unsigned* bits = reinterpret_cast<unsigned*>(seg + (long long)nseg * g.m);  // [ceil(m * topk / 32)] valid entries
+  const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int32_t* idx = block_idx + (long long)u * g.m * g.topk;
   int32_t* off = csr_off + (long long)u * (g.m + 1);
   int32_t* outq = csr_q + (long long)u * g.m * g.topk;
-  const int E = g.m * g.topk;
-  for (int j = tid; j < g.m; j += blockDim.x) cur[j] = 0;
+  const int E = g.m * g.topk, rps = (g.m + nseg - 1) / nseg;  // rows per segment
+  for (int x = tid; x < (nseg + 1) * g.m; x += blockDim.x) csr_sm[x] = 0;
+  for (int x = tid; x < (E + 31) / 32; x += blockDim.x) bits[x] = 0u;
   __syncthreads();
-  for (int e = tid; e < E; e += blockDim.x) {
-    const int i = e / g.topk;
-    bool report;
-    if (selected_entry_ok(g, idx + (long long)i * g.topk, i, e - i * g.topk, &report)) atomicAdd(&cur[idx[e]], 1);
+  for (int i = tid; i < g.m; i += blockDim.x) {
+    const int32_t* row = idx + (long long)i * g.topk;
+    int* cnt = seg + (long long)(i / rps) * g.m;
+    for (int r = 0; r < g.topk; ++r) {
+      bool report;
+      if (selected_entry_ok(g, row, i, r, &report)) {
+        atomicAdd(&cnt[row[r]], 1);
+        const int e = i * g.topk + r;
+        atomicOr(&bits[e >> 5], 1u << (e & 31));
+      }
+    }
+  }
+  __syncthreads();
+  for (int j = tid; j < g.m; j += blockDim.x) {
+    int t = 0;
+    for (int sgm = 0; sgm < nseg; ++sgm) {
+      const int c = seg[(long long)sgm * g.m + j];
+      seg[(long long)sgm * g.m + j] = t;
+      t += c;
+    }
+    tot[j] = t;
   }
   __syncthreads();
   if (tid < 32) {
     int carry = 0;
     for (int base = 0; base < g.m; base += 32) {
-      int j = base + lane;
-      int v = j < g.m ? cur[j] : 0, incl = v;
+      const int j = base + lane;
+      const int v = j < g.m ? tot[j] : 0;
+      int incl = v;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
-        int n = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += n;
+        const int nb = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += nb;
       }
-      if (j < g.m) { off[j] = carry + incl - v; cur[j] = carry + incl - v; }
+      if (j < g.m) { off[j] = carry + incl - v; tot[j] = carry + incl - v; }
       carry += __shfl_sync(0xffffffffu, incl, 31);
     }
     if (lane == 0) off[g.m] = carry;
-    __syncwarp();
-    for (int e0 = 0; e0 < E; e0 += 32) {
-      int e = e0 + lane;
+  }
+  __syncthreads();
+  for (int sgm = warp; sgm < nseg; sgm += (int)(blockDim.x >> 5)) {
+    int* cur = seg + (long long)sgm * g.m;  // only this warp touches this segment's cursors
+    const int e_beg = sgm * rps * g.topk, e_end = min(E, (sgm + 1) * rps * g.topk);
+    for (int e0 = e_beg; e0 < e_end; e0 += 32) {
+      const int e = e0 + lane;
       int j = -1;
-      if (e < E) {
-        const int i = e / g.topk;
-        bool report;
-        if (selected_entry_ok(g, idx + (long long)i * g.topk, i, e - i * g.topk, &report)) j = idx[e];
-      }
-      int key = j < 0 ? -1 - lane : j;  // invalid entries never match each other
-      unsigned mask = __match_any_sync(0xffffffffu, key);
-      int rank = __popc(mask & ((1u << lane) - 1u));
-      int base = j >= 0 ? cur[j] : 0;
+      if (e < e_end && ((bits[e >> 5] >> (e & 31)) & 1u)) j = idx[e];
+      const int key = j < 0 ? -1 - lane : j;  // invalid entries never match each other
+      const unsigned same = __match_any_sync(0xffffffffu, key);
+      const int rank = __popc(same & ((1u << lane) - 1u));
+      const int base = j >= 0 ? tot[j] + cur[j] : 0;
       __syncwarp();
       if (j >= 0) {
         outq[base + rank] = e / g.topk;
-        if (rank == 0) cur[j] = base + __popc(mask);
+        if (rank == 0) cur[j] += __popc(same);
       }
       __syncwarp();
     }
   }
+}
+
+// segments of the transposed-pattern kernel that fit the shared memory (8 when possible: one per warp)
+static int csr_segments(const Geo& g, size_t* smem) {
+  const size_t budget = 200 * 1024, bits = 4 * (((size_t)g.m * g.topk + 31) / 32);
+  int nseg = 8;
+  while (nseg > 1 && (size_t)(nseg + 1) * g.m * sizeof(int) + bits > budget) --nseg;
+  *smem = (size_t)(nseg + 1) * g.m * sizeof(int) + bits;
+  return *smem <= budget ? nseg : 0;
 }
 
 int launch_bwd(const HostCtx& c, const void* q, const void* k, const void* v, const void* o, const float* lse,
@@ -119,12 +157,18 @@ int launch_bwd(const HostCtx& c, const void* q, const void* k, const void* v, co
     if (cudaGetLastError() != cudaSuccess) return MOSAIC_E_CUDA;
   }
   if (g.topk > 0) {
-    size_t smem = sizeof(int) * (size_t)g.m;
-    if (smem > 48 * 1024) {
-      if (cudaFuncSetAttribute(csr_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    size_t smem = 0;
+    const int nseg = csr_segments(g, &smem);
+    if (nseg == 0) return MOSAIC_E_UNSUPPORTED;
+    static unsigned long long configured = 0;  // devices on which the kernel's shared-memory opt-in is set
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return MOSAIC_E_CUDA;
+    if (dev >= 0 && dev < 64 && !((configured >> dev) & 1ull)) {
+      if (cudaFuncSetAttribute(csr_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
         return MOSAIC_E_CUDA;
+      configured |= 1ull << dev;
     }
-    csr_kernel<<<g.U, 256, smem, c.stream>>>(g, block_idx, csr_off, csr_q);
+    csr_kernel<<<g.U, 256, smem, c.stream>>>(g, block_idx, csr_off, csr_q, nseg);
   } else {
     if (cudaMemsetAsync(csr_off, 0, sizeof(int32_t) * (size_t)g.U * (g.m + 1), c.stream) != cudaSuccess)
       return MOSAIC_E_CUDA;

@@ -28,7 +28,7 @@ namespace mosaic {
 namespace {
 
 constexpr int kStages = 6;       // ring depth of query-side chunks
-constexpr int kThreads = 384;    // warps 0-7 row threads, 8 TMA producer, 9 MMA issuer, 10 idle, 11 planner
+constexpr int kThreads = 384;    // warps 0-7 row threads, 8 TMA producer, 9 and 10 MMA issuers, 11 planner
 constexpr uint32_t kTmemCols = 512;
 // dK, dV accumulators; S^T and dP^T (fp32); P^T and dS^T (bf16 pairs)
 constexpr uint32_t kColDK = 0, kColDV = 64, kColS = 128, kColDP = 192, kColP = 256, kColDS = 288;
@@ -155,7 +155,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     mbar_init(s32(&sm.pv_done), 1);
     for (int i = 0; i < kLists; ++i) {
       mbar_init(s32(&sm.list_full[i]), 1);
-      mbar_init(s32(&sm.list_empty[i]), 10);  // 8 row-thread warps + MMA warp + TMA producer
+      mbar_init(s32(&sm.list_empty[i]), 11);  // 8 row-thread warps + 2 MMA issuers + TMA producer
     }
     sm.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -233,84 +233,92 @@ __global__ void __launch_bounds__(kThreads, 1)
       }
     }
   } else if (warp == 9) {
-    // ------------------------------------------------------------- MMA issuer
-    // The whole warp walks the loop; one elected lane issues the tensor-core instructions.
-    constexpr uint32_t idesc_nt = make_idesc(false), idesc_nn = make_idesc(true);
-    const uint64_t kdesc = smem_desc(s32(sm.k)), vdesc = smem_desc(s32(sm.v));
-    long long step = 0;   // ring position
-    uint32_t nt = 0;      // products started so far (phase of the per-product barriers)
-    int items = 0;
-    bool ok = true, fresh = true, first = true;
-    bool pend = false, pend_first = false;
-    int pend_st = 0;
-    // dV += P^T dO and dK += dS^T Q of the previous product (its chunks sit in ring stage `pst`)
-    auto issue_grads = [&](int pst, bool pfirst) {
-      ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.p_full), (nt - 1) & 1, abort, status));
-      if (!ok) return;
-      tc_fence_after();
-      const uint64_t qmn = smem_desc(s32(sm.ring[pst].q)), domn = smem_desc(s32(sm.ring[pst].d_o));
-      if (elect_one()) {
-#pragma unroll
-        for (int kk = 0; kk < 4; ++kk)
-          umma_ts(tmem + kColDV, tmem + kColP + 8 * kk, domn + (uint64_t)((2048 * kk) >> 4), idesc_nn,
-                  (!pfirst || kk > 0));
-#pragma unroll
-        for (int kk = 0; kk < 4; ++kk)
-          umma_ts(tmem + kColDK, tmem + kColDS + 8 * kk, qmn + (uint64_t)((2048 * kk) >> 4), idesc_nn,
-                  (!pfirst || kk > 0));
-        tc_commit(s32(&sm.ring_empty[pst]));
-        tc_commit(s32(&sm.pv_done));
-      }
-      __syncwarp();
-    };
-    for (int lb = 0; ok; ++lb) {
-      const int buf = lb % kLists;
-      ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.list_full[buf]), (lb / kLists) & 1, abort, status));
-      if (!ok) break;
-      const int n = sm.info[buf].n;
-      if (n < 0) break;
-      const bool more = sm.info[buf].more != 0;
-      if (fresh) {
-        ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.kv_full), items & 1, abort, status));
+    // ------------------------------------------------------------- issuer of S^T = K Q^T and dP^T = V dO^T (one thread)
+    // A thread issues an N = 64 product no faster than one in about 50 cycles; the sixteen products of a step are
+    // split over two issuing threads (this one and warp 10), which are ordered by barriers only.
+    if (lane == 0) {
+      constexpr uint32_t idesc_nt = make_idesc(false);
+      const uint64_t kdesc = smem_desc(s32(sm.k)), vdesc = smem_desc(s32(sm.v));
+      long long step = 0;   // ring position
+      uint32_t nt = 0;      // products started so far (phase of the per-product barriers)
+      int items = 0;
+      bool ok = true, fresh = true;
+      for (int lb = 0; ok; ++lb) {
+        const int buf = lb % kLists;
+        ok = mbar_wait(s32(&sm.list_full[buf]), (lb / kLists) & 1, abort, status);
         if (!ok) break;
-        ++items;
-        first = true;
-      }
-      fresh = !more;
-      for (int e = 0; e < n && ok; ++e) {
-        for (int c = 0; c < g.cpb && ok; ++c, ++step) {
-          const int st = (int)(step % kStages);
-          ok = __all_sync(0xffffffffu,
-                          mbar_wait(s32(&sm.ring_full[st]), (uint32_t)((step / kStages) & 1), abort, status));
+        const int n = sm.info[buf].n;
+        if (n < 0) break;
+        const bool more = sm.info[buf].more != 0;
+        if (fresh) {
+          ok = mbar_wait(s32(&sm.kv_full), items & 1, abort, status);
           if (!ok) break;
-          // S^T and dP^T may be overwritten once the row threads hold the previous product in registers
-          if (nt > 0) {
-            ok = __all_sync(0xffffffffu, mbar_wait(s32(&sm.sdp_free), (nt - 1) & 1, abort, status));
+          ++items;
+        }
+        fresh = !more;
+        for (int e = 0; e < n && ok; ++e) {
+          for (int c = 0; c < g.cpb && ok; ++c, ++step) {
+            const int st = (int)(step % kStages);
+            ok = mbar_wait(s32(&sm.ring_full[st]), (uint32_t)((step / kStages) & 1), abort, status);
+            // S^T and dP^T may be overwritten once the row threads hold the previous product in registers
+            if (ok && nt > 0) ok = mbar_wait(s32(&sm.sdp_free), (nt - 1) & 1, abort, status);
             if (!ok) break;
-          }
-          tc_fence_after();
-          const uint64_t qdesc = smem_desc(s32(sm.ring[st].q)), dodesc = smem_desc(s32(sm.ring[st].d_o));
-          if (elect_one()) {
+            tc_fence_after();
+            const uint64_t qdesc = smem_desc(s32(sm.ring[st].q)), dodesc = smem_desc(s32(sm.ring[st].d_o));
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk) umma_ss(tmem + kColS, kdesc + 2 * kk, qdesc + 2 * kk, idesc_nt, kk > 0);
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk) umma_ss(tmem + kColDP, vdesc + 2 * kk, dodesc + 2 * kk, idesc_nt, kk > 0);
             tc_commit(s32(&sm.s_full));
+            ++nt;
           }
-          __syncwarp();
-          if (pend) issue_grads(pend_st, pend_first);
-          if (!ok) break;
-          pend = true; pend_st = st; pend_first = first;
-          first = false;
-          ++nt;
         }
+        // the K and V tiles are read by this thread's products only: all of the item's are behind this commit
+        if (ok && !more) tc_commit(s32(&sm.kv_empty));
+        if (ok) mbar_arrive(s32(&sm.list_empty[buf]));
       }
-      if (ok && !more) {
-        if (pend) issue_grads(pend_st, pend_first);  // the item's last product
-        pend = false;
-        if (ok && elect_one()) tc_commit(s32(&sm.kv_empty));  // all products of the item are behind it
+    }
+  } else if (warp == 10) {
+    // ------------------------------------------------------------- issuer of dV += P^T dO and dK += dS^T Q (one thread)
+    if (lane == 0) {
+      constexpr uint32_t idesc_nn = make_idesc(true);
+      long long step = 0;
+      uint32_t nt = 0;
+      bool ok = true, first = true;
+      for (int lb = 0; ok; ++lb) {
+        const int buf = lb % kLists;
+        ok = mbar_wait(s32(&sm.list_full[buf]), (lb / kLists) & 1, abort, status);
+        if (!ok) break;
+        const int n = sm.info[buf].n;
+        if (n < 0) break;
+        const bool more = sm.info[buf].more != 0;
+        for (int e = 0; e < n && ok; ++e) {
+          for (int c = 0; c < g.cpb && ok; ++c, ++step) {
+            const int st = (int)(step % kStages);
+            // the stage landed before S^T could be produced; this wait makes the copied Q and dO visible here too
+            ok = mbar_wait(s32(&sm.ring_full[st]), (uint32_t)((step / kStages) & 1), abort, status);
+            if (ok) ok = mbar_wait(s32(&sm.p_full), nt & 1, abort, status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint64_t qmn = smem_desc(s32(sm.ring[st].q)), domn = smem_desc(s32(sm.ring[st].d_o));
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+              umma_ts(tmem + kColDV, tmem + kColP + 8 * kk, domn + (uint64_t)((2048 * kk) >> 4), idesc_nn,
+                      (!first || kk > 0));
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+              umma_ts(tmem + kColDK, tmem + kColDS + 8 * kk, qmn + (uint64_t)((2048 * kk) >> 4), idesc_nn,
+                      (!first || kk > 0));
+            // the stage's S^T and dP^T completed before P^T could be formed, so this thread's completion frees it
+            tc_commit(s32(&sm.ring_empty[st]));
+            tc_commit(s32(&sm.pv_done));
+            first = false;
+            ++nt;
+          }
+        }
+        if (!more) first = true;  // the next list buffer starts a new item: new accumulation
+        if (ok) mbar_arrive(s32(&sm.list_empty[buf]));
       }
-      if (ok && elect_one()) mbar_arrive(s32(&sm.list_empty[buf]));
     }
   } else if (warp < 8) {
     // ------------------------------------------------------------- row threads (TMEM lane = key row)

@@ -190,6 +190,41 @@ def bwd_blocks(g: Geom, q, k, v, d_o, idx, qblocks, kblocks):
     return dQ[:qb.size], dK[:kb.size], dV[:kb.size]
 
 
+def fwd3(g: Geom, q, k, v, idx, gates):
+    """Three-branch form of one unit (compression + selection + local, gated).  `gates` is [N, 3] (CG, FG, L).
+    Returns a dict of fp64 arrays in token order: o, o_cg, o_fg, o_l [N, d]; lse_fg, lse_l [N]; abar [m, m]."""
+    q, k, v = _u16(q, g), _u16(k, g), _u16(v, g)
+    idx = np.ascontiguousarray(idx, np.int32).reshape(g.m, g.topk)
+    gt = np.ascontiguousarray(gates, np.float64)
+    assert gt.shape == (g.N, 3)
+    out = {n: np.zeros((g.N, g.d)) for n in ("o", "o_cg", "o_fg", "o_l")}
+    out["lse_fg"] = np.zeros(g.N); out["lse_l"] = np.zeros(g.N); out["abar"] = np.zeros((g.m, g.m))
+    gc = g.c()
+    dp = ctypes.c_double
+    rc = _load().mo_fwd3_unit(ctypes.byref(gc), _p(q, ctypes.c_uint16), _p(k, ctypes.c_uint16), _p(v, ctypes.c_uint16),
+                              _p(idx, ctypes.c_int32), _p(gt, dp), _p(out["o"], dp), _p(out["o_cg"], dp),
+                              _p(out["o_fg"], dp), _p(out["o_l"], dp), _p(out["lse_fg"], dp), _p(out["lse_l"], dp),
+                              _p(out["abar"], dp))
+    assert rc == 0
+    return out
+
+
+def bwd3(g: Geom, q, k, v, d_o, idx, gates):
+    """Backward of the three-branch form of one unit: (dQ, dK, dV [N, d], dGates [N, 3]) in fp64, token order."""
+    q, k, v, d_o = _u16(q, g), _u16(k, g), _u16(v, g), _u16(d_o, g)
+    idx = np.ascontiguousarray(idx, np.int32).reshape(g.m, g.topk)
+    gt = np.ascontiguousarray(gates, np.float64)
+    assert gt.shape == (g.N, 3)
+    dQ = np.zeros((g.N, g.d)); dK = np.zeros((g.N, g.d)); dV = np.zeros((g.N, g.d)); dG = np.zeros((g.N, 3))
+    gc = g.c()
+    dp = ctypes.c_double
+    rc = _load().mo_bwd3_unit(ctypes.byref(gc), _p(q, ctypes.c_uint16), _p(k, ctypes.c_uint16), _p(v, ctypes.c_uint16),
+                              _p(d_o, ctypes.c_uint16), _p(idx, ctypes.c_int32), _p(gt, dp), _p(dQ, dp), _p(dK, dp),
+                              _p(dV, dp), _p(dG, dp))
+    assert rc == 0
+    return dQ, dK, dV, dG
+
+
 def block_tokens(g: Geom, j: int) -> np.ndarray:
     """Token ids of block j in row-major order inside the block (layout helper)."""
     by, bx = divmod(j, g.nbw)

@@ -29,10 +29,16 @@
  *                   held constant; dK/dV visit only the query blocks connected to a
  *                   key/value block ("Kernel Design" paragraph of the appendix).
  *
+ *   three-branch -- mo_fwd3_unit / mo_bwd3_unit at the end of this file: the paper's own gated sum of the
+ *                   compression, selection and local branches (Eq. of the aggregated output), each
+ *                   branch with its own softmax, gradient into the routing scores through the
+ *                   compression branch.
+ *
  * Pins (tests/test_oracle_*.py): dense attention when top-k covers every block,
  * brute-force selection on tiny grids, hand-built winners and ties, row-stochastic
  * weights, convex-hull bound, finite differences, longitude-roll equivariance,
- * zero gradient for unconnected blocks, the cost-model pair count.
+ * zero gradient for unconnected blocks, the cost-model pair count; NaN ordering; for the three-branch
+ * form each branch against a textbook routine, its link to the union form, finite differences.
  * Parity unpinned: agreement with the authors' own kernels (not available).
  */
 #include <math.h>
@@ -483,5 +489,259 @@ int mo_bwd_blocks(const mo_geom *g, const uint16_t *q, const uint16_t *k, const 
     free(conn);
   }
   free(need); free(list); free(Ob); free(Lb); free(LSE); free(D);
+  return 0;
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * Three-branch output (the paper's own form of the operator: Eq. of the aggregated output in the
+ * section "Native Sparse Attention", and the "Compression", "Selection" and "Local Attention"
+ * paragraphs of the section "Block-Sparse Attention").  For token l of query block i:
+ *   compression  oCG_l = sum_{j=1..m} abar_ij vbar_j,  abar_i,: = softmax_j(qbar_i . kbar_j * scale) over ALL
+ *                m blocks, qbar, kbar, vbar the block MEANS (fp32-rounded block sum / b); the same vector for
+ *                every token of the block;
+ *   selection    oFG_l = softmax attention of q_l over the tokens of the selected blocks (own normaliser);
+ *                an empty selection gives oFG_l = 0 and LSE = -inf;
+ *   local        oL_l  = softmax attention of q_l over the tokens of the local neighbourhood (own normaliser);
+ *   output       o_l   = gates[l][0] * oCG_l + gates[l][1] * oFG_l + gates[l][2] * oL_l.
+ * The gates are functions of the layer input in the paper and therefore inputs here.
+ * ------------------------------------------------------------------------------------------------ */
+
+/* softmax attention of one query row over the tokens of a list of blocks; returns LSE (-inf if none) */
+static double branch_row(const mo_geom *g, const uint16_t *q, const uint16_t *k, const uint16_t *v, int64_t l,
+                         const int32_t *blk, int nb, double *x, double *o) {
+  int b = g_b(g), d = g->d, nt = nb * b;
+  for (int c = 0; c < d; ++c) o[c] = 0.0;
+  if (nb == 0) return -INFINITY;
+  row_logits(g, q, k, l, blk, nb, x);
+  double M = -INFINITY, Z = 0.0;
+  for (int t = 0; t < nt; ++t) M = x[t] > M ? x[t] : M;
+  for (int t = 0; t < nt; ++t) Z += exp(x[t] - M);
+  for (int a = 0; a < nb; ++a)
+    for (int e2 = 0; e2 < b; ++e2) {
+      double w = exp(x[(size_t)a * b + e2] - M) / Z;
+      int64_t t = block_token(g, blk[a], e2);
+      for (int c = 0; c < d; ++c) o[c] += w * bf16_widen(v[t * d + c]);
+    }
+  return M + log(Z);
+}
+
+/* block means of one tensor: fp32-rounded block sum (as in the selection) divided by b, in double */
+static void block_means(const mo_geom *g, const uint16_t *x, double *mean /* [m,d] */) {
+  int m = g_m(g), d = g->d;
+  float *p = (float *)malloc(sizeof(float) * (size_t)m * d);
+  mo_pool_unit(g, x, p);
+  for (size_t z = 0; z < (size_t)m * d; ++z) mean[z] = (double)p[z] / (double)g_b(g);
+  free(p);
+}
+
+/*
+ * Forward of the three-branch form for one unit.  gates is [N,3] (CG, FG, L) in token order.
+ * Outputs in token order: O [N,d]; optional OCG, OFG, OL [N,d] (branch outputs before gating),
+ * LSE_FG, LSE_L [N], ABAR [m,m] (block-level attention).
+ */
+int mo_fwd3_unit(const mo_geom *g, const uint16_t *q, const uint16_t *k, const uint16_t *v, const int32_t *idx,
+                 const double *gates, double *O, double *OCG, double *OFG, double *OL, double *LSE_FG,
+                 double *LSE_L, double *ABAR) {
+  if (!g_ok(g)) return -1;
+  int m = g_m(g), b = g_b(g), d = g->d;
+  double sc = g_scale(g);
+  double *qm = (double *)malloc(sizeof(double) * (size_t)m * d);
+  double *km = (double *)malloc(sizeof(double) * (size_t)m * d);
+  double *vm = (double *)malloc(sizeof(double) * (size_t)m * d);
+  double *ocg = (double *)malloc(sizeof(double) * (size_t)m * d);
+  if (!qm || !km || !vm || !ocg) { free(qm); free(km); free(vm); free(ocg); return -2; }
+  block_means(g, q, qm);
+  block_means(g, k, km);
+  block_means(g, v, vm);
+  /* compression branch: block-to-block softmax attention on the means */
+#pragma omp parallel
+  {
+    double *s = (double *)malloc(sizeof(double) * (size_t)m);
+#pragma omp for schedule(static)
+    for (int i = 0; i < m; ++i) {
+      double M = -INFINITY, Z = 0.0;
+      for (int j = 0; j < m; ++j) {
+        double a = 0.0;
+        for (int c = 0; c < d; ++c) a += qm[(size_t)i * d + c] * km[(size_t)j * d + c];
+        s[j] = sc * a;
+        M = s[j] > M ? s[j] : M;
+      }
+      for (int j = 0; j < m; ++j) Z += exp(s[j] - M);
+      for (int c = 0; c < d; ++c) ocg[(size_t)i * d + c] = 0.0;
+      for (int j = 0; j < m; ++j) {
+        double a = exp(s[j] - M) / Z;
+        if (ABAR) ABAR[(size_t)i * m + j] = a;
+        for (int c = 0; c < d; ++c) ocg[(size_t)i * d + c] += a * vm[(size_t)j * d + c];
+      }
+    }
+    free(s);
+  }
+  /* selection and local branches, then the gated sum */
+  int max_att = MO_MAX_LOCAL + g->topk;
+#pragma omp parallel
+  {
+    int32_t *loc = (int32_t *)malloc(sizeof(int32_t) * MO_MAX_LOCAL);
+    int32_t *sel = (int32_t *)malloc(sizeof(int32_t) * (size_t)(g->topk > 0 ? g->topk : 1));
+    double *x = (double *)malloc(sizeof(double) * (size_t)max_att * b);
+    double *ofg = (double *)malloc(sizeof(double) * (size_t)d), *ol = (double *)malloc(sizeof(double) * (size_t)d);
+#pragma omp for schedule(dynamic, 1)
+    for (int i = 0; i < m; ++i) {
+      int nl = mo_local_set(g, i, loc), ns = 0;
+      for (int r = 0; r < g->topk; ++r)
+        if (idx[(size_t)i * g->topk + r] >= 0) sel[ns++] = idx[(size_t)i * g->topk + r];
+      for (int e = 0; e < b; ++e) {
+        int64_t l = block_token(g, i, e);
+        double lf = branch_row(g, q, k, v, l, sel, ns, x, ofg);
+        double ll = branch_row(g, q, k, v, l, loc, nl, x, ol);
+        for (int c = 0; c < d; ++c) {
+          double cg = ocg[(size_t)i * d + c];
+          O[l * d + c] = gates[l * 3 + 0] * cg + gates[l * 3 + 1] * ofg[c] + gates[l * 3 + 2] * ol[c];
+          if (OCG) OCG[l * d + c] = cg;
+          if (OFG) OFG[l * d + c] = ofg[c];
+          if (OL) OL[l * d + c] = ol[c];
+        }
+        if (LSE_FG) LSE_FG[l] = lf;
+        if (LSE_L) LSE_L[l] = ll;
+      }
+    }
+    free(loc); free(sel); free(x); free(ofg); free(ol);
+  }
+  free(qm); free(km); free(vm); free(ocg);
+  return 0;
+}
+
+/*
+ * Backward of the three-branch form for one unit, selection held constant.  Unlike the union form, gradient
+ * reaches the block-level (routing) scores through the compression branch (the paper's ablation appendix notes
+ * that the routing scores are trained through that branch only).  The rounding of the pooled sums to fp32 is
+ * treated as the identity.  Outputs in token order: dQ, dK, dV [N,d]; dG [N,3] (gradient of the gates).
+ */
+int mo_bwd3_unit(const mo_geom *g, const uint16_t *q, const uint16_t *k, const uint16_t *v, const uint16_t *d_o,
+                 const int32_t *idx, const double *gates, double *dQ, double *dK, double *dV, double *dG) {
+  if (!g_ok(g)) return -1;
+  int m = g_m(g), b = g_b(g), d = g->d;
+  int64_t N = (int64_t)g->nlat * g->nlon;
+  double sc = g_scale(g);
+  int max_att = MO_MAX_LOCAL + g->topk;
+  size_t nd = (size_t)N * d;
+  double *O = (double *)malloc(sizeof(double) * nd), *OCG = (double *)malloc(sizeof(double) * nd);
+  double *OFG = (double *)malloc(sizeof(double) * nd), *OL = (double *)malloc(sizeof(double) * nd);
+  double *LF = (double *)malloc(sizeof(double) * (size_t)N), *LL = (double *)malloc(sizeof(double) * (size_t)N);
+  double *AB = (double *)malloc(sizeof(double) * (size_t)m * m);
+  double *qm = (double *)malloc(sizeof(double) * (size_t)m * d), *km = (double *)malloc(sizeof(double) * (size_t)m * d);
+  double *vm = (double *)malloc(sizeof(double) * (size_t)m * d);
+  double *dob = (double *)calloc((size_t)m * d, sizeof(double));   /* gradient of the block's compression output */
+  double *dqm = (double *)calloc((size_t)m * d, sizeof(double)), *dkm = (double *)calloc((size_t)m * d, sizeof(double));
+  double *dvm = (double *)calloc((size_t)m * d, sizeof(double));
+  if (!O || !OCG || !OFG || !OL || !LF || !LL || !AB || !qm || !km || !vm || !dob || !dqm || !dkm || !dvm) return -2;
+  mo_fwd3_unit(g, q, k, v, idx, gates, O, OCG, OFG, OL, LF, LL, AB);
+  block_means(g, q, qm);
+  block_means(g, k, km);
+  block_means(g, v, vm);
+  /* gates, and the gradient that reaches each block's compression output */
+  for (int i = 0; i < m; ++i)
+    for (int e = 0; e < b; ++e) {
+      int64_t l = block_token(g, i, e);
+      double gc = 0.0, gf = 0.0, gl = 0.0;
+      for (int c = 0; c < d; ++c) {
+        double go = bf16_widen(d_o[l * d + c]);
+        gc += go * OCG[l * d + c];
+        gf += go * OFG[l * d + c];
+        gl += go * OL[l * d + c];
+        dob[(size_t)i * d + c] += gates[l * 3 + 0] * go;
+      }
+      dG[l * 3 + 0] = gc; dG[l * 3 + 1] = gf; dG[l * 3 + 2] = gl;
+    }
+  /* compression branch: softmax attention backward on the block means */
+  for (int i = 0; i < m; ++i) {
+    double Dc = 0.0;
+    for (int c = 0; c < d; ++c) Dc += dob[(size_t)i * d + c] * OCG[block_token(g, i, 0) * d + c];
+    for (int j = 0; j < m; ++j) {
+      double a = AB[(size_t)i * m + j], dp = 0.0;
+      for (int c = 0; c < d; ++c) dp += dob[(size_t)i * d + c] * vm[(size_t)j * d + c];
+      double ds = a * (dp - Dc);
+      for (int c = 0; c < d; ++c) {
+        dvm[(size_t)j * d + c] += a * dob[(size_t)i * d + c];
+        dqm[(size_t)i * d + c] += sc * ds * km[(size_t)j * d + c];
+        dkm[(size_t)j * d + c] += sc * ds * qm[(size_t)i * d + c];
+      }
+    }
+  }
+  /* the mean spreads its gradient evenly over the block's tokens */
+  for (int j = 0; j < m; ++j)
+    for (int e = 0; e < b; ++e) {
+      int64_t t = block_token(g, j, e);
+      for (int c = 0; c < d; ++c) {
+        dQ[t * d + c] = dqm[(size_t)j * d + c] / b;
+        dK[t * d + c] = dkm[(size_t)j * d + c] / b;
+        dV[t * d + c] = dvm[(size_t)j * d + c] / b;
+      }
+    }
+  /* selection (branch 1) and local (branch 2) attention: per query row; dK, dV gathered per key block */
+#pragma omp parallel
+  {
+    int32_t *blk = (int32_t *)malloc(sizeof(int32_t) * (size_t)max_att);
+    double *x = (double *)malloc(sizeof(double) * (size_t)max_att * b);
+#pragma omp for schedule(dynamic, 1)
+    for (int i = 0; i < m; ++i)
+      for (int br = 1; br <= 2; ++br) {
+        int nb = 0;
+        if (br == 1) { for (int r = 0; r < g->topk; ++r) if (idx[(size_t)i * g->topk + r] >= 0) blk[nb++] = idx[(size_t)i * g->topk + r]; }
+        else nb = mo_local_set(g, i, blk);
+        if (nb == 0) continue;
+        const double *OB = br == 1 ? OFG : OL, *LSE = br == 1 ? LF : LL;
+        for (int e = 0; e < b; ++e) {
+          int64_t l = block_token(g, i, e);
+          double gate = gates[l * 3 + br], D = 0.0;
+          for (int c = 0; c < d; ++c) D += gate * bf16_widen(d_o[l * d + c]) * OB[l * d + c];
+          row_logits(g, q, k, l, blk, nb, x);
+          for (int a = 0; a < nb; ++a)
+            for (int e2 = 0; e2 < b; ++e2) {
+              int64_t t = block_token(g, blk[a], e2);
+              double w = exp(x[(size_t)a * b + e2] - LSE[l]), dP = 0.0;
+              for (int c = 0; c < d; ++c) dP += gate * bf16_widen(d_o[l * d + c]) * bf16_widen(v[t * d + c]);
+              double dS = w * (dP - D);
+              for (int c = 0; c < d; ++c) dQ[l * d + c] += sc * dS * bf16_widen(k[t * d + c]);
+            }
+        }
+      }
+    free(blk); free(x);
+  }
+#pragma omp parallel
+  {
+    int32_t *blk = (int32_t *)malloc(sizeof(int32_t) * (size_t)max_att);
+#pragma omp for schedule(dynamic, 1)
+    for (int j = 0; j < m; ++j)
+      for (int i = 0; i < m; ++i)
+        for (int br = 1; br <= 2; ++br) {
+          int nb = 0, connected = 0;
+          if (br == 1) { for (int r = 0; r < g->topk; ++r) if (idx[(size_t)i * g->topk + r] >= 0) blk[nb++] = idx[(size_t)i * g->topk + r]; }
+          else nb = mo_local_set(g, i, blk);
+          for (int a = 0; a < nb; ++a) connected |= (blk[a] == j);
+          if (!connected) continue;
+          const double *OB = br == 1 ? OFG : OL, *LSE = br == 1 ? LF : LL;
+          for (int e = 0; e < b; ++e) {
+            int64_t l = block_token(g, i, e);
+            double gate = gates[l * 3 + br], D = 0.0;
+            for (int c = 0; c < d; ++c) D += gate * bf16_widen(d_o[l * d + c]) * OB[l * d + c];
+            for (int e2 = 0; e2 < b; ++e2) {
+              int64_t t = block_token(g, j, e2);
+              double s = 0.0, dP = 0.0;
+              for (int c = 0; c < d; ++c) {
+                s += bf16_widen(q[l * d + c]) * bf16_widen(k[t * d + c]);
+                dP += gate * bf16_widen(d_o[l * d + c]) * bf16_widen(v[t * d + c]);
+              }
+              double w = exp(sc * s - LSE[l]), dS = w * (dP - D);
+              for (int c = 0; c < d; ++c) {
+                dV[t * d + c] += w * gate * bf16_widen(d_o[l * d + c]);
+                dK[t * d + c] += sc * dS * bf16_widen(q[l * d + c]);
+              }
+            }
+          }
+        }
+    free(blk);
+  }
+  free(O); free(OCG); free(OFG); free(OL); free(LF); free(LL); free(AB); free(qm); free(km); free(vm);
+  free(dob); free(dqm); free(dkm); free(dvm);
   return 0;
 }

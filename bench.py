@@ -355,6 +355,24 @@ def run_ours(args, w):
     torch.cuda.synchronize()
     t_bwd = sum(e[0].elapsed_time(e[1]) for e in evb) / kb
 
+    # the paper's three-branch form of the same workload (compression + selection + local, gated), same selection
+    gates = torch.randn((w.B, w.H, w.N, 3), dtype=torch.float32, device=dev)
+    ws3 = torch.empty(mb.workspace_bytes(p, mb.OP_FWD_BRANCHES), dtype=torch.uint8, device=dev)
+    lse_fg, lse_l = torch.empty_like(lse), torch.empty_like(lse)
+    k3 = min(K, 50)
+    ev3 = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(k3)]
+    for s in range(k3 + 2):
+        flush_buf.zero_()
+        if s >= 2:
+            ev3[s - 2][0].record(stream)
+        mb.mosaic_bsa_fwd_branches(p, dx["q"], dx["k"], dx["v"], idx, gates, o=dq, lse_fg=lse_fg, lse_l=lse_l, ws=ws3)
+        if s >= 2:
+            ev3[s - 2][1].record(stream)
+    torch.cuda.synchronize()
+    mb.check_status(ws3, "three-branch forward")
+    t_br = sum(e[0].elapsed_time(e[1]) for e in ev3) / k3
+    del ws3, gates, lse_fg, lse_l
+
     # end to end: pinned host -> device, step, device -> pinned host
     ke = min(K, 20)
     o_host = torch.empty(o.shape, dtype=torch.int16).pin_memory()
@@ -398,6 +416,7 @@ def run_ours(args, w):
                      "traffic": traffic, "traffic_source": traffic_source, "peak_source": peaks["source"] + " (burst)",
                      "frac_of_nominal_2250": fwd_tflops / NOMINAL_BF16_TFLOPS, "ms": t_fwd},
         "stages": {"select_ms": t_sel, "fwd_ms": t_fwd, "bwd_ms": t_bwd, "ms_layer_fwd": t_step,
+                   "fwd_three_branch_ms": t_br,
                    "fwd_tflops": fwd_tflops, "bwd_tflops": flops.bwd_flops(w) / (t_bwd * 1e-3) / 1e12,
                    "select_pool_gbs_lower_bound": pool_bytes / (t_sel * 1e-3) / 1e9,
                    "pct_of_nominal_peak": 100 * fwd_tflops / NOMINAL_BF16_TFLOPS,

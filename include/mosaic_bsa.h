@@ -58,7 +58,7 @@ typedef struct mosaic_bsa_params {
   uint32_t flags;     /* reserved, must be 0                                           */
 } mosaic_bsa_params;
 
-enum { MOSAIC_OP_SELECT = 0, MOSAIC_OP_FWD = 1, MOSAIC_OP_BWD = 2 };
+enum { MOSAIC_OP_SELECT = 0, MOSAIC_OP_FWD = 1, MOSAIC_OP_BWD = 2, MOSAIC_OP_FWD_BRANCHES = 3 };
 
 enum {
   MOSAIC_OK = 0,
@@ -107,6 +107,29 @@ int mosaic_bsa_select(const mosaic_bsa_params *p, const void *q, const void *k, 
 int mosaic_bsa_fwd(const mosaic_bsa_params *p, const void *q, const void *k, const void *v,
                    const int32_t *block_idx, void *o, float *lse, void *ws, size_t ws_bytes,
                    void *cuda_stream);
+
+/*
+ * Forward in the paper's three-branch form (Eq. of the aggregated output, section "Native Sparse
+ * Attention"; "Compression", "Selection" and "Local Attention" paragraphs of the section
+ * "Block-Sparse Attention"):  for token l of query block i
+ *     o_l = gates[l][0] * oCG_i + gates[l][1] * oFG_l + gates[l][2] * oL_l
+ *   oCG_i  block-level softmax attention over ALL m blocks on the mean-pooled queries, keys and
+ *          values (the same vector for every token of the block),
+ *   oFG_l  softmax attention of q_l over the tokens of the selected blocks of row i of block_idx
+ *          (own normaliser; an empty row gives 0 and a log-sum-exp of -inf),
+ *   oL_l   softmax attention of q_l over the tokens of the local neighbourhood (own normaliser).
+ * The gates are learned functions of the layer input in the paper and therefore inputs here.
+ *   q, k, v    in   [B,H,N,d] bf16
+ *   block_idx  in   [B,H,m,topk] int32, same rules as mosaic_bsa_fwd
+ *   gates      in   [B,H,N,3] fp32, order (compression, selection, local)
+ *   o          out  [B,H,N,d] bf16
+ *   lse_fg, lse_l  out  [B,H,N] fp32, natural-log sum-exp of the selection and local branches
+ * Workspace: mosaic_bsa_workspace_bytes(p, MOSAIC_OP_FWD_BRANCHES) (pooled sums, the block-level output
+ * and the two branch outputs in bf16).
+ */
+int mosaic_bsa_fwd_branches(const mosaic_bsa_params *p, const void *q, const void *k, const void *v,
+                            const int32_t *block_idx, const float *gates, void *o, float *lse_fg,
+                            float *lse_l, void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
  * Backward (gradient of the forward with the selection held constant; dK/dV visit only

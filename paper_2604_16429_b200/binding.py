@@ -17,10 +17,10 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmosaic_bsa.so")
 _lib = None
 
-OP_SELECT, OP_FWD, OP_BWD = 0, 1, 2
+OP_SELECT, OP_FWD, OP_BWD, OP_FWD_BRANCHES = 0, 1, 2, 3
 EXPORTS = ("mosaic_bsa_workspace_bytes", "mosaic_bsa_select", "mosaic_bsa_fwd", "mosaic_bsa_bwd",
            "mosaic_bsa_last_status", "mosaic_bsa_strerror", "mosaic_bsa_select_static",
-           "mosaic_bsa_descriptor_encodes")
+           "mosaic_bsa_descriptor_encodes", "mosaic_bsa_fwd_branches")
 STATIC_SCRATCH_BYTES = 4 << 20
 
 
@@ -88,6 +88,8 @@ def lib():
         L.mosaic_bsa_select_static.argtypes = [pp, vp, vp, i32p, vp]
         L.mosaic_bsa_fwd.restype = ctypes.c_int
         L.mosaic_bsa_fwd.argtypes = [pp, vp, vp, vp, i32p, vp, fp, vp, ctypes.c_size_t, vp]
+        L.mosaic_bsa_fwd_branches.restype = ctypes.c_int
+        L.mosaic_bsa_fwd_branches.argtypes = [pp, vp, vp, vp, i32p, fp, vp, fp, fp, vp, ctypes.c_size_t, vp]
         L.mosaic_bsa_bwd.restype = ctypes.c_int
         L.mosaic_bsa_bwd.argtypes = [pp, vp, vp, vp, vp, fp, vp, i32p, vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.mosaic_bsa_last_status.restype = ctypes.c_int
@@ -172,6 +174,25 @@ def mosaic_bsa_fwd(p: Params, q, k, v, block_idx, o=None, lse=None, ws=None, str
     if rc:
         raise MosaicError(rc, "mosaic_bsa_fwd")
     return o, lse
+
+
+def mosaic_bsa_fwd_branches(p: Params, q, k, v, block_idx, gates, o=None, lse_fg=None, lse_l=None, ws=None, stream=None):
+    """Three-branch form: gated sum of the compression, selection and local branches.  `gates` is
+    [B, H, N, 3] fp32 (compression, selection, local).  Returns (o, lse_fg, lse_l)."""
+    _chk_qkv(p, q, k, v)
+    if gates.dtype != torch.float32 or not gates.is_contiguous() or tuple(gates.shape) != (p.B, p.H, p.N, 3):
+        raise ValueError(f"expected contiguous cuda fp32 gates [{p.B},{p.H},{p.N},3]")
+    o = torch.empty_like(q) if o is None else o
+    lse_fg = torch.empty((p.B, p.H, p.N), dtype=torch.float32, device=q.device) if lse_fg is None else lse_fg
+    lse_l = torch.empty((p.B, p.H, p.N), dtype=torch.float32, device=q.device) if lse_l is None else lse_l
+    if ws is None:
+        ws = alloc_workspace(p, OP_FWD_BRANCHES, q.device)
+    pc = p.c()
+    rc = lib().mosaic_bsa_fwd_branches(ctypes.byref(pc), _ptr(q), _ptr(k), _ptr(v), _ptr(block_idx), _ptr(gates), _ptr(o),
+                                       _ptr(lse_fg), _ptr(lse_l), _ptr(ws), ws.numel(), _stream(stream))
+    if rc:
+        raise MosaicError(rc, "mosaic_bsa_fwd_branches")
+    return o, lse_fg, lse_l
 
 
 def mosaic_bsa_bwd(p: Params, q, k, v, o, lse, d_o, block_idx, dq=None, dk=None, dv=None, ws=None, stream=None):

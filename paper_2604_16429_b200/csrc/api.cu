@@ -32,6 +32,7 @@ int validate(const mosaic_bsa_params* p, Geo* g) {
   g->nbh = p->nlat / p->bh; g->nbw = p->nlon / p->bw; g->m = (int)m;
   g->b = p->bh * p->bw; g->cpb = cpb; g->crows = crows;
   g->rlat = p->rlat; g->rlon = p->rlon; g->topk = p->topk;
+  g->local_off = 0;
   g->scale = p->scale > 0.f ? p->scale : 1.0f / sqrtf((float)p->d);
   g->scale_log2 = g->scale * 1.4426950408889634f;
   g->N = N;
@@ -46,6 +47,21 @@ SelectWs select_layout(const Geo& g) {
   w.nq = w.pk + pooled;
   w.nk = w.nq + norms;
   w.total = w.nk + norms;
+  return w;
+}
+
+BranchWs branch_layout(const Geo& g) {
+  BranchWs w;
+  const size_t pooled = align256(sizeof(float) * (size_t)g.U * g.m * kD), norms = align256(sizeof(float) * (size_t)g.U * g.m);
+  const size_t full = align256(2 * (size_t)g.U * g.N * kD);
+  w.pq = kStatusBytes;
+  w.pk = w.pq + pooled;
+  w.pv = w.pk + pooled;
+  w.nrm = w.pv + pooled;
+  w.ocg = w.nrm + 2 * norms;
+  w.ofg = w.ocg + pooled;
+  w.ol = w.ofg + full;
+  w.total = w.ol + full;
   return w;
 }
 
@@ -105,6 +121,7 @@ size_t mosaic_bsa_workspace_bytes(const mosaic_bsa_params* p, int op) {
     case MOSAIC_OP_SELECT: return select_total(g);
     case MOSAIC_OP_FWD: return kStatusBytes;
     case MOSAIC_OP_BWD: return bwd_layout(g).total;
+    case MOSAIC_OP_FWD_BRANCHES: return branch_layout(g).total;
     default: return 0;
   }
 }
@@ -135,7 +152,41 @@ int mosaic_bsa_fwd(const mosaic_bsa_params* p, const void* q, const void* k, con
       !aligned(block_idx, 4))
     return MOSAIC_E_MISALIGNED;
   if ((rc = begin(p, ws, ws_bytes, kStatusBytes, cuda_stream, &c))) return rc;
-  return launch_fwd_tc(c, q, k, v, block_idx, o, lse);
+  return launch_fwd_tc(c, q, k, v, block_idx, o, lse, c.status + 1);
+}
+
+int mosaic_bsa_fwd_branches(const mosaic_bsa_params* p, const void* q, const void* k, const void* v,
+                            const int32_t* block_idx, const float* gates, void* o, float* lse_fg, float* lse_l, void* ws,
+                            size_t ws_bytes, void* cuda_stream) {
+  HostCtx c;
+  Geo g;
+  int rc = validate(p, &g);
+  if (rc) return rc;
+  if (!q || !k || !v || !gates || !o || !lse_fg || !lse_l || (!block_idx && g.topk > 0)) return MOSAIC_E_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(o, 16) || !aligned(gates, 4) ||
+      !aligned(lse_fg, 4) || !aligned(lse_l, 4) || !aligned(block_idx, 4))
+    return MOSAIC_E_MISALIGNED;
+  const BranchWs w = branch_layout(g);
+  if ((rc = begin(p, ws, ws_bytes, w.total, cuda_stream, &c))) return rc;
+  char* base = (char*)ws;
+  float *pq = (float*)(base + w.pq), *pk = (float*)(base + w.pk), *pv = (float*)(base + w.pv);
+  float *nrm = (float*)(base + w.nrm), *ocg = (float*)(base + w.ocg);
+  void *ofg = base + w.ofg, *ol = base + w.ol;
+  // compression branch: pooled sums of Q, K (with their norms, unused here) and V, then block-level attention
+  HostCtx cp = c;
+  cp.g.topk = 0;  // pooling only
+  if ((rc = launch_select(cp, q, k, nullptr, pq, pk, nrm, nrm + (size_t)g.U * g.m))) return rc;
+  if ((rc = launch_pool_one(c, v, pv, nrm))) return rc;
+  if ((rc = launch_compress(c, pq, pk, pv, ocg))) return rc;
+  // local branch: the neighbourhood only (no selected blocks); work queue in the second word of the status block
+  HostCtx cl = c;
+  cl.g.topk = 0;
+  if ((rc = launch_fwd_tc(cl, q, k, v, nullptr, ol, lse_l, c.status + 1))) return rc;
+  // selection branch: the selected blocks only; work queue in the third word
+  HostCtx cs = c;
+  cs.g.local_off = 1;
+  if ((rc = launch_fwd_tc(cs, q, k, v, block_idx, ofg, lse_fg, c.status + 2))) return rc;
+  return launch_combine(c, ocg, ofg, ol, gates, o);
 }
 
 int mosaic_bsa_bwd(const mosaic_bsa_params* p, const void* q, const void* k, const void* v, const void* o,

@@ -23,6 +23,7 @@ struct Geo {
   int cpb;          // 64-token chunks per block (b / 64)
   int crows;        // grid rows per chunk (64 / bw)
   int rlat, rlon, topk;
+  int local_off;    // 1: the local neighbourhood is not attended (selection branch of the three-branch form)
   float scale;      // softmax scale
   float scale_log2; // scale * log2(e)
   long long N;      // tokens per unit
@@ -89,7 +90,13 @@ SelectWs select_layout(const Geo& g);
 int launch_select(const HostCtx& c, const void* q, const void* k, int32_t* block_idx, float* pooled_q,
                   float* pooled_k, float* norm_q, float* norm_k);
 int launch_fwd_tc(const HostCtx& c, const void* q, const void* k, const void* v, const int32_t* block_idx,
-                  void* o, float* lse);
+                  void* o, float* lse, int* work_counter);
+// Layout of the three-branch forward's scratch behind the status block
+struct BranchWs { size_t pq, pk, pv, nrm, ocg, ofg, ol, total; };
+BranchWs branch_layout(const Geo& g);
+int launch_pool_one(const HostCtx& c, const void* x, float* pooled, float* norm_scratch);
+int launch_compress(const HostCtx& c, const float* pooled_q, const float* pooled_k, const float* pooled_v, float* ocg);
+int launch_combine(const HostCtx& c, const float* ocg, const void* o_fg, const void* o_l, const float* gates, void* o);
 int launch_dq_tc(const HostCtx& c, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
                  const float* D, const int32_t* block_idx, void* dq, int* work_counter);
 int launch_dkdv_tc(const HostCtx& c, const void* q, const void* k, const void* v, const void* d_o,

@@ -405,7 +405,7 @@ __global__ void __launch_bounds__(kThreads, 1)
           const int e = tid & 63;
           const long long tok =
               (long long)sm.info[buf].unit * g.N + chunk_token(g, sm.info[buf].hb[h], sm.info[buf].hc[h], e);
-          const float inv = 1.f / l;
+          const float inv = l > 0.f ? 1.f / l : 0.f;  // a row that attends nothing (empty selection): O = 0
           uint4* dst = reinterpret_cast<uint4*>(o + tok * kD);
 #pragma unroll
           for (int part = 0; part < 2; ++part) {
@@ -420,8 +420,16 @@ __global__ void __launch_bounds__(kThreads, 1)
             for (int i = 0; i < 4; ++i)
               dst[part * 4 + i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
           }
-          lse[tok] = (m_ref + log2f(l)) * 0.6931471805599453f;
+          lse[tok] = l > 0.f ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
         }
+      } else if ((sm.info[buf].hvalid >> h) & 1) {
+        // the tile attends nothing in this item (selection branch with empty rows): O = 0, log-sum-exp = -inf
+        const long long tok =
+            (long long)sm.info[buf].unit * g.N + chunk_token(g, sm.info[buf].hb[h], sm.info[buf].hc[h], tid & 63);
+        uint4* dst = reinterpret_cast<uint4*>(o + tok * kD);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) dst[i] = make_uint4(0u, 0u, 0u, 0u);
+        lse[tok] = -INFINITY;
       }
       tc_fence_before();
       __syncwarp();
@@ -439,8 +447,9 @@ __global__ void __launch_bounds__(kThreads, 1)
 }
 
 // ---------------------------------------------------------------------------------------------
+// `work_counter` must be zero when the kernel starts (a word of the workspace status block).
 int launch_fwd_tc(const HostCtx& c, const void* q, const void* k, const void* v, const int32_t* block_idx, void* o,
-                  float* lse) {
+                  float* lse, int* work_counter) {
   const Geo& g = c.g;
   CUtensorMap mq, mk, mv;
   if (!make_map(&mq, q, g) || !make_map(&mk, k, g) || !make_map(&mv, v, g)) return MOSAIC_E_CUDA;
@@ -452,9 +461,8 @@ int launch_fwd_tc(const HostCtx& c, const void* q, const void* k, const void* v,
   const long long total = (long long)g.U * ipu;
   if (total > 0x7fffff00ll) return MOSAIC_E_UNSUPPORTED;
   const long long grid = total < (long long)sms ? total : (long long)sms;
-  // the work counter is the second word of the status block, zeroed with it when the op starts
   fwd_tc_kernel<<<(unsigned)grid, kThreads, smem, c.stream>>>(g, mq, mk, mv, block_idx, (__nv_bfloat16*)o, lse,
-                                                             c.status, c.status + 1, ipu, (int)total);
+                                                             c.status, work_counter, ipu, (int)total);
   return cudaGetLastError() == cudaSuccess ? MOSAIC_OK : MOSAIC_E_CUDA;
 }
 

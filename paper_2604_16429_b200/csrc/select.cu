@@ -23,11 +23,11 @@ namespace mosaic {
 template <int BW>
 __global__ void __launch_bounds__(256) pool_kernel(Geo g, const uint4* __restrict__ q, const uint4* __restrict__ k,
                                                    float* __restrict__ pq, float* __restrict__ pk,
-                                                   float* __restrict__ nq, float* __restrict__ nk) {
+                                                   float* __restrict__ nq, float* __restrict__ nk, int ntens) {
   const int sub = threadIdx.x & 7;  // which 8 channels
   const long long grp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 3;
   const long long per_tensor = (long long)g.U * g.m;
-  const bool live = grp < 2 * per_tensor;  // the last warp may be partly idle; it still takes part in the shuffles
+  const bool live = grp < ntens * per_tensor;  // the last warp may be partly idle; it still takes part in the shuffles
   const int which = live && grp >= per_tensor;
   const long long w = live ? grp - which * per_tensor : 0;
   const int u = (int)(w / g.m), j = (int)(w - (long long)u * g.m);
@@ -487,6 +487,20 @@ int launch_topk(const HostCtx& c, const float* pooled_q, const float* pooled_k, 
   return cudaGetLastError() == cudaSuccess ? MOSAIC_OK : MOSAIC_E_CUDA;
 }
 
+// block sums of one more tensor (the values, for the compression branch of the three-branch form)
+int launch_pool_one(const HostCtx& c, const void* x, float* pooled, float* norm_scratch) {
+  const Geo& g = c.g;
+  const long long threads = 1ll * g.U * g.m * 8;
+  const unsigned blocks = (unsigned)((threads + 255) / 256);
+  if (g.bw == 8)
+    pool_kernel<8><<<blocks, 256, 0, c.stream>>>(g, (const uint4*)x, (const uint4*)x, pooled, pooled, norm_scratch,
+                                                 norm_scratch, 1);
+  else
+    pool_kernel<16><<<blocks, 256, 0, c.stream>>>(g, (const uint4*)x, (const uint4*)x, pooled, pooled, norm_scratch,
+                                                  norm_scratch, 1);
+  return cudaGetLastError() == cudaSuccess ? MOSAIC_OK : MOSAIC_E_CUDA;
+}
+
 int launch_select(const HostCtx& c, const void* q, const void* k, int32_t* block_idx, float* pooled_q,
                   float* pooled_k, float* norm_q, float* norm_k) {
   const Geo& g = c.g;
@@ -495,10 +509,10 @@ int launch_select(const HostCtx& c, const void* q, const void* k, int32_t* block
     const unsigned blocks = (unsigned)((threads + 255) / 256);
     if (g.bw == 8)
       pool_kernel<8><<<blocks, 256, 0, c.stream>>>(g, (const uint4*)q, (const uint4*)k, pooled_q, pooled_k, norm_q,
-                                                   norm_k);
+                                                   norm_k, 2);
     else
       pool_kernel<16><<<blocks, 256, 0, c.stream>>>(g, (const uint4*)q, (const uint4*)k, pooled_q, pooled_k, norm_q,
-                                                    norm_k);
+                                                    norm_k, 2);
     if (cudaGetLastError() != cudaSuccess) return MOSAIC_E_CUDA;
   }
   if (g.topk > 0) {

@@ -299,7 +299,7 @@ __host__ __device__ inline int items_per_unit(const Geo& g) {
 // ids[n0..); returns the new count.  `j` is this lane's entry of the block's row of block_idx (-1 beyond top-k).
 __device__ __forceinline__ int warp_attended(const Geo& g, int j, int i, int* ids, int n0, int lane, int* status) {
   const int by = i / g.nbw, bx = i - by * g.nbw;
-  const int wl = 2 * g.rlon + 1, nl = (2 * g.rlat + 1) * wl;
+  const int wl = 2 * g.rlon + 1, nl = g.local_off ? 0 : (2 * g.rlat + 1) * wl;
   int id = -1 - lane;
   if (lane < nl) {
     const int dy = lane / wl - g.rlat, dx = lane - (lane / wl) * wl - g.rlon;

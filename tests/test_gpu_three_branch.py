@@ -1,0 +1,103 @@
+"""GPU parity of the three-branch form (compression + selection + local, gated) against the oracle's
+`fwd3`, element by element, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2604_16429_b200 import binding as mb
+from paper_2604_16429_b200 import synth
+from tests import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(w, x, idx, gates, scale=0.0):
+    p = mb.Params.from_workload(w, scale=scale)
+    dx = G.device_inputs(x)
+    ws = G.Guarded((mb.workspace_bytes(p, mb.OP_FWD_BRANCHES),), torch.uint8)
+    o = G.Guarded(tuple(dx["q"].shape), torch.bfloat16, fill=float("nan"))
+    lf = G.Guarded((w.B, w.H, w.N), torch.float32, fill=float("nan"))
+    ll = G.Guarded((w.B, w.H, w.N), torch.float32, fill=float("nan"))
+    gt = torch.from_numpy(gates.astype(np.float32)).cuda().contiguous()
+    mb.mosaic_bsa_fwd_branches(p, dx["q"], dx["k"], dx["v"], idx, gt, o=o.t, lse_fg=lf.t, lse_l=ll.t, ws=ws.t)
+    mb.check_status(ws.t, "fwd_branches")
+    for b_, n_ in ((ws, "workspace"), (o, "o"), (lf, "lse_fg"), (ll, "lse_l")):
+        b_.check(n_)
+    return o.t.float().cpu().numpy().astype(np.float64), lf.t.cpu().numpy().astype(np.float64), ll.t.cpu().numpy().astype(np.float64)
+
+
+def _compare(w, x, idx_h, gates, got, scale=0.0):
+    o, lf, ll = got
+    g = G.geom_of(w, scale)
+    for b in range(w.B):
+        for h in range(w.H):
+            r = oracle.fwd3(g, x["q"][b, h], x["k"][b, h], x["v"][b, h], idx_h[b, h], gates[b, h].astype(np.float32).astype(np.float64))
+            assert np.isfinite(o[b, h]).all(), "unwritten or non-finite output"
+            bound = G.FWD_MAX_ABS * np.maximum(1.0, np.abs(gates[b, h]).sum(axis=1, keepdims=True))
+            err = np.abs(o[b, h] - r["o"])
+            assert (err <= bound).all(), f"o max-abs {err.max():.4g} (unit {b},{h})"
+            assert err.mean() <= G.FWD_MEAN_ABS * max(1.0, np.abs(gates[b, h]).sum(axis=1).mean())
+            for name, got_l in (("lse_fg", lf[b, h]), ("lse_l", ll[b, h])):
+                inf = np.isneginf(r[name])
+                assert np.array_equal(inf, np.isneginf(got_l)), name
+                assert inf.all() or np.abs(got_l[~inf] - r[name][~inf]).max() <= G.LSE_ABS, name
+
+
+CASES = [
+    (synth.WORKLOADS["c1_tiny"], 0.0),
+    (synth.small_case(40, 56, 8, 8, 5, B=1, H=2, kind="smooth", seed=81), 0.0),      # odd block grid
+    (synth.small_case(32, 64, 16, 16, 3, B=1, H=1, kind="smooth", seed=82), 0.0),    # 16x16 blocks
+    (synth.small_case(136, 160, 8, 8, 8, B=1, H=1, kind="smooth", seed=83), 0.2),    # m = 340: several key chunks in the compression kernel
+]
+
+
+@pytest.mark.parametrize("w,scale", CASES, ids=lambda a: a.name if hasattr(a, "name") else str(a))
+def test_three_branch_forward_matches_oracle(w, scale):
+    x = synth.make_inputs(w)
+    idx = G.gpu_select(w, G.device_inputs(x))
+    rng = np.random.default_rng(w.cfg)
+    gates = rng.standard_normal((w.B, w.H, w.N, 3))
+    _compare(w, x, idx.cpu().numpy(), gates, _run(w, x, idx, gates, scale), scale)
+
+
+def test_each_branch_alone_and_empty_selection_rows():
+    w = synth.small_case(32, 64, 8, 8, 4, B=1, H=1, seed=84)
+    x = synth.make_inputs(w)
+    idx = G.gpu_select(w, G.device_inputs(x))
+    idx[0, 0, 5, :] = -1                                   # a query block that selects nothing
+    idx[0, 0, 6, 1:] = -1
+    idx_h = idx.cpu().numpy()
+    for col in range(3):
+        gates = np.zeros((1, 1, w.N, 3)); gates[..., col] = 1.0
+        got = _run(w, x, idx, gates)
+        _compare(w, x, idx_h, gates, got)
+    tok5 = oracle.block_tokens(G.geom_of(w), 5)
+    assert np.all(got[0][0, 0][tok5] != 0)                  # local branch of block 5 is alive ...
+    gates = np.zeros((1, 1, w.N, 3)); gates[..., 1] = 1.0
+    o, lf, _ = _run(w, x, idx, gates)
+    assert np.all(o[0, 0][tok5] == 0) and np.all(np.isneginf(lf[0, 0][tok5]))   # ... its selection branch is empty
+
+
+def test_three_branch_without_selection():
+    w = synth.small_case(48, 64, 8, 8, 0, B=1, H=2, seed=85)
+    x = synth.make_inputs(w)
+    idx = torch.zeros((w.B, w.H, w.m, 0), dtype=torch.int32, device="cuda")
+    gates = np.random.default_rng(85).standard_normal((w.B, w.H, w.N, 3))
+    _compare(w, x, idx.cpu().numpy(), gates, _run(w, x, idx, gates))
+
+
+def test_three_branch_at_the_1p5_degree_size_sampled_units():
+    w = synth.WORKLOADS["c2_1p5deg"]
+    x = synth.make_inputs(w)
+    idx = G.gpu_select(w, G.device_inputs(x))
+    gates = np.random.default_rng(86).standard_normal((w.B, w.H, w.N, 3))
+    o, lf, ll = _run(w, x, idx, gates)
+    assert np.isfinite(o).all()
+    g = G.geom_of(w)
+    idx_h = idx.cpu().numpy()
+    for h in (0, 5):
+        r = oracle.fwd3(g, x["q"][0, h], x["k"][0, h], x["v"][0, h], idx_h[0, h], gates[0, h].astype(np.float32).astype(np.float64))
+        bound = G.FWD_MAX_ABS * np.maximum(1.0, np.abs(gates[0, h]).sum(axis=1, keepdims=True))
+        assert (np.abs(o[0, h] - r["o"]) <= bound).all()
+        assert np.abs(lf[0, h] - r["lse_fg"]).max() <= G.LSE_ABS and np.abs(ll[0, h] - r["lse_l"]).max() <= G.LSE_ABS

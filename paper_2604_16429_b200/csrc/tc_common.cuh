@@ -14,7 +14,11 @@ namespace {
 constexpr int kTile = 8192;                      // bytes of one 64 x 64 bf16 chunk
 constexpr int kMaxUnion = 4 * kMaxList;          // most entries of an item's merged key list
 constexpr int kLists = 4;                        // key lists in flight (the planner runs this far ahead)
+#ifdef MOSAIC_TEST_SPIN_CYCLES                   // test build only: a short bound, so that a wait that nothing ends runs out quickly
+constexpr long long kSpinCycles = MOSAIC_TEST_SPIN_CYCLES;
+#else
 constexpr long long kSpinCycles = 4000000000ll;  // bound of a single wait (~2 s)
+#endif
 constexpr uint32_t kSuspendHintNs = 20000;       // longest park of one mbarrier poll
 
 struct ItemInfo {
@@ -512,6 +516,9 @@ __device__ __forceinline__ void planner_loop(SM& sm, const Geo& g, const int32_t
       for (int h = 0; h < 4; ++h) { inf.hb[h] = hb[h]; inf.hc[h] = hc[h]; }
     }
     __syncwarp();
+#ifdef MOSAIC_TEST_WITHHOLD_FIRST_LIST  // test build only: the CTA's first list is never published, so every consumer's wait runs out
+    if (it == 0) continue;
+#endif
     if (lane == 0) mbar_arrive(s32(&sm.list_full[buf]));
   }
 }

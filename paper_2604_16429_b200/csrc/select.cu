@@ -114,16 +114,15 @@ __device__ __forceinline__ float from_ordered_bits(unsigned o) {
   return __uint_as_float((o >> 31) ? (o & 0x7fffffffu) : ~o);
 }
 
-constexpr int kJT = 128;        // keys per chunk
 constexpr int kKStr = kD + 4;   // padded row of the staged vectors (floats): 16-byte reads of one row per lane hit every bank once
 constexpr int kExact = 64;      // most survivors of a row that the counting rank handles (more: insertion path)
 
-template <int NW, int RI, int CAP>
+template <int NW, int RI, int CAP, int JT>
 struct TopkSmem {
   union {
     struct {
-      float ks[2][kJT][kKStr];  // pooled keys of two chunks (one being read, one in flight)
-      float nk[2][kJT];         // their norm bounds
+      float ks[2][JT][kKStr];  // pooled keys of two chunks (one being read, one in flight)
+      float nk[2][JT];         // their norm bounds
     } scr;
     unsigned long long ekey[NW * RI][kExact];  // exact phase: score keys of the rows' survivors
   };
@@ -190,14 +189,14 @@ __device__ __forceinline__ unsigned long long exact_key(const float* qrow, const
   return score_key(s);
 }
 
-template <int NW, int RI, int CAP>
+template <int NW, int RI, int CAP, int JT>
 __global__ void __launch_bounds__(NW * 32) topk_kernel(Geo g, const float* __restrict__ pq,
                                                        const float* __restrict__ pk, const float* __restrict__ nq,
                                                        const float* __restrict__ nk, int32_t* __restrict__ block_idx) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  using SM = TopkSmem<NW, RI, CAP>;
+  using SM = TopkSmem<NW, RI, CAP, JT>;
   SM& sm = *reinterpret_cast<SM*>(smem_raw);
-  constexpr int TI = NW * RI, NT = NW * 32;
+  constexpr int TI = NW * RI, NT = NW * 32, KB = JT / 32;  // KB: keys of a chunk per lane
   const float kInf = __int_as_float(0x7f800000);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int tiles = (g.m + TI - 1) / TI;
@@ -205,16 +204,16 @@ __global__ void __launch_bounds__(NW * 32) topk_kernel(Geo g, const float* __res
   const float* pq_u = pq + (long long)u * g.m * kD;
   const float* pk_u = pk + (long long)u * g.m * kD;
   const float* nk_u = nk + (long long)u * g.m;
-  const int nchunks = (g.m + kJT - 1) / kJT;
+  const int nchunks = (g.m + JT - 1) / JT;
 
   auto load_chunk = [&](int ch, int buf) {
-    const int j0 = ch * kJT;
-    for (int e = tid; e < kJT * (kD / 4); e += NT) {
+    const int j0 = ch * JT;
+    for (int e = tid; e < JT * (kD / 4); e += NT) {
       const int jj = e / (kD / 4), c4 = e - jj * (kD / 4);
       const bool valid = j0 + jj < g.m;
       cp_async16(&sm.scr.ks[buf][jj][4 * c4], pk_u + (long long)(valid ? j0 + jj : 0) * kD + 4 * c4, valid);
     }
-    for (int jj = tid; jj < kJT; jj += NT) {
+    for (int jj = tid; jj < JT; jj += NT) {
       const bool valid = j0 + jj < g.m;
       cp_async4(&sm.scr.nk[buf][jj], nk_u + (valid ? j0 + jj : 0), valid);
     }
@@ -222,7 +221,7 @@ __global__ void __launch_bounds__(NW * 32) topk_kernel(Geo g, const float* __res
   };
   // visiting order: the chunk that holds the middle of this CTA's rows, then alternately the next one above and
   // below (every chunk once).  seq_next() hands out that sequence.
-  const int c_home = min((i0 + TI / 2) / kJT, nchunks - 1);
+  const int c_home = min((i0 + TI / 2) / JT, nchunks - 1);
   int seq_lo = c_home - 1, seq_hi = c_home + 1, seq_n = 0;
   auto seq_next = [&]() {
     int c;
@@ -310,22 +309,22 @@ __global__ void __launch_bounds__(NW * 32) topk_kernel(Geo g, const float* __res
       asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
     __syncthreads();
-    const int j0 = ch * kJT;
-    float acc[RI][4];
+    const int j0 = ch * JT;
+    float acc[RI][KB];
 #pragma unroll
     for (int a = 0; a < RI; ++a)
 #pragma unroll
-      for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+      for (int b = 0; b < KB; ++b) acc[a][b] = 0.f;
 #pragma unroll 4
     for (int c4 = 0; c4 < kD / 4; ++c4) {
-      float4 kv[4];
+      float4 kv[KB];
 #pragma unroll
-      for (int b = 0; b < 4; ++b) kv[b] = *reinterpret_cast<const float4*>(&sm.scr.ks[buf][lane + 32 * b][4 * c4]);
+      for (int b = 0; b < KB; ++b) kv[b] = *reinterpret_cast<const float4*>(&sm.scr.ks[buf][lane + 32 * b][4 * c4]);
 #pragma unroll
       for (int a = 0; a < RI; ++a) {
         const float4 qv = *reinterpret_cast<const float4*>(&sm.qs[warp * RI + a][4 * c4]);
 #pragma unroll
-        for (int b = 0; b < 4; ++b) {
+        for (int b = 0; b < KB; ++b) {
           acc[a][b] = fmaf(qv.x, kv[b].x, acc[a][b]);
           acc[a][b] = fmaf(qv.y, kv[b].y, acc[a][b]);
           acc[a][b] = fmaf(qv.z, kv[b].z, acc[a][b]);
@@ -333,10 +332,10 @@ __global__ void __launch_bounds__(NW * 32) topk_kernel(Geo g, const float* __res
         }
       }
     }
-    int jy[4], jx[4];
-    float nkv[4];
+    int jy[KB], jx[KB];
+    float nkv[KB];
 #pragma unroll
-    for (int b = 0; b < 4; ++b) {
+    for (int b = 0; b < KB; ++b) {
       const int j = min(j0 + lane + 32 * b, g.m - 1);
       jy[b] = j / g.nbw;
       jx[b] = j - jy[b] * g.nbw;
@@ -348,7 +347,7 @@ __global__ void __launch_bounds__(NW * 32) topk_kernel(Geo g, const float* __res
       const bool row_ok = i0 + warp * RI + a < g.m;  // warp-uniform
       const int row = warp * RI + a;
 #pragma unroll
-      for (int b = 0; b < 4; ++b) {
+      for (int b = 0; b < KB; ++b) {
         const int j = j0 + lane + 32 * b;
         int dx = jx[b] - ix[a];
         dx += dx < 0 ? g.nbw : 0;  // (jx - ix) mod nbw
@@ -466,23 +465,23 @@ __global__ void __launch_bounds__(NW * 32) topk_kernel(Geo g, const float* __res
   }
 }
 
-template <int NW, int RI, int CAP>
+template <int NW, int RI, int CAP, int JT>
 int launch_topk(const HostCtx& c, const float* pooled_q, const float* pooled_k, const float* norm_q,
                 const float* norm_k, int32_t* block_idx) {
   const Geo& g = c.g;
-  const size_t smem = sizeof(TopkSmem<NW, RI, CAP>);
+  const size_t smem = sizeof(TopkSmem<NW, RI, CAP, JT>);
   static unsigned long long configured = 0;  // devices on which the kernel's shared-memory opt-in is set
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return MOSAIC_E_CUDA;
   if (dev < 0 || dev >= 64) return MOSAIC_E_UNSUPPORTED;
   if (!((configured >> dev) & 1ull)) {
-    if (cudaFuncSetAttribute(topk_kernel<NW, RI, CAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+    if (cudaFuncSetAttribute(topk_kernel<NW, RI, CAP, JT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
         cudaSuccess)
       return MOSAIC_E_CUDA;
     configured |= 1ull << dev;
   }
   const int tiles = (g.m + NW * RI - 1) / (NW * RI);
-  topk_kernel<NW, RI, CAP><<<(unsigned)(g.U * tiles), NW * 32, smem, c.stream>>>(g, pooled_q, pooled_k, norm_q,
+  topk_kernel<NW, RI, CAP, JT><<<(unsigned)(g.U * tiles), NW * 32, smem, c.stream>>>(g, pooled_q, pooled_k, norm_q,
                                                                                 norm_k, block_idx);
   return cudaGetLastError() == cudaSuccess ? MOSAIC_OK : MOSAIC_E_CUDA;
 }
@@ -516,11 +515,13 @@ int launch_select(const HostCtx& c, const void* q, const void* k, int32_t* block
     if (cudaGetLastError() != cudaSuccess) return MOSAIC_E_CUDA;
   }
   if (g.topk > 0) {
-    // the most query blocks per CTA (64, 32, 16) that still gives every SM about two CTAs; 16 otherwise
+    // the most query blocks per CTA (64, 32, 16) that still gives every SM about two CTAs; small problems are
+    // latency-bound and take 8 rows per CTA and 64-key chunks, so that more warps are resident
     auto ctas = [&](int ti) { return (long long)g.U * ((g.m + ti - 1) / ti); };
-    const int rc = ctas(64) >= 296 ? launch_topk<8, 8, 128>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx)
-                 : ctas(32) >= 296 ? launch_topk<4, 8, 128>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx)
-                                   : launch_topk<4, 4, 192>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx);
+    const int rc = ctas(64) >= 296   ? launch_topk<8, 8, 128, 128>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx)
+                   : ctas(32) >= 296 ? launch_topk<4, 8, 128, 128>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx)
+                   : ctas(16) >= 296 ? launch_topk<4, 4, 192, 128>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx)
+                                     : launch_topk<4, 2, 96, 64>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx);
     if (rc) return rc;
   }
   return MOSAIC_OK;

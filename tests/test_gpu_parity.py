@@ -23,6 +23,7 @@ SELECT_CASES = [
     synth.small_case(48, 64, 8, 8, 0, B=1, H=1, seed=26, rlat=0, rlon=0),       # nothing selected
     synth.small_case(240, 320, 8, 8, 8, B=1, H=8, kind="smooth", seed=28),      # m = 1200, 8 units: the 32-rows-per-CTA ranking path
     synth.small_case(32, 64, 8, 16, 3, B=1, H=1, kind="smooth", seed=29),       # 8 x 16 blocks
+    synth.small_case(240, 320, 8, 8, 8, B=1, H=5, kind="smooth", seed=30),      # m = 1200, 5 units: the 16-rows-per-CTA ranking path
 ]
 
 

@@ -131,7 +131,8 @@ class ClockSampler:
 
 def describe(w) -> str:
     return (f"{w.name}: {w.nlat}x{w.nlon} grid, {w.bh}x{w.bw} blocks (m={w.m}), B={w.B}, H={w.H}, d={w.d}, "
-            f"local {2 * w.rlat + 1}x{2 * w.rlon + 1}, top-k {w.topk}, {w.kind} bf16 inputs")
+            + (f"local groups of {w.rlat}x{w.rlon} blocks" if w.local_groups else f"local {2 * w.rlat + 1}x{2 * w.rlon + 1}")
+            + f", top-k {w.topk}, {w.kind} bf16 inputs")
 
 
 # ------------------------------------------------------------------------------------------
@@ -157,7 +158,7 @@ def cpu_baseline(w, x, idx_gpu, o_gpu, lse_gpu) -> dict:
     import oracle
     from oracle import Geom
     oracle.build()
-    g = Geom(w.nlat, w.nlon, d=w.d, bh=w.bh, bw=w.bw, rlat=w.rlat, rlon=w.rlon, topk=w.topk)
+    g = Geom(w.nlat, w.nlon, d=w.d, bh=w.bh, bw=w.bw, rlat=w.rlat, rlon=w.rlon, topk=w.topk, local_groups=w.local_groups)
     rng = np.random.default_rng(0)
     if w.b <= 64:
         units = [(u // w.H, u % w.H) for u in range(min(40, w.U))]
@@ -193,7 +194,7 @@ def run_reference(args, w):
     import oracle
     from oracle import Geom
     oracle.build()
-    g = Geom(w.nlat, w.nlon, d=w.d, bh=w.bh, bw=w.bw, rlat=w.rlat, rlon=w.rlon, topk=w.topk)
+    g = Geom(w.nlat, w.nlon, d=w.d, bh=w.bh, bw=w.bw, rlat=w.rlat, rlon=w.rlon, topk=w.topk, local_groups=w.local_groups)
     one = synth.Workload(**{**w.__dict__, "B": 1, "H": 1})
     x = synth.make_inputs(one, with_do=False)
     rng = np.random.default_rng(0)

@@ -33,7 +33,8 @@
  *     in the first word of the workspace, skips the offending work and returns; read it
  *     with mosaic_bsa_last_status().
  *   - Supported in this version: d = 64; bw = 8 or 16 with bh a multiple of 64/bw
- *     (8x8 and 16x16 are the tested shapes); rlat, rlon in 0..2; (local blocks + topk)
+ *     (8x8, 16x16 and 8x16 are the tested shapes); rlat, rlon in 0..2 (group mode: rlat*rlon
+ *     <= 32); (local blocks + topk)
  *     <= 64; topk <= 32; any B, H and any grid with nlat % bh == 0, nlon % bw == 0
  *     (grids with fewer than 2*rlon+1 block columns de-duplicate the neighbourhood).
  */
@@ -52,11 +53,19 @@ typedef struct mosaic_bsa_params {
   int32_t nlat, nlon; /* grid; N = nlat*nlon                                           */
   int32_t d;          /* head dimension (64)                                           */
   int32_t bh, bw;     /* block shape in grid points                                    */
-  int32_t rlat, rlon; /* local neighbourhood radius in blocks (1,1 = 3x3)              */
+  int32_t rlat, rlon; /* local neighbourhood radius in blocks (1,1 = 3x3); with
+                         MOSAIC_FLAG_LOCAL_GROUPS: height and width of the local group    */
   int32_t topk;       /* selected non-local blocks per query block, >= 0               */
   float scale;        /* softmax scale; <= 0 means 1/sqrt(d)                           */
-  uint32_t flags;     /* reserved, must be 0                                           */
+  uint32_t flags;     /* 0 or MOSAIC_FLAG_LOCAL_GROUPS                                 */
 } mosaic_bsa_params;
+
+/* Local attention inside aligned groups of blocks instead of a sliding neighbourhood (the paper's "Local
+ * Attention" paragraph: dense attention inside large blocks, computed independently): the local set of a block
+ * is the aligned tile of rlat x rlon blocks that contains it (rlat, rlon >= 1, rlat*rlon <= 32; the last group
+ * of a row or column may be ragged).  The paper's HEALPix layout -- 128 contiguous tokens per block, local
+ * blocks of 1024 tokens -- is nlat = N/16, nlon = 16, bh = 8, bw = 16, rlat = 8, rlon = 1 with this flag. */
+#define MOSAIC_FLAG_LOCAL_GROUPS 1u
 
 enum { MOSAIC_OP_SELECT = 0, MOSAIC_OP_FWD = 1, MOSAIC_OP_BWD = 2, MOSAIC_OP_FWD_BRANCHES = 3 };
 

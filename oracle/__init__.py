@@ -38,6 +38,7 @@ class _Geom(ctypes.Structure):
         ("rlat", ctypes.c_int32), ("rlon", ctypes.c_int32),
         ("topk", ctypes.c_int32),
         ("scale", ctypes.c_double),
+        ("local_groups", ctypes.c_int32),
     ]
 
 
@@ -52,6 +53,7 @@ class Geom:
     rlon: int = 1
     topk: int = 0
     scale: float = 0.0
+    local_groups: bool = False
 
     @property
     def N(self): return self.nlat * self.nlon
@@ -66,7 +68,7 @@ class Geom:
 
     def c(self):
         return _Geom(self.nlat, self.nlon, self.d, self.bh, self.bw, self.rlat, self.rlon,
-                     self.topk, float(self.scale))
+                     self.topk, float(self.scale), int(self.local_groups))
 
 
 def _load():

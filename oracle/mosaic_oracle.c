@@ -55,6 +55,9 @@ typedef struct mo_geom {
   int32_t rlat, rlon;
   int32_t topk;
   double scale; /* softmax scale; <= 0 means 1/sqrt(d) */
+  int32_t local_groups; /* 0: local set = sliding neighbourhood of radius (rlat, rlon);
+                           1: local set = the aligned group of rlat x rlon blocks that holds the block
+                              (the paper's "Local Attention": dense attention inside large blocks) */
 } mo_geom;
 
 #define MO_MAX_LOCAL 256
@@ -63,7 +66,9 @@ static int g_ok(const mo_geom *g) {
   if (!g || g->nlat <= 0 || g->nlon <= 0 || g->d <= 0 || g->bh <= 0 || g->bw <= 0) return 0;
   if (g->nlat % g->bh || g->nlon % g->bw) return 0;
   if (g->rlat < 0 || g->rlon < 0 || g->topk < 0) return 0;
-  if ((2 * g->rlat + 1) * (2 * g->rlon + 1) > MO_MAX_LOCAL) return 0;
+  if (g->local_groups) {
+    if (g->rlat < 1 || g->rlon < 1 || g->rlat * g->rlon > MO_MAX_LOCAL) return 0;
+  } else if ((2 * g->rlat + 1) * (2 * g->rlon + 1) > MO_MAX_LOCAL) return 0;
   return 1;
 }
 static int g_nbh(const mo_geom *g) { return g->nlat / g->bh; }
@@ -98,11 +103,18 @@ int mo_num_threads(void) {
 /*
  * Local set of query block i: rows clamp(by+dy), columns (bx+dx) mod nbw, as a SET
  * (each block once), listed in first-occurrence order over dy, then dx ascending.
+ * With local_groups: the aligned group of rlat x rlon blocks that holds block i.
  */
 int mo_local_set(const mo_geom *g, int32_t i, int32_t *out) {
   if (!g_ok(g)) return -1;
   int nbh = g_nbh(g), nbw = g_nbw(g);
   int by = i / nbw, bx = i % nbw, n = 0;
+  if (g->local_groups) { /* the blocks of the aligned rlat x rlon group, row-major, those inside the grid */
+    int y0 = (by / g->rlat) * g->rlat, x0 = (bx / g->rlon) * g->rlon;
+    for (int y = y0; y < y0 + g->rlat && y < nbh; ++y)
+      for (int x = x0; x < x0 + g->rlon && x < nbw; ++x) out[n++] = y * nbw + x;
+    return n;
+  }
   for (int dy = -g->rlat; dy <= g->rlat; ++dy) {
     int y = by + dy;
     if (y < 0) y = 0;

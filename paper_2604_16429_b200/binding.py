@@ -22,6 +22,7 @@ EXPORTS = ("mosaic_bsa_workspace_bytes", "mosaic_bsa_select", "mosaic_bsa_fwd", 
            "mosaic_bsa_last_status", "mosaic_bsa_strerror", "mosaic_bsa_select_static",
            "mosaic_bsa_descriptor_encodes", "mosaic_bsa_fwd_branches")
 STATIC_SCRATCH_BYTES = 4 << 20
+FLAG_LOCAL_GROUPS = 1
 
 
 class MosaicError(RuntimeError):
@@ -66,7 +67,7 @@ class Params:
     @staticmethod
     def from_workload(w, **over):
         kw = dict(B=w.B, H=w.H, nlat=w.nlat, nlon=w.nlon, d=w.d, bh=w.bh, bw=w.bw, rlat=w.rlat, rlon=w.rlon,
-                  topk=w.topk)
+                  topk=w.topk, flags=FLAG_LOCAL_GROUPS if getattr(w, "local_groups", False) else 0)
         kw.update(over)
         return Params(**kw)
 

@@ -12,7 +12,7 @@ size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 int validate(const mosaic_bsa_params* p, Geo* g) {
   if (!p) return MOSAIC_E_INVALID_ARG;
   if (p->B <= 0 || p->H <= 0 || p->nlat <= 0 || p->nlon <= 0 || p->bh <= 0 || p->bw <= 0 || p->topk < 0 ||
-      p->rlat < 0 || p->rlon < 0 || p->flags != 0)
+      p->rlat < 0 || p->rlon < 0 || (p->flags & ~MOSAIC_FLAG_LOCAL_GROUPS) != 0)
     return MOSAIC_E_INVALID_ARG;
   if (p->nlat % p->bh || p->nlon % p->bw) return MOSAIC_E_INVALID_ARG;
   if (!(p->scale == p->scale) || isinf(p->scale)) return MOSAIC_E_INVALID_ARG;
@@ -22,8 +22,12 @@ int validate(const mosaic_bsa_params* p, Geo* g) {
   if (p->bh % crows) return MOSAIC_E_UNSUPPORTED;
   const int cpb = p->bh * p->bw / kChunk;
   if (!(cpb == 1 || cpb % 2 == 0)) return MOSAIC_E_UNSUPPORTED;
-  if (p->rlat > 2 || p->rlon > 2 || p->topk > kMaxTopk) return MOSAIC_E_UNSUPPORTED;
-  if ((2 * p->rlat + 1) * (2 * p->rlon + 1) + p->topk > kMaxList) return MOSAIC_E_UNSUPPORTED;
+  const bool groups = (p->flags & MOSAIC_FLAG_LOCAL_GROUPS) != 0;
+  if (groups && (p->rlat < 1 || p->rlon < 1)) return MOSAIC_E_INVALID_ARG;
+  if (p->topk > kMaxTopk) return MOSAIC_E_UNSUPPORTED;
+  if (groups ? (long long)p->rlat * p->rlon > 32 : (p->rlat > 2 || p->rlon > 2)) return MOSAIC_E_UNSUPPORTED;
+  const int nlocal = groups ? p->rlat * p->rlon : (2 * p->rlat + 1) * (2 * p->rlon + 1);
+  if (nlocal + p->topk > kMaxList) return MOSAIC_E_UNSUPPORTED;
   const long long U = (long long)p->B * p->H, N = (long long)p->nlat * p->nlon;
   const long long m = (long long)(p->nlat / p->bh) * (p->nlon / p->bw);
   if (U > (1 << 24) || m > (1 << 24) || U * m * cpb > 0x7fffffffll || U * N > (1ll << 40)) return MOSAIC_E_UNSUPPORTED;
@@ -33,6 +37,7 @@ int validate(const mosaic_bsa_params* p, Geo* g) {
   g->b = p->bh * p->bw; g->cpb = cpb; g->crows = crows;
   g->rlat = p->rlat; g->rlon = p->rlon; g->topk = p->topk;
   g->local_off = 0;
+  g->local_groups = groups ? 1 : 0;
   g->scale = p->scale > 0.f ? p->scale : 1.0f / sqrtf((float)p->d);
   g->scale_log2 = g->scale * 1.4426950408889634f;
   g->N = N;

@@ -24,6 +24,7 @@ struct Geo {
   int crows;        // grid rows per chunk (64 / bw)
   int rlat, rlon, topk;
   int local_off;    // 1: the local neighbourhood is not attended (selection branch of the three-branch form)
+  int local_groups; // 1: the local set is the aligned group of rlat x rlon blocks that holds the block
   float scale;      // softmax scale
   float scale_log2; // scale * log2(e)
   long long N;      // tokens per unit
@@ -32,10 +33,12 @@ struct Geo {
 // Record the first device-side fault in the workspace status word (never traps).
 __device__ __forceinline__ void set_status(int* status, int code) { atomicCAS(status, 0, code); }
 
-// Is key block j inside the local neighbourhood of query block i (rows clamp(by+dy), columns (bx+dx) mod nbw)?
+// Is key block j inside the local set of query block i (window: rows clamp(by+dy), columns (bx+dx) mod nbw;
+// group mode: the same aligned group of rlat x rlon blocks)?
 __device__ __forceinline__ bool is_local(const Geo& g, int i, int j) {
   int by = i / g.nbw, bx = i - by * g.nbw;
   int jy = j / g.nbw, jx = j - jy * g.nbw;
+  if (g.local_groups) return by / g.rlat == jy / g.rlat && bx / g.rlon == jx / g.rlon;
   // clamping only folds an out-of-range row onto a row already in the window
   bool row_ok = abs(jy - by) <= g.rlat;
   int dx = jx - bx;

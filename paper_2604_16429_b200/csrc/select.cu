@@ -351,7 +351,8 @@ __global__ void __launch_bounds__(NW * 32) topk_kernel(Geo g, const float* __res
         const int j = j0 + lane + 32 * b;
         int dx = jx[b] - ix[a];
         dx += dx < 0 ? g.nbw : 0;  // (jx - ix) mod nbw
-        const bool local = abs(jy[b] - iy[a]) <= g.rlat && (dx <= g.rlon || g.nbw - dx <= g.rlon);
+        const bool local = g.local_groups ? (jy[b] / g.rlat == iy[a] / g.rlat && jx[b] / g.rlon == ix[a] / g.rlon)
+                                          : (abs(jy[b] - iy[a]) <= g.rlat && (dx <= g.rlon || g.nbw - dx <= g.rlon));
         const bool cand = row_ok && j < g.m && !local;
         const float s = acc[a][b], eps = fmaf(nqv[a] * nkv[b], 1.52587890625e-5f, 1e-37f);
         const bool fin = fabsf(s) <= 1e38f && eps <= 1e38f;
@@ -455,7 +456,8 @@ __global__ void __launch_bounds__(NW * 32) topk_kernel(Geo g, const float* __res
             const int jy = j / g.nbw, jx = j - jy * g.nbw;
             int dx = jx - ix[a];
             dx += dx < 0 ? g.nbw : 0;
-            cand = !(abs(jy - iy[a]) <= g.rlat && (dx <= g.rlon || g.nbw - dx <= g.rlon));
+            cand = g.local_groups ? !(jy / g.rlat == iy[a] / g.rlat && jx / g.rlon == ix[a] / g.rlon)
+                                  : !(abs(jy - iy[a]) <= g.rlat && (dx <= g.rlon || g.nbw - dx <= g.rlon));
           }
           insert_batch(cand ? exact_key(sm.qs[row], pk_u, j) : 0ull, j, lkey, lid, g.topk, lane);
         }

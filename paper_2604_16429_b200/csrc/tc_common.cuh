@@ -269,14 +269,24 @@ __device__ __forceinline__ int item_halves(const Geo& g, int it, int (&hb)[4], i
         valid |= (bx0 + h < g.nbw) << h;
       }
     }
-  } else if (g.cpb == 2) {  // two neighbouring 128-token blocks
-    const int ntx = (g.nbw + 1) >> 1, by = it / ntx, tx = it - by * ntx;
+  } else if (g.cpb == 2) {  // two neighbouring 128-token blocks: side by side, or one above the other in a one-column grid
+    if (g.nbw > 1) {
+      const int ntx = (g.nbw + 1) >> 1, by = it / ntx, tx = it - by * ntx;
 #pragma unroll
-    for (int h = 0; h < 4; ++h) {
-      const int bx = 2 * tx + (h >> 1);
-      hb[h] = by * g.nbw + bx;
-      hc[h] = h & 1;
-      valid |= (bx < g.nbw) << h;
+      for (int h = 0; h < 4; ++h) {
+        const int bx = 2 * tx + (h >> 1);
+        hb[h] = by * g.nbw + bx;
+        hc[h] = h & 1;
+        valid |= (bx < g.nbw) << h;
+      }
+    } else {
+#pragma unroll
+      for (int h = 0; h < 4; ++h) {
+        const int by = 2 * it + (h >> 1);
+        hb[h] = by;
+        hc[h] = h & 1;
+        valid |= (by < g.nbh) << h;
+      }
     }
   } else {                  // four chunks of one block
     const int ipb = (g.cpb + 3) >> 2, blk = it / ipb, c0 = 4 * (it - blk * ipb);
@@ -295,7 +305,7 @@ __device__ __forceinline__ int item_halves(const Geo& g, int it, int (&hb)[4], i
 
 __host__ __device__ inline int items_per_unit(const Geo& g) {
   if (g.cpb == 1) return (g.nbh >> 1) * ((g.nbw + 1) >> 1) + (g.nbh & 1) * ((g.nbw + 3) >> 2);
-  if (g.cpb == 2) return g.nbh * ((g.nbw + 1) >> 1);
+  if (g.cpb == 2) return g.nbw > 1 ? g.nbh * ((g.nbw + 1) >> 1) : (g.nbh + 1) >> 1;
   return g.m * ((g.cpb + 3) >> 2);
 }
 
@@ -303,17 +313,28 @@ __host__ __device__ inline int items_per_unit(const Geo& g) {
 // ids[n0..); returns the new count.  `j` is this lane's entry of the block's row of block_idx (-1 beyond top-k).
 __device__ __forceinline__ int warp_attended(const Geo& g, int j, int i, int* ids, int n0, int lane, int* status) {
   const int by = i / g.nbw, bx = i - by * g.nbw;
-  const int wl = 2 * g.rlon + 1, nl = g.local_off ? 0 : (2 * g.rlat + 1) * wl;
-  int id = -1 - lane;
-  if (lane < nl) {
-    const int dy = lane / wl - g.rlat, dx = lane - (lane / wl) * wl - g.rlon;
-    const int y = min(max(by + dy, 0), g.nbh - 1);
-    int x = (bx + dx) % g.nbw;
-    x += x < 0 ? g.nbw : 0;
-    id = y * g.nbw + x;
+  int id = -1 - lane;  // lanes without a block hold distinct negative values
+  int nl;
+  if (g.local_groups) {   // the aligned group of rlat x rlon blocks that holds block i (ragged at the grid's edge)
+    nl = g.local_off ? 0 : g.rlat * g.rlon;
+    if (lane < nl) {
+      const int dy = lane / g.rlon, dx = lane - dy * g.rlon;
+      const int y = (by / g.rlat) * g.rlat + dy, x = (bx / g.rlon) * g.rlon + dx;
+      if (y < g.nbh && x < g.nbw) id = y * g.nbw + x;
+    }
+  } else {
+    const int wl = 2 * g.rlon + 1;
+    nl = g.local_off ? 0 : (2 * g.rlat + 1) * wl;
+    if (lane < nl) {
+      const int dy = lane / wl - g.rlat, dx = lane - (lane / wl) * wl - g.rlon;
+      const int y = min(max(by + dy, 0), g.nbh - 1);
+      int x = (bx + dx) % g.nbw;
+      x += x < 0 ? g.nbw : 0;
+      id = y * g.nbw + x;
+    }
   }
   const unsigned same = __match_any_sync(0xffffffffu, id);
-  const bool keep = lane < nl && (__ffs(same) - 1) == lane;  // first occurrence of a block
+  const bool keep = id >= 0 && (__ffs(same) - 1) == lane;  // first occurrence of a block
   const unsigned km = __ballot_sync(0xffffffffu, keep);
   if (keep) ids[n0 + __popc(km & ((1u << lane) - 1u))] = id;
   int n = n0 + __popc(km);

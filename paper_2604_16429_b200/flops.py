@@ -13,6 +13,13 @@ def local_count(by: int, nbh: int, nbw: int, rlat: int, rlon: int) -> int:
 def pairs_per_unit(w) -> int:
     nbh, nbw = w.nlat // w.bh, w.nlon // w.bw
     total = 0
+    if getattr(w, "local_groups", False):   # local set = the aligned group of rlat x rlon blocks (ragged at the edges)
+        for by in range(nbh):
+            for bx in range(nbw):
+                nl = (min(nbh, (by // w.rlat + 1) * w.rlat) - (by // w.rlat) * w.rlat) * \
+                     (min(nbw, (bx // w.rlon + 1) * w.rlon) - (bx // w.rlon) * w.rlon)
+                total += nl + min(w.topk, w.m - nl)
+        return total
     for by in range(nbh):
         nl = local_count(by, nbh, nbw, w.rlat, w.rlon)
         total += nbw * (nl + min(w.topk, w.m - nl))

@@ -43,6 +43,7 @@ class Workload:
     d: int = 64
     rlat: int = 1
     rlon: int = 1
+    local_groups: bool = False   # local set = aligned group of rlat x rlon blocks (the paper's large local blocks)
 
     @property
     def N(self): return self.nlat * self.nlon
@@ -60,6 +61,12 @@ WORKLOADS = {
     "c3_1p5deg_ens24": Workload("c3_1p5deg_ens24", 3, 24, 8, 120, 240, 8, 8, 8, "smooth"),
     "c4_1p5deg_train": Workload("c4_1p5deg_train", 4, 4, 16, 120, 240, 8, 8, 8, "smooth", True),
     "c5_0p25deg": Workload("c5_0p25deg", 5, 1, 8, 720, 1440, 16, 16, 16, "smooth"),
+    # The paper's own layout and shapes (architecture table): HEALPix NESTED sequence of 12 * nside^2 tokens, sparse
+    # blocks of 128 contiguous tokens (8 rows of a 16-wide view of the sequence), local attention inside aligned
+    # 1024-token blocks (8 sparse blocks), 24 / 12 / 4 selected blocks, d = 64 per head.
+    "hp_nside64": Workload("hp_nside64", 6, 1, 12, 3072, 16, 8, 16, 24, "smooth", rlat=8, rlon=1, local_groups=True),
+    "hp_nside32": Workload("hp_nside32", 7, 1, 16, 768, 16, 8, 16, 12, "smooth", rlat=8, rlon=1, local_groups=True),
+    "hp_nside16": Workload("hp_nside16", 8, 1, 20, 192, 16, 8, 16, 4, "smooth", rlat=8, rlon=1, local_groups=True),
 }
 
 
@@ -113,7 +120,8 @@ def make_inputs(w: Workload, with_do: bool | None = None) -> dict:
     return out
 
 
-def small_case(nlat, nlon, bh, bw, topk, B=1, H=1, d=64, kind="iid", seed=7, rlat=1, rlon=1, backward=False):
+def small_case(nlat, nlon, bh, bw, topk, B=1, H=1, d=64, kind="iid", seed=7, rlat=1, rlon=1, backward=False,
+               local_groups=False):
     """A free-form small workload for tests (cfg number = seed)."""
-    return Workload(f"small_{nlat}x{nlon}_{bh}x{bw}_k{topk}", seed, B, H, nlat, nlon, bh, bw, topk, kind,
-                    backward, d, rlat, rlon)
+    return Workload(f"small_{nlat}x{nlon}_{bh}x{bw}_k{topk}" + ("_groups" if local_groups else ""), seed, B, H, nlat,
+                    nlon, bh, bw, topk, kind, backward, d, rlat, rlon, local_groups)

@@ -43,7 +43,8 @@ class Guarded:
 
 
 def geom_of(w, scale=0.0) -> Geom:
-    return Geom(w.nlat, w.nlon, d=w.d, bh=w.bh, bw=w.bw, rlat=w.rlat, rlon=w.rlon, topk=w.topk, scale=scale)
+    return Geom(w.nlat, w.nlon, d=w.d, bh=w.bh, bw=w.bw, rlat=w.rlat, rlon=w.rlon, topk=w.topk, scale=scale,
+                local_groups=getattr(w, "local_groups", False))
 
 
 def device_inputs(x: dict) -> dict:

@@ -424,3 +424,30 @@ def test_golden_fixture_is_reproduced():
     _, L = oracle.fwd(g, x["q"][0, 0], x["k"][0, 0], x["v"][0, 0], idx, blocks)
     for n, r in enumerate(want_lse):
         assert np.allclose(L[n, :4], [float(t) for t in r[1:]], rtol=0, atol=1e-12)
+
+
+# ------------------------------------------------------------------ aligned local groups (the paper's large local blocks)
+
+def test_local_groups_set_and_forward_against_masked_dense():
+    """With local_groups the local set is the aligned group of rlat x rlon blocks (ragged at the grid's edge):
+    checked against the definition written here, and the forward against masked dense attention."""
+    g = Geom(40, 48, d=8, bh=8, bw=8, rlat=2, rlon=4, topk=2, local_groups=True)   # 5 x 6 blocks
+    for i in range(g.m):
+        by, bx = divmod(i, g.nbw)
+        want = [y * g.nbw + x for y in range(by // 2 * 2, min(by // 2 * 2 + 2, g.nbh))
+                for x in range(bx // 4 * 4, min(bx // 4 * 4 + 4, g.nbw))]
+        assert oracle.local_set(g, i) == want
+    # one-column grid: the paper's layout (blocks of contiguous tokens, groups of 8 blocks)
+    gh = Geom(256, 16, d=8, bh=8, bw=16, rlat=8, rlon=1, topk=3, local_groups=True)  # 32 blocks of 128 tokens
+    assert oracle.local_set(gh, 13) == list(range(8, 16))
+    rng = np.random.default_rng(21)
+    q, k, v = (rand_bits(rng, gh.N, gh.d) for _ in range(3))
+    idx = oracle.select(gh, q, k)
+    assert all(j // 8 != i // 8 for i in range(gh.m) for j in idx[i])                # selected blocks are never local
+    O, L = oracle.fwd(gh, q, k, v, idx)
+    qf, kf, vf = f64(q), f64(k), f64(v)
+    for i in (0, 13, 31):
+        blocks = list(range(i // 8 * 8, i // 8 * 8 + 8)) + idx[i].tolist()
+        toks = np.concatenate([np.arange(j * 128, (j + 1) * 128) for j in blocks])   # block j = tokens 128 j .. 128 j + 127
+        od, ld = dense_attention(qf[i * 128:(i + 1) * 128], kf[toks], vf[toks], 1 / math.sqrt(gh.d))
+        assert np.abs(O[i] - od).max() < 1e-12 and np.abs(L[i] - ld).max() < 1e-12

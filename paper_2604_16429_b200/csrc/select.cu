@@ -174,23 +174,26 @@ __device__ __forceinline__ void insert_batch(unsigned long long key, int id, uns
 // exact score of (pooled query row in shared memory, pooled key row j in global memory) as a sortable key
 __device__ __forceinline__ unsigned long long exact_key(const float* qrow, const float* __restrict__ pk_u, int j) {
   const float4* krow = reinterpret_cast<const float4*>(pk_u + (long long)j * kD);
-  float4 kv[kD / 4];
-#pragma unroll
-  for (int c4 = 0; c4 < kD / 4; ++c4) kv[c4] = __ldg(krow + c4);
   double s = 0.0;
 #pragma unroll
-  for (int c4 = 0; c4 < kD / 4; ++c4) {
-    const float4 qv = *reinterpret_cast<const float4*>(qrow + 4 * c4);
-    s = fma((double)qv.x, (double)kv[c4].x, s);
-    s = fma((double)qv.y, (double)kv[c4].y, s);
-    s = fma((double)qv.z, (double)kv[c4].z, s);
-    s = fma((double)qv.w, (double)kv[c4].w, s);
+  for (int half = 0; half < 2; ++half) {  // eight 16-byte loads in flight, then their 32 sequential FMAs
+    float4 kv[kD / 8];
+#pragma unroll
+    for (int c4 = 0; c4 < kD / 8; ++c4) kv[c4] = __ldg(krow + half * (kD / 8) + c4);
+#pragma unroll
+    for (int c4 = 0; c4 < kD / 8; ++c4) {
+      const float4 qv = *reinterpret_cast<const float4*>(qrow + 4 * (half * (kD / 8) + c4));
+      s = fma((double)qv.x, (double)kv[c4].x, s);
+      s = fma((double)qv.y, (double)kv[c4].y, s);
+      s = fma((double)qv.z, (double)kv[c4].z, s);
+      s = fma((double)qv.w, (double)kv[c4].w, s);
+    }
   }
   return score_key(s);
 }
 
-template <int NW, int RI, int CAP, int JT>
-__global__ void __launch_bounds__(NW * 32) topk_kernel(Geo g, const float* __restrict__ pq,
+template <int NW, int RI, int CAP, int JT, int MB>
+__global__ void __launch_bounds__(NW * 32, MB) topk_kernel(Geo g, const float* __restrict__ pq,
                                                        const float* __restrict__ pk, const float* __restrict__ nq,
                                                        const float* __restrict__ nk, int32_t* __restrict__ block_idx) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -332,49 +335,74 @@ __global__ void __launch_bounds__(NW * 32) topk_kernel(Geo g, const float* __res
         }
       }
     }
-    int jy[KB], jx[KB];
-    float nkv[KB];
+    float nkc[KB];  // norm bound of the lane's keys times 2^-16
 #pragma unroll
-    for (int b = 0; b < KB; ++b) {
-      const int j = min(j0 + lane + 32 * b, g.m - 1);
-      jy[b] = j / g.nbw;
-      jx[b] = j - jy[b] * g.nbw;
-      nkv[b] = sm.scr.nk[buf][lane + 32 * b];
-    }
+    for (int b = 0; b < KB; ++b) nkc[b] = sm.scr.nk[buf][lane + 32 * b] * 1.52587890625e-5f;
     unsigned stale = 0;  // rows whose threshold should be recomputed
-#pragma unroll
-    for (int a = 0; a < RI; ++a) {
-      const bool row_ok = i0 + warp * RI + a < g.m;  // warp-uniform
-      const int row = warp * RI + a;
-#pragma unroll
-      for (int b = 0; b < KB; ++b) {
-        const int j = j0 + lane + 32 * b;
-        int dx = jx[b] - ix[a];
-        dx += dx < 0 ? g.nbw : 0;  // (jx - ix) mod nbw
-        const bool local = g.local_groups ? (jy[b] / g.rlat == iy[a] / g.rlat && jx[b] / g.rlon == ix[a] / g.rlon)
-                                          : (abs(jy[b] - iy[a]) <= g.rlat && (dx <= g.rlon || g.nbw - dx <= g.rlon));
-        const bool cand = row_ok && j < g.m && !local;
-        const float s = acc[a][b], eps = fmaf(nqv[a] * nkv[b], 1.52587890625e-5f, 1e-37f);
-        const bool fin = fabsf(s) <= 1e38f && eps <= 1e38f;
-        const float lb = fin ? s - eps : -kInf, ub = fin ? s + eps : kInf;
-        if (v >= 1) {
-          const bool keep = cand && !(ub < thr[a]);
-          const unsigned km = __ballot_sync(0xffffffffu, keep);
+    // One candidate: bounds of its exact score, filter against the row's threshold, tracking of the lower bounds.
+    // A non-finite screening score gives the interval (-inf, +inf); a non-finite eps does so by itself (s + eps is
+    // then +inf or NaN, which the filter keeps, and s - eps is -inf or NaN, which the tracking ignores).
+    auto candidate = [&](int a, int b, bool cand) {
+      const float sc = acc[a][b], eps = fmaf(nqv[a], nkc[b], 1e-37f);
+      const bool fin = fabsf(sc) <= 1e38f;
+      const float lb = fin ? sc - eps : -kInf, ub = fin ? sc + eps : kInf;
+      if (v >= 1) {
+        const bool keep = cand && !(ub < thr[a]);
+        const unsigned km = __ballot_sync(0xffffffffu, keep);
+        if (km) {  // warp-uniform
           if (keep) {
             const int at = cnt[a] + __popc(km & lower);
-            if (at < CAP) { sm.surv[row][at] = j; sm.surv_ub[row][at] = ub; }
+            if (at < CAP) { sm.surv[warp * RI + a][at] = j0 + lane + 32 * b; sm.surv_ub[warp * RI + a][at] = ub; }
           }
           cnt[a] += __popc(km);
         }
-        if (v != 1 && cand) {  // the home chunk's bounds were tracked in the threshold-only visit
-          if (lb > m1[a]) { m2[a] = m1[a]; m1[a] = lb; }
-          else m2[a] = fmaxf(m2[a], lb);
+      }
+      if (v != 1 && cand) {  // the home chunk's bounds were tracked in the threshold-only visit
+        if (lb > m1[a]) { m2[a] = m1[a]; m1[a] = lb; }
+        else m2[a] = fmaxf(m2[a], lb);
+      }
+    };
+    // Plain chunk for this warp (the common case): wholly inside the grid, every row of the warp exists, and no key of
+    // the chunk can be local to any of the warp's rows, so every (row, key) pair is a candidate.
+    const int i_lo = i0 + warp * RI, i_hi = i_lo + RI - 1;
+    bool plain = j0 + JT <= g.m && i_hi < g.m;
+    if (plain) {
+      const int jy_lo = j0 / g.nbw, jy_hi = (j0 + JT - 1) / g.nbw, iy_lo = i_lo / g.nbw, iy_hi = i_hi / g.nbw;
+      plain = g.local_groups ? (jy_lo / g.rlat > iy_hi / g.rlat || jy_hi / g.rlat < iy_lo / g.rlat)
+                             : (jy_lo > iy_hi + g.rlat || jy_hi < iy_lo - g.rlat);
+    }
+    if (plain) {
+#pragma unroll
+      for (int a = 0; a < RI; ++a)
+#pragma unroll
+        for (int b = 0; b < KB; ++b) candidate(a, b, true);
+    } else {
+      int jy[KB], jx[KB];
+#pragma unroll
+      for (int b = 0; b < KB; ++b) {
+        const int j = min(j0 + lane + 32 * b, g.m - 1);
+        jy[b] = j / g.nbw;
+        jx[b] = j - jy[b] * g.nbw;
+      }
+#pragma unroll
+      for (int a = 0; a < RI; ++a) {
+        const bool row_ok = i_lo + a < g.m;  // warp-uniform
+#pragma unroll
+        for (int b = 0; b < KB; ++b) {
+          int dx = jx[b] - ix[a];
+          dx += dx < 0 ? g.nbw : 0;  // (jx - ix) mod nbw
+          const bool local = g.local_groups ? (jy[b] / g.rlat == iy[a] / g.rlat && jx[b] / g.rlon == ix[a] / g.rlon)
+                                            : (abs(jy[b] - iy[a]) <= g.rlat && (dx <= g.rlon || g.nbw - dx <= g.rlon));
+          candidate(a, b, row_ok && j0 + lane + 32 * b < g.m && !local);
         }
       }
+    }
+#pragma unroll
+    for (int a = 0; a < RI; ++a) {
       // recompute when the row has no threshold yet, gathered enough new survivors to suggest it is stale, fills
       // up, or is about to be scored
       const bool due = v <= 1 || v == nchunks || cnt[a] - cnt_upd[a] >= g.topk / 2 + 4 || cnt[a] > CAP / 2;
-      if (row_ok && due && cnt[a] <= CAP) stale |= 1u << a;
+      if (i_lo + a < g.m && due && cnt[a] <= CAP) stale |= 1u << a;
     }
     if (stale) {  // warp-uniform
       __syncwarp();
@@ -467,7 +495,7 @@ __global__ void __launch_bounds__(NW * 32) topk_kernel(Geo g, const float* __res
   }
 }
 
-template <int NW, int RI, int CAP, int JT>
+template <int NW, int RI, int CAP, int JT, int MB>
 int launch_topk(const HostCtx& c, const float* pooled_q, const float* pooled_k, const float* norm_q,
                 const float* norm_k, int32_t* block_idx) {
   const Geo& g = c.g;
@@ -477,13 +505,13 @@ int launch_topk(const HostCtx& c, const float* pooled_q, const float* pooled_k, 
   if (cudaGetDevice(&dev) != cudaSuccess) return MOSAIC_E_CUDA;
   if (dev < 0 || dev >= 64) return MOSAIC_E_UNSUPPORTED;
   if (!((configured >> dev) & 1ull)) {
-    if (cudaFuncSetAttribute(topk_kernel<NW, RI, CAP, JT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+    if (cudaFuncSetAttribute(topk_kernel<NW, RI, CAP, JT, MB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
         cudaSuccess)
       return MOSAIC_E_CUDA;
     configured |= 1ull << dev;
   }
   const int tiles = (g.m + NW * RI - 1) / (NW * RI);
-  topk_kernel<NW, RI, CAP, JT><<<(unsigned)(g.U * tiles), NW * 32, smem, c.stream>>>(g, pooled_q, pooled_k, norm_q,
+  topk_kernel<NW, RI, CAP, JT, MB><<<(unsigned)(g.U * tiles), NW * 32, smem, c.stream>>>(g, pooled_q, pooled_k, norm_q,
                                                                                 norm_k, block_idx);
   return cudaGetLastError() == cudaSuccess ? MOSAIC_OK : MOSAIC_E_CUDA;
 }
@@ -520,10 +548,10 @@ int launch_select(const HostCtx& c, const void* q, const void* k, int32_t* block
     // the most query blocks per CTA (64, 32, 16) that still gives every SM about two CTAs; small problems are
     // latency-bound and take 8 rows per CTA and 64-key chunks, so that more warps are resident
     auto ctas = [&](int ti) { return (long long)g.U * ((g.m + ti - 1) / ti); };
-    const int rc = ctas(64) >= 296   ? launch_topk<8, 8, 128, 128>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx)
-                   : ctas(32) >= 296 ? launch_topk<4, 8, 128, 128>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx)
-                   : ctas(16) >= 296 ? launch_topk<4, 4, 192, 128>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx)
-                                     : launch_topk<4, 2, 96, 64>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx);
+    const int rc = ctas(64) >= 296   ? launch_topk<8, 4, 96, 64, 3>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx)
+                   : ctas(32) >= 296 ? launch_topk<4, 8, 128, 128, 1>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx)
+                   : ctas(16) >= 296 ? launch_topk<4, 4, 192, 128, 2>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx)
+                                     : launch_topk<4, 2, 96, 64, 4>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx);
     if (rc) return rc;
   }
   return MOSAIC_OK;

@@ -139,8 +139,9 @@ def describe(w) -> str:
 def oracle_sample_step(w, x, g, blocks, unit=(0, 0)):
     import oracle
     b, h = unit
-    idx = oracle.select(g, x["q"][b, h], x["k"][b, h])
-    oracle.fwd(g, x["q"][b, h], x["k"][b, h], x["v"][b, h], idx, blocks)
+    hk = h // (w.H // w.kv_heads)
+    idx = oracle.select(g, x["q"][b, h], x["k"][b, hk])
+    oracle.fwd(g, x["q"][b, h], x["k"][b, hk], x["v"][b, hk], idx, blocks)
     return idx
 
 
@@ -170,8 +171,9 @@ def cpu_baseline(w, x, idx_gpu, o_gpu, lse_gpu) -> dict:
     fl, dt, worst = 0.0, 0.0, 0.0
     for (b, h) in units:
         t0 = time.perf_counter()
-        idx0 = oracle.select(g, x["q"][b, h], x["k"][b, h])
-        O, L = oracle.fwd(g, x["q"][b, h], x["k"][b, h], x["v"][b, h], idx0, blocks)
+        hk = h // (w.H // w.kv_heads)
+        idx0 = oracle.select(g, x["q"][b, h], x["k"][b, hk])
+        O, L = oracle.fwd(g, x["q"][b, h], x["k"][b, hk], x["v"][b, hk], idx0, blocks)
         dt += time.perf_counter() - t0
         fl += sample_flops(w, g, blocks)
         assert np.array_equal(idx_gpu[b, h].cpu().numpy(), idx0), "selection differs from the oracle"
@@ -296,7 +298,7 @@ def run_ours(args, w):
     idx = torch.empty((w.B, w.H, w.m, w.topk), dtype=torch.int32, device=dev)
     o = torch.empty_like(dx["q"])
     lse = torch.empty((w.B, w.H, w.N), dtype=torch.float32, device=dev)
-    dq, dk, dv = (torch.empty_like(dx["q"]) for _ in range(3))
+    dq, dk, dv = torch.empty_like(dx["q"]), torch.empty_like(dx["k"]), torch.empty_like(dx["k"])
     flush_buf = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
 

@@ -15,7 +15,10 @@
  * Common rules for every entry point
  *   - All tensor pointers are DEVICE pointers on the current CUDA device.  Q, K, V, O,
  *     dO are contiguous [B, H, N, d] bf16 with token t = lat*nlon + lon, base address
- *     16-byte aligned.  "unit" u = b*H + h; units are independent.
+ *     16-byte aligned.  "unit" u = b*H + h; units are independent.  With grouped-query
+ *     attention (Hkv < H; paper: "Overall architecture" paragraph, GQA ratio 4) K, V, dK, dV
+ *     are [B, Hkv, N, d] and query head h reads key/value head h / (H / Hkv); the selection
+ *     stays per query head, dK and dV sum over the query heads of a group.
  *   - block_idx is contiguous [B, H, m, topk] int32, m = (nlat/bh)*(nlon/bw), block id
  *     j = by*(nlon/bw) + bx.  Row i holds the selected non-local block ids of query
  *     block i, best first, padded with -1.  The local set is implicit.
@@ -58,6 +61,8 @@ typedef struct mosaic_bsa_params {
   int32_t topk;       /* selected non-local blocks per query block, >= 0               */
   float scale;        /* softmax scale; <= 0 means 1/sqrt(d)                           */
   uint32_t flags;     /* 0 or MOSAIC_FLAG_LOCAL_GROUPS                                 */
+  int32_t Hkv;        /* heads of K and V (grouped-query attention, the paper's GQA ratio
+                         H / Hkv); 0 means H; H % Hkv == 0                                */
 } mosaic_bsa_params;
 
 /* Local attention inside aligned groups of blocks instead of a sliding neighbourhood (the paper's "Local

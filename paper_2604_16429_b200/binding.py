@@ -35,7 +35,7 @@ class _Params(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("nlat", ctypes.c_int32), ("nlon", ctypes.c_int32),
                 ("d", ctypes.c_int32), ("bh", ctypes.c_int32), ("bw", ctypes.c_int32),
                 ("rlat", ctypes.c_int32), ("rlon", ctypes.c_int32), ("topk", ctypes.c_int32),
-                ("scale", ctypes.c_float), ("flags", ctypes.c_uint32)]
+                ("scale", ctypes.c_float), ("flags", ctypes.c_uint32), ("Hkv", ctypes.c_int32)]
 
 
 @dataclass(frozen=True)
@@ -52,7 +52,10 @@ class Params:
     topk: int = 8
     scale: float = 0.0
     flags: int = 0
+    Hkv: int = 0          # heads of K and V (grouped-query attention); 0 = H
 
+    @property
+    def kv_heads(self): return self.Hkv or self.H
     @property
     def N(self): return self.nlat * self.nlon
     @property
@@ -62,12 +65,13 @@ class Params:
 
     def c(self):
         return _Params(self.B, self.H, self.nlat, self.nlon, self.d, self.bh, self.bw, self.rlat, self.rlon,
-                       self.topk, self.scale, self.flags)
+                       self.topk, self.scale, self.flags, self.Hkv)
 
     @staticmethod
     def from_workload(w, **over):
         kw = dict(B=w.B, H=w.H, nlat=w.nlat, nlon=w.nlon, d=w.d, bh=w.bh, bw=w.bw, rlat=w.rlat, rlon=w.rlon,
-                  topk=w.topk, flags=FLAG_LOCAL_GROUPS if getattr(w, "local_groups", False) else 0)
+                  topk=w.topk, flags=FLAG_LOCAL_GROUPS if getattr(w, "local_groups", False) else 0,
+                  Hkv=getattr(w, "Hkv", 0))
         kw.update(over)
         return Params(**kw)
 
@@ -121,10 +125,11 @@ def _ptr(t) -> int:
     return 0 if t is None else int(t.data_ptr())
 
 
-def _chk_qkv(p: Params, *ts):
+def _chk_qkv(p: Params, *ts, heads=None):
+    h = p.H if heads is None else heads
     for t in ts:
-        if t.dtype != torch.bfloat16 or not t.is_cuda or not t.is_contiguous() or tuple(t.shape) != (p.B, p.H, p.N, p.d):
-            raise ValueError(f"expected contiguous cuda bf16 [{p.B},{p.H},{p.N},{p.d}], got {t.dtype} {tuple(t.shape)}")
+        if t.dtype != torch.bfloat16 or not t.is_cuda or not t.is_contiguous() or tuple(t.shape) != (p.B, h, p.N, p.d):
+            raise ValueError(f"expected contiguous cuda bf16 [{p.B},{h},{p.N},{p.d}], got {t.dtype} {tuple(t.shape)}")
 
 
 def alloc_workspace(p: Params, op: int, device="cuda") -> torch.Tensor:
@@ -135,7 +140,8 @@ def alloc_workspace(p: Params, op: int, device="cuda") -> torch.Tensor:
 
 
 def mosaic_bsa_select(p: Params, q, k, block_idx=None, ws=None, stream=None):
-    _chk_qkv(p, q, k)
+    _chk_qkv(p, q)
+    _chk_qkv(p, k, heads=p.kv_heads)
     if block_idx is None:
         block_idx = torch.empty((p.B, p.H, p.m, p.topk), dtype=torch.int32, device=q.device)
     if ws is None:
@@ -151,7 +157,8 @@ def mosaic_bsa_select(p: Params, q, k, block_idx=None, ws=None, stream=None):
 def mosaic_bsa_select_static(p: Params, q, k, block_idx=None, stream=None):
     """Selection through the entry point that allocates nothing (scratch inside the library image).
     Only `block_idx` is created here when the caller passes none."""
-    _chk_qkv(p, q, k)
+    _chk_qkv(p, q)
+    _chk_qkv(p, k, heads=p.kv_heads)
     if block_idx is None:
         block_idx = torch.empty((p.B, p.H, p.m, p.topk), dtype=torch.int32, device=q.device)
     pc = p.c()
@@ -162,7 +169,8 @@ def mosaic_bsa_select_static(p: Params, q, k, block_idx=None, stream=None):
 
 
 def mosaic_bsa_fwd(p: Params, q, k, v, block_idx, o=None, lse=None, ws=None, stream=None):
-    _chk_qkv(p, q, k, v)
+    _chk_qkv(p, q)
+    _chk_qkv(p, k, v, heads=p.kv_heads)
     if o is None:
         o = torch.empty_like(q)
     if lse is None:
@@ -180,7 +188,8 @@ def mosaic_bsa_fwd(p: Params, q, k, v, block_idx, o=None, lse=None, ws=None, str
 def mosaic_bsa_fwd_branches(p: Params, q, k, v, block_idx, gates, o=None, lse_fg=None, lse_l=None, ws=None, stream=None):
     """Three-branch form: gated sum of the compression, selection and local branches.  `gates` is
     [B, H, N, 3] fp32 (compression, selection, local).  Returns (o, lse_fg, lse_l)."""
-    _chk_qkv(p, q, k, v)
+    _chk_qkv(p, q)
+    _chk_qkv(p, k, v, heads=p.kv_heads)
     if gates.dtype != torch.float32 or not gates.is_contiguous() or tuple(gates.shape) != (p.B, p.H, p.N, 3):
         raise ValueError(f"expected contiguous cuda fp32 gates [{p.B},{p.H},{p.N},3]")
     o = torch.empty_like(q) if o is None else o
@@ -197,10 +206,11 @@ def mosaic_bsa_fwd_branches(p: Params, q, k, v, block_idx, gates, o=None, lse_fg
 
 
 def mosaic_bsa_bwd(p: Params, q, k, v, o, lse, d_o, block_idx, dq=None, dk=None, dv=None, ws=None, stream=None):
-    _chk_qkv(p, q, k, v, o, d_o)
+    _chk_qkv(p, q, o, d_o)
+    _chk_qkv(p, k, v, heads=p.kv_heads)
     dq = torch.empty_like(q) if dq is None else dq
-    dk = torch.empty_like(q) if dk is None else dk
-    dv = torch.empty_like(q) if dv is None else dv
+    dk = torch.empty_like(k) if dk is None else dk
+    dv = torch.empty_like(k) if dv is None else dv
     if ws is None:
         ws = alloc_workspace(p, OP_BWD, q.device)
     pc = p.c()

@@ -31,7 +31,10 @@ int validate(const mosaic_bsa_params* p, Geo* g) {
   const long long U = (long long)p->B * p->H, N = (long long)p->nlat * p->nlon;
   const long long m = (long long)(p->nlat / p->bh) * (p->nlon / p->bw);
   if (U > (1 << 24) || m > (1 << 24) || U * m * cpb > 0x7fffffffll || U * N > (1ll << 40)) return MOSAIC_E_UNSUPPORTED;
+  const int hkv = p->Hkv == 0 ? p->H : p->Hkv;
+  if (hkv <= 0 || p->H % hkv) return MOSAIC_E_INVALID_ARG;
   g->U = (int)U;
+  g->H = p->H; g->Hkv = hkv; g->Ukv = p->B * hkv;
   g->nlat = p->nlat; g->nlon = p->nlon; g->bh = p->bh; g->bw = p->bw;
   g->nbh = p->nlat / p->bh; g->nbw = p->nlon / p->bw; g->m = (int)m;
   g->b = p->bh * p->bw; g->cpb = cpb; g->crows = crows;
@@ -181,7 +184,7 @@ int mosaic_bsa_fwd_branches(const mosaic_bsa_params* p, const void* q, const voi
   HostCtx cp = c;
   cp.g.topk = 0;  // pooling only
   if ((rc = launch_select(cp, q, k, nullptr, pq, pk, nrm, nrm + (size_t)g.U * g.m))) return rc;
-  if ((rc = launch_pool_one(c, v, pv, nrm))) return rc;
+  if ((rc = launch_pool_one(c, v, pv, nrm, g.Ukv))) return rc;
   if ((rc = launch_compress(c, pq, pk, pv, ocg))) return rc;
   // local branch: the neighbourhood only (no selected blocks); work queue in the second word of the status block
   HostCtx cl = c;

@@ -43,8 +43,8 @@ __global__ void __launch_bounds__(kCW * 32) compress_kernel(Geo g, const float* 
   const int tiles = (g.m + TI - 1) / TI;
   const int u = blockIdx.x / tiles, i0 = (blockIdx.x - u * tiles) * TI;
   const float* pq_u = pq + (long long)u * g.m * kD;
-  const float* pk_u = pk + (long long)u * g.m * kD;
-  const float* pv_u = pv + (long long)u * g.m * kD;
+  const float* pk_u = pk + (long long)kv_unit(g, u) * g.m * kD;   // grouped-query attention: the group's key/value head
+  const float* pv_u = pv + (long long)kv_unit(g, u) * g.m * kD;
   const float inv_b = 1.0f / (float)g.b;
   const float sl2 = g.scale_log2 * inv_b * inv_b;  // logits in base-2 units
 

@@ -77,19 +77,20 @@ __device__ __forceinline__ void planner_kv_loop(Smem& sm, const Geo& g, const in
       if (lane == 0) { sm.info[lb % kLists].n = -1; mbar_arrive(s32(&sm.list_full[lb % kLists])); }
       break;
     }
-    // item = 2 * (256-row item) + tile
+    // item = 2 * (256-row item) + tile of a key/value unit
     const int i256 = item >> 1, t = item & 1;
-    const int u = i256 / ipu;
+    const int u = i256 / ipu;  // key/value unit
     int hb4[4], hc4[4];
     const int valid4 = item_halves(g, i256 - u * ipu, hb4, hc4);
     const int hb[2] = {hb4[2 * t], hb4[2 * t + 1]}, hc[2] = {hc4[2 * t], hc4[2 * t + 1]};
     const int valid = (valid4 >> (2 * t)) & 3;
-    int n = 0;
+    const int ratio = g.H / g.Hkv, qu0 = (u / g.Hkv) * g.H + (u - (u / g.Hkv) * g.Hkv) * ratio;
+    int n = 0, qu = qu0;  // qu: the query unit whose connected query blocks are being listed
     auto publish = [&](int more) {
       const int buf = lb % kLists;
       if (lane == 0) {
         ItemInfo& inf = sm.info[buf];
-        inf.n = n; inf.unit = u; inf.hvalid = valid; inf.more = more;
+        inf.n = n; inf.unit = qu; inf.kvunit = u; inf.hvalid = valid; inf.more = more;
         inf.hb[0] = hb[0]; inf.hb[1] = hb[1]; inf.hc[0] = hc[0]; inf.hc[1] = hc[1];
       }
       __syncwarp();
@@ -101,34 +102,44 @@ __device__ __forceinline__ void planner_kv_loop(Smem& sm, const Geo& g, const in
     const bool same = (valid == 3) && hb[0] == hb[1];
     const unsigned char bits0 = same ? 3 : 1, bits1 = 2;
     const bool use0 = (valid & 1) != 0, use1 = (valid & 2) != 0 && !same;
-    // local neighbourhoods (at most 64 entries per block, merged with masks), straight into the list buffer
-    if (use0) n = merge_block(g, -1, hb[0], bits0, sm.ids[lb % kLists], sm.mask[lb % kLists], n, lane, status);
-    if (use1) n = merge_block(g, -1, hb[1], bits1, sm.ids[lb % kLists], sm.mask[lb % kLists], n, lane, status);
-    // query blocks that selected the key block (ascending ids), appended 32 at a time
-    const int32_t* off = csr_off + (long long)u * (g.m + 1);
-    const int32_t* sel = csr_q + (long long)u * g.m * g.topk;
-#pragma unroll
-    for (int hh = 0; hh < 2 && ok; ++hh) {
-      if (!(hh == 0 ? use0 : use1)) continue;
-      const unsigned char bits = hh == 0 ? bits0 : bits1;
-      const int s_beg = __ldg(off + hb[hh]), s_end = __ldg(off + hb[hh] + 1);
-      for (int base = s_beg; base < s_end && ok; base += 32) {
-        if (n + 32 > kMaxUnion) {
-          publish(1);
-          acquire();
-          if (!ok) break;
-        }
-        const int e = base + lane;
-        if (e < s_end) {
-          sm.ids[lb % kLists][n + lane] = __ldg(sel + e);
-          sm.mask[lb % kLists][n + lane] = bits;
-        }
-        n += min(32, s_end - base);
-        __syncwarp();
+    // One pass per query head of the group (grouped-query attention: the tile's dK and dV sum over them); the
+    // passes are list buffers of the same item, chained by `more`.
+    for (int r = 0; r < ratio && ok; ++r) {
+      qu = qu0 + r;
+      if (r > 0) {
+        acquire();
+        if (!ok) break;
       }
+      // local neighbourhoods (at most 64 entries per block, merged with masks), straight into the list buffer
+      if (use0) n = merge_block(g, -1, hb[0], bits0, sm.ids[lb % kLists], sm.mask[lb % kLists], n, lane, status);
+      if (use1) n = merge_block(g, -1, hb[1], bits1, sm.ids[lb % kLists], sm.mask[lb % kLists], n, lane, status);
+      // query blocks that selected the key block (ascending ids), appended 32 at a time
+      const int32_t* off = csr_off + (long long)qu * (g.m + 1);
+      const int32_t* sel = csr_q + (long long)qu * g.m * g.topk;
+#pragma unroll
+      for (int hh = 0; hh < 2 && ok; ++hh) {
+        if (!(hh == 0 ? use0 : use1)) continue;
+        const unsigned char bits = hh == 0 ? bits0 : bits1;
+        const int s_beg = __ldg(off + hb[hh]), s_end = __ldg(off + hb[hh] + 1);
+        for (int base = s_beg; base < s_end && ok; base += 32) {
+          if (n + 32 > kMaxUnion) {
+            publish(1);
+            acquire();
+            if (!ok) break;
+          }
+          const int e = base + lane;
+          if (e < s_end) {
+            sm.ids[lb % kLists][n + lane] = __ldg(sel + e);
+            sm.mask[lb % kLists][n + lane] = bits;
+          }
+          n += min(32, s_end - base);
+          __syncwarp();
+        }
+      }
+      if (!ok) break;
+      publish(r + 1 < ratio ? 1 : 0);
     }
     if (!ok) break;
-    publish(0);
   }
 }
 
@@ -198,9 +209,9 @@ __global__ void __launch_bounds__(kThreads, 1)
           for (int hh = 0; hh < 2; ++hh) {
             const int by = inf.hb[hh] / g.nbw, bx = inf.hb[hh] - by * g.nbw;
             tma_load_4d(s32(sm.k + hh * kTile), &map_k, s32(&sm.kv_full), 0, bx * g.bw,
-                        by * g.bh + inf.hc[hh] * g.crows, u);
+                        by * g.bh + inf.hc[hh] * g.crows, inf.kvunit);
             tma_load_4d(s32(sm.v + hh * kTile), &map_v, s32(&sm.kv_full), 0, bx * g.bw,
-                        by * g.bh + inf.hc[hh] * g.crows, u);
+                        by * g.bh + inf.hc[hh] * g.crows, inf.kvunit);
           }
           ++items;
         }
@@ -411,7 +422,7 @@ __global__ void __launch_bounds__(kThreads, 1)
           if (!ok) break;
           tc_fence_after();
           if ((sm.info[buf].hvalid >> hh) & 1) {
-            const long long tok = (long long)sm.info[buf].unit * g.N +
+            const long long tok = (long long)sm.info[buf].kvunit * g.N +
                                   chunk_token(g, sm.info[buf].hb[hh], sm.info[buf].hc[hh], (quad & 1) * 32 + lane);
 #pragma unroll
             for (int which = 0; which < 2; ++which) {  // 0: dK (scaled), 1: dV
@@ -451,7 +462,7 @@ int launch_dkdv_tc(const HostCtx& c, const void* q, const void* k, const void* v
                    void* dv, int* work_counter) {
   const Geo& g = c.g;
   CUtensorMap mq, mdo, mk, mv, mnl, mnd;
-  if (!make_map(&mq, q, g) || !make_map(&mdo, d_o, g) || !make_map(&mk, k, g) || !make_map(&mv, v, g) ||
+  if (!make_map(&mq, q, g, g.U) || !make_map(&mdo, d_o, g, g.U) || !make_map(&mk, k, g, g.Ukv) || !make_map(&mv, v, g, g.Ukv) ||
       !make_map_rows(&mnl, neg_lse2, g) || !make_map_rows(&mnd, neg_d, g))
     return MOSAIC_E_CUDA;
   const size_t smem = sizeof(Smem) + 1024;
@@ -459,7 +470,7 @@ int launch_dkdv_tc(const HostCtx& c, const void* q, const void* k, const void* v
   int sms = 0;
   if (const int rc = launch_setup(reinterpret_cast<const void*>(dkdv_tc_kernel), smem, &configured, &sms)) return rc;
   const int ipu = items_per_unit(g);
-  const long long total = 2ll * g.U * ipu;  // one item per 128-row tile
+  const long long total = 2ll * g.Ukv * ipu;  // one item per 128-row tile of a key/value unit
   if (total > 0x7fffff00ll) return MOSAIC_E_UNSUPPORTED;
   const long long grid = total < (long long)sms ? total : (long long)sms;
   dkdv_tc_kernel<<<(unsigned)grid, kThreads, smem, c.stream>>>(g, mq, mdo, mk, mv, mnl, mnd, csr_off, csr_q,

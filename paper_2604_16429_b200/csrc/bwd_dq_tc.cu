@@ -100,6 +100,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         const ItemInfo& inf = sm.info[buf];
         const int n = inf.n, u = inf.unit;
         if (n < 0) break;
+        const int ukv = kv_unit(g, u);  // key/value head of this query head's group
         // Q and dO tiles: free once the tile's last S / dP products of the previous item have completed
         for (int t = 0; t < 2 && ok; ++t) {
           ok = mbar_wait(s32(&sm.q_empty[t]), (it & 1) ^ 1, abort, status);
@@ -120,8 +121,8 @@ __global__ void __launch_bounds__(kThreads, 1)
             ok = mbar_wait(s32(&sm.kv_empty[st]), (uint32_t)((step / kStages) & 1) ^ 1, abort, status);
             if (!ok) break;
             mbar_expect_tx(s32(&sm.kv_full[st]), 2 * kTile);
-            tma_load_4d(s32(sm.kv[st][0]), &map_k, s32(&sm.kv_full[st]), 0, bx * g.bw, by * g.bh + c * g.crows, u);
-            tma_load_4d(s32(sm.kv[st][1]), &map_v, s32(&sm.kv_full[st]), 0, bx * g.bw, by * g.bh + c * g.crows, u);
+            tma_load_4d(s32(sm.kv[st][0]), &map_k, s32(&sm.kv_full[st]), 0, bx * g.bw, by * g.bh + c * g.crows, ukv);
+            tma_load_4d(s32(sm.kv[st][1]), &map_v, s32(&sm.kv_full[st]), 0, bx * g.bw, by * g.bh + c * g.crows, ukv);
           }
         }
         if (ok) mbar_arrive(s32(&sm.list_empty[buf]));
@@ -333,7 +334,7 @@ int launch_dq_tc(const HostCtx& c, const void* q, const void* k, const void* v, 
                  const float* D, const int32_t* block_idx, void* dq, int* work_counter) {
   const Geo& g = c.g;
   CUtensorMap mq, mdo, mk, mv;
-  if (!make_map(&mq, q, g) || !make_map(&mdo, d_o, g) || !make_map(&mk, k, g) || !make_map(&mv, v, g))
+  if (!make_map(&mq, q, g, g.U) || !make_map(&mdo, d_o, g, g.U) || !make_map(&mk, k, g, g.Ukv) || !make_map(&mv, v, g, g.Ukv))
     return MOSAIC_E_CUDA;
   const size_t smem = sizeof(Smem) + 1024;
   static unsigned long long configured = 0;  // devices on which the kernel's shared-memory opt-in is set

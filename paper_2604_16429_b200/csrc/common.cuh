@@ -16,6 +16,8 @@ constexpr int kStatusBytes = 256; // status block at the start of every workspac
 // Geometry of one call, passed by value to the kernels.
 struct Geo {
   int U;            // B*H independent units
+  int H, Hkv;       // query heads, key/value heads (grouped-query attention: H / Hkv query heads share a key/value head)
+  int Ukv;          // B*Hkv key/value units
   int nlat, nlon;   // grid
   int bh, bw;       // block shape
   int nbh, nbw, m;  // blocks per column / row / unit
@@ -29,6 +31,12 @@ struct Geo {
   float scale_log2; // scale * log2(e)
   long long N;      // tokens per unit
 };
+
+// key/value unit read by query unit u
+__host__ __device__ __forceinline__ int kv_unit(const Geo& g, int u) {
+  const int b = u / g.H;
+  return b * g.Hkv + (u - b * g.H) / (g.H / g.Hkv);
+}
 
 // Record the first device-side fault in the workspace status word (never traps).
 __device__ __forceinline__ void set_status(int* status, int code) { atomicCAS(status, 0, code); }
@@ -97,7 +105,7 @@ int launch_fwd_tc(const HostCtx& c, const void* q, const void* k, const void* v,
 // Layout of the three-branch forward's scratch behind the status block
 struct BranchWs { size_t pq, pk, pv, nrm, ocg, ofg, ol, total; };
 BranchWs branch_layout(const Geo& g);
-int launch_pool_one(const HostCtx& c, const void* x, float* pooled, float* norm_scratch);
+int launch_pool_one(const HostCtx& c, const void* x, float* pooled, float* norm, int units);
 int launch_compress(const HostCtx& c, const float* pooled_q, const float* pooled_k, const float* pooled_v, float* ocg);
 int launch_combine(const HostCtx& c, const float* ocg, const void* o_fg, const void* o_l, const float* gates, void* o);
 int launch_dq_tc(const HostCtx& c, const void* q, const void* k, const void* v, const void* d_o, const float* lse,

@@ -128,6 +128,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         const ItemInfo& inf = sm.info[buf];
         const int n = inf.n, u = inf.unit;
         if (n < 0) break;
+        const int ukv = kv_unit(g, u);  // key/value head of this query head's group
         // query tiles (double-buffered by item parity): free once the softmax threads have copied the rows of
         // the item before the previous one to TMEM, so this load runs while the previous item still computes
         for (int t = 0; t < 2 && ok; ++t) {
@@ -148,8 +149,8 @@ __global__ void __launch_bounds__(kThreads, 1)
             ok = mbar_wait(s32(&sm.kv_empty[st]), (uint32_t)((step / kStages) & 1) ^ 1, abort, status);
             if (!ok) break;
             mbar_expect_tx(s32(&sm.kv_full[st]), 2 * kTile);
-            tma_load_4d(s32(sm.kv[st][0]), &map_k, s32(&sm.kv_full[st]), 0, bx * g.bw, by * g.bh + c * g.crows, u);
-            tma_load_4d(s32(sm.kv[st][1]), &map_v, s32(&sm.kv_full[st]), 0, bx * g.bw, by * g.bh + c * g.crows, u);
+            tma_load_4d(s32(sm.kv[st][0]), &map_k, s32(&sm.kv_full[st]), 0, bx * g.bw, by * g.bh + c * g.crows, ukv);
+            tma_load_4d(s32(sm.kv[st][1]), &map_v, s32(&sm.kv_full[st]), 0, bx * g.bw, by * g.bh + c * g.crows, ukv);
             // a tile that does not attend this entry never looks at the stage: its release is given here (the other
             // tile's release, after its P V, is what lets the stage be reused)
             if (!(mk & 3u)) mbar_arrive(s32(&sm.kv_empty[st]));
@@ -452,7 +453,7 @@ int launch_fwd_tc(const HostCtx& c, const void* q, const void* k, const void* v,
                   float* lse, int* work_counter) {
   const Geo& g = c.g;
   CUtensorMap mq, mk, mv;
-  if (!make_map(&mq, q, g) || !make_map(&mk, k, g) || !make_map(&mv, v, g)) return MOSAIC_E_CUDA;
+  if (!make_map(&mq, q, g, g.U) || !make_map(&mk, k, g, g.Ukv) || !make_map(&mv, v, g, g.Ukv)) return MOSAIC_E_CUDA;
   const size_t smem = sizeof(Smem) + 1024;
   static unsigned long long configured = 0;  // devices on which the kernel's shared-memory opt-in is set
   int sms = 0;

@@ -23,10 +23,10 @@ namespace mosaic {
 template <int BW>
 __global__ void __launch_bounds__(256) pool_kernel(Geo g, const uint4* __restrict__ q, const uint4* __restrict__ k,
                                                    float* __restrict__ pq, float* __restrict__ pk,
-                                                   float* __restrict__ nq, float* __restrict__ nk, int ntens) {
+                                                   float* __restrict__ nq, float* __restrict__ nk, int ntens, int units) {
   const int sub = threadIdx.x & 7;  // which 8 channels
   const long long grp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 3;
-  const long long per_tensor = (long long)g.U * g.m;
+  const long long per_tensor = (long long)units * g.m;
   const bool live = grp < ntens * per_tensor;  // the last warp may be partly idle; it still takes part in the shuffles
   const int which = live && grp >= per_tensor;
   const long long w = live ? grp - which * per_tensor : 0;
@@ -205,8 +205,8 @@ __global__ void __launch_bounds__(NW * 32, MB) topk_kernel(Geo g, const float* _
   const int tiles = (g.m + TI - 1) / TI;
   const int u = blockIdx.x / tiles, i0 = (blockIdx.x - u * tiles) * TI;
   const float* pq_u = pq + (long long)u * g.m * kD;
-  const float* pk_u = pk + (long long)u * g.m * kD;
-  const float* nk_u = nk + (long long)u * g.m;
+  const float* pk_u = pk + (long long)kv_unit(g, u) * g.m * kD;   // grouped-query attention: the group's key head
+  const float* nk_u = nk + (long long)kv_unit(g, u) * g.m;
   const int nchunks = (g.m + JT - 1) / JT;
 
   auto load_chunk = [&](int ch, int buf) {
@@ -516,32 +516,34 @@ int launch_topk(const HostCtx& c, const float* pooled_q, const float* pooled_k, 
   return cudaGetLastError() == cudaSuccess ? MOSAIC_OK : MOSAIC_E_CUDA;
 }
 
-// block sums of one more tensor (the values, for the compression branch of the three-branch form)
-int launch_pool_one(const HostCtx& c, const void* x, float* pooled, float* norm_scratch) {
+// block sums (and norm bounds) of one tensor of `units` units
+int launch_pool_one(const HostCtx& c, const void* x, float* pooled, float* norm, int units) {
   const Geo& g = c.g;
-  const long long threads = 1ll * g.U * g.m * 8;
+  const long long threads = 1ll * units * g.m * 8;
   const unsigned blocks = (unsigned)((threads + 255) / 256);
   if (g.bw == 8)
-    pool_kernel<8><<<blocks, 256, 0, c.stream>>>(g, (const uint4*)x, (const uint4*)x, pooled, pooled, norm_scratch,
-                                                 norm_scratch, 1);
+    pool_kernel<8><<<blocks, 256, 0, c.stream>>>(g, (const uint4*)x, (const uint4*)x, pooled, pooled, norm, norm, 1, units);
   else
-    pool_kernel<16><<<blocks, 256, 0, c.stream>>>(g, (const uint4*)x, (const uint4*)x, pooled, pooled, norm_scratch,
-                                                  norm_scratch, 1);
+    pool_kernel<16><<<blocks, 256, 0, c.stream>>>(g, (const uint4*)x, (const uint4*)x, pooled, pooled, norm, norm, 1, units);
   return cudaGetLastError() == cudaSuccess ? MOSAIC_OK : MOSAIC_E_CUDA;
 }
 
 int launch_select(const HostCtx& c, const void* q, const void* k, int32_t* block_idx, float* pooled_q,
                   float* pooled_k, float* norm_q, float* norm_k) {
   const Geo& g = c.g;
-  {
+  if (g.Ukv != g.U) {  // grouped-query attention: Q and K have different head counts, one launch each
+    int rc = launch_pool_one(c, q, pooled_q, norm_q, g.U);
+    if (!rc) rc = launch_pool_one(c, k, pooled_k, norm_k, g.Ukv);
+    if (rc) return rc;
+  } else {
     const long long threads = 2ll * g.U * g.m * 8;
     const unsigned blocks = (unsigned)((threads + 255) / 256);
     if (g.bw == 8)
       pool_kernel<8><<<blocks, 256, 0, c.stream>>>(g, (const uint4*)q, (const uint4*)k, pooled_q, pooled_k, norm_q,
-                                                   norm_k, 2);
+                                                   norm_k, 2, g.U);
     else
       pool_kernel<16><<<blocks, 256, 0, c.stream>>>(g, (const uint4*)q, (const uint4*)k, pooled_q, pooled_k, norm_q,
-                                                    norm_k, 2);
+                                                    norm_k, 2, g.U);
     if (cudaGetLastError() != cudaSuccess) return MOSAIC_E_CUDA;
   }
   if (g.topk > 0) {

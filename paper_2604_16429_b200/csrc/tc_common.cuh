@@ -28,6 +28,7 @@ struct ItemInfo {
   int hb[4];    // query block of half h
   int hc[4];    // 64-token chunk of that block
   int more;     // 1: the item's list continues in the next list buffer (lists longer than a buffer)
+  int kvunit;   // key-stationary kernel: the key/value unit of the item's tile (`unit` is the query unit of this buffer's list)
 };
 
 __device__ __forceinline__ uint32_t s32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -557,8 +558,8 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
 // ---- host side (tmap.cu) -------------------------------------------------------------------
 // TMA descriptors are cached per (device, base pointer, geometry), so a call that sees the same tensors
 // again encodes nothing.
-// [U, nlat, nlon, d] bf16 view, box = one 64-token chunk {d, bw, 64/bw, 1}, 128-byte swizzle.
-bool make_map(CUtensorMap* map, const void* base, const Geo& g);
+// [units, nlat, nlon, d] bf16 view, box = one 64-token chunk {d, bw, 64/bw, 1}, 128-byte swizzle.
+bool make_map(CUtensorMap* map, const void* base, const Geo& g, int units);
 // [U, nlat, nlon] fp32 view (one value per token), box = the 64 tokens of one chunk {bw, 64/bw, 1}, no swizzle.
 bool make_map_rows(CUtensorMap* map, const void* base, const Geo& g);
 // Current device, its SM count (cached), and the opt-in to `smem` bytes of dynamic shared memory for `func`

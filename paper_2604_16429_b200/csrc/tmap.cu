@@ -47,13 +47,13 @@ struct MapCache {
 MapCache g_cache;
 std::atomic<long long> g_encodes{0};
 
-bool encode(CUtensorMap* map, const MapKey& k, const Geo& g) {
+bool encode(CUtensorMap* map, const MapKey& k, const Geo& g) {  // k.U units
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   g_encodes.fetch_add(1, std::memory_order_relaxed);
   void* base = const_cast<void*>(k.base);
   if (k.kind == 0) {
-    cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)g.nlon, (cuuint64_t)g.nlat, (cuuint64_t)g.U};
+    cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)g.nlon, (cuuint64_t)g.nlat, (cuuint64_t)k.U};
     cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)g.nlon * kD * 2, (cuuint64_t)g.N * kD * 2};
     cuuint32_t box[4] = {(cuuint32_t)kD, (cuuint32_t)g.bw, (cuuint32_t)g.crows, 1u};
     cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
@@ -61,7 +61,7 @@ bool encode(CUtensorMap* map, const MapKey& k, const Geo& g) {
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
   }
-  cuuint64_t dims[3] = {(cuuint64_t)g.nlon, (cuuint64_t)g.nlat, (cuuint64_t)g.U};
+  cuuint64_t dims[3] = {(cuuint64_t)g.nlon, (cuuint64_t)g.nlat, (cuuint64_t)k.U};
   cuuint64_t strides[2] = {(cuuint64_t)g.nlon * 4, (cuuint64_t)g.N * 4};
   cuuint32_t box[3] = {(cuuint32_t)g.bw, (cuuint32_t)g.crows, 1u};
   cuuint32_t estr[3] = {1u, 1u, 1u};
@@ -70,10 +70,10 @@ bool encode(CUtensorMap* map, const MapKey& k, const Geo& g) {
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-bool cached_map(CUtensorMap* out, const void* base, const Geo& g, int kind) {
+bool cached_map(CUtensorMap* out, const void* base, const Geo& g, int kind, int units) {
   MapKey k;
   if (cudaGetDevice(&k.dev) != cudaSuccess) return false;
-  k.kind = kind; k.U = g.U; k.nlat = g.nlat; k.nlon = g.nlon; k.bw = g.bw; k.crows = g.crows; k.base = base;
+  k.kind = kind; k.U = units; k.nlat = g.nlat; k.nlon = g.nlon; k.bw = g.bw; k.crows = g.crows; k.base = base;
   std::lock_guard<std::mutex> hold(g_cache.lock);
   for (int s = 0; s < kCacheSlots; ++s)
     if (g_cache.used[s] && g_cache.key[s] == k) { *out = g_cache.map[s]; return true; }
@@ -89,8 +89,8 @@ std::atomic<int> g_sms[kMaxDevices];
 
 }  // namespace
 
-bool make_map(CUtensorMap* map, const void* base, const Geo& g) { return cached_map(map, base, g, 0); }
-bool make_map_rows(CUtensorMap* map, const void* base, const Geo& g) { return cached_map(map, base, g, 1); }
+bool make_map(CUtensorMap* map, const void* base, const Geo& g, int units) { return cached_map(map, base, g, 0, units); }
+bool make_map_rows(CUtensorMap* map, const void* base, const Geo& g) { return cached_map(map, base, g, 1, g.U); }
 
 int launch_setup(const void* func, size_t smem, unsigned long long* done, int* sms) {
   int dev = 0;

@@ -44,6 +44,7 @@ class Workload:
     rlat: int = 1
     rlon: int = 1
     local_groups: bool = False   # local set = aligned group of rlat x rlon blocks (the paper's large local blocks)
+    Hkv: int = 0                 # heads of K and V (grouped-query attention); 0 = H
 
     @property
     def N(self): return self.nlat * self.nlon
@@ -53,6 +54,8 @@ class Workload:
     def b(self): return self.bh * self.bw
     @property
     def U(self): return self.B * self.H
+    @property
+    def kv_heads(self): return self.Hkv or self.H
 
 
 WORKLOADS = {
@@ -67,6 +70,8 @@ WORKLOADS = {
     "hp_nside64": Workload("hp_nside64", 6, 1, 12, 3072, 16, 8, 16, 24, "smooth", rlat=8, rlon=1, local_groups=True),
     "hp_nside32": Workload("hp_nside32", 7, 1, 16, 768, 16, 8, 16, 12, "smooth", rlat=8, rlon=1, local_groups=True),
     "hp_nside16": Workload("hp_nside16", 8, 1, 20, 192, 16, 8, 16, 4, "smooth", rlat=8, rlon=1, local_groups=True),
+    # stage 1 with the paper's grouped-query attention (ratio 4): 12 query heads on 3 key/value heads
+    "hp_nside64_gqa": Workload("hp_nside64_gqa", 9, 1, 12, 3072, 16, 8, 16, 24, "smooth", rlat=8, rlon=1, local_groups=True, Hkv=3),
 }
 
 
@@ -111,17 +116,17 @@ def make_inputs(w: Workload, with_do: bool | None = None) -> dict:
     """Q, K, V (and dO when the workload trains) as uint16 bf16 bits [B,H,N,d]."""
     base = 1000 * w.cfg
     if w.kind == "iid":
-        gen = lambda s: iid_normal(w.B, w.H, w.N, w.d, s)
+        gen = lambda s, h=w.H: iid_normal(w.B, h, w.N, w.d, s)
     else:
-        gen = lambda s: smooth_plus_noise(w.B, w.H, w.nlat, w.nlon, w.d, s)
-    out = {"q": gen(base + 0), "k": gen(base + 1), "v": gen(base + 2)}
+        gen = lambda s, h=w.H: smooth_plus_noise(w.B, h, w.nlat, w.nlon, w.d, s)
+    out = {"q": gen(base + 0), "k": gen(base + 1, w.kv_heads), "v": gen(base + 2, w.kv_heads)}   # K, V: [B, Hkv, N, d]
     if w.backward if with_do is None else with_do:
         out["do"] = iid_normal(w.B, w.H, w.N, w.d, base + 3)
     return out
 
 
 def small_case(nlat, nlon, bh, bw, topk, B=1, H=1, d=64, kind="iid", seed=7, rlat=1, rlon=1, backward=False,
-               local_groups=False):
+               local_groups=False, Hkv=0):
     """A free-form small workload for tests (cfg number = seed)."""
-    return Workload(f"small_{nlat}x{nlon}_{bh}x{bw}_k{topk}" + ("_groups" if local_groups else ""), seed, B, H, nlat,
-                    nlon, bh, bw, topk, kind, backward, d, rlat, rlon, local_groups)
+    return Workload(f"small_{nlat}x{nlon}_{bh}x{bw}_k{topk}" + ("_groups" if local_groups else "") + (f"_kv{Hkv}" if Hkv else ""),
+                    seed, B, H, nlat, nlon, bh, bw, topk, kind, backward, d, rlat, rlon, local_groups, Hkv)

@@ -11,7 +11,7 @@
 // each half one 64-token chunk of a key block; tile t of the 256-row items the other kernels use).  The K
 // and V tiles stay in shared memory; query-side chunks (Q, dO, and per query row -LSE*log2(e) and -D)
 // stream through a ring.  Per product:  S^T = K Q^T and dP^T = V dO^T (eight MMAs into two 64-column TMEM
-// buffers); the row threads (TMEM lane = key row, two threads per row, each half of the query columns; the
+// buffers); the row threads (TMEM lane = key row, four threads per row, each a quarter of the query columns; the
 // backward has no reduction along a row, so they never talk) pull their share into registers and hand the
 // buffers back at once, so the next product's S^T and dP^T are computed while they form P^T and dS^T (bf16,
 // own TMEM columns); then dV += P^T dO and dK += dS^T Q (TMEM A operands, the staged dO and Q chunks as
@@ -28,10 +28,13 @@ namespace mosaic {
 namespace {
 
 constexpr int kStages = 6;       // ring depth of query-side chunks
-constexpr int kThreads = 384;    // warps 0-7 row threads, 8 TMA producer, 9 and 10 MMA issuers, 11 planner
+constexpr int kRowWarps = 16;    // two groups of eight: two threads per key row in each
+constexpr int kThreads = 32 * (kRowWarps + 4);  // row threads, then TMA producer, two MMA issuers, planner
+constexpr int kWProd = kRowWarps, kWMma0 = kRowWarps + 1, kWMma1 = kRowWarps + 2, kWPlan = kRowWarps + 3;
+constexpr int kGroupWarps = kRowWarps / 2;  // row-thread warps of one group (products alternate between two groups)
 constexpr uint32_t kTmemCols = 512;
-// dK, dV accumulators; S^T and dP^T (fp32); P^T and dS^T (bf16 pairs)
-constexpr uint32_t kColDK = 0, kColDV = 64, kColS = 128, kColDP = 192, kColP = 256, kColDS = 288;
+// dK, dV accumulators; two buffers each of S^T and dP^T (fp32, 64 columns) and of P^T and dS^T (bf16 pairs, 32 columns)
+constexpr uint32_t kColDK = 0, kColDV = 64, kColS = 128, kColDP = 256, kColP = 384, kColDS = 448;
 constexpr uint32_t kStageBytes = 2 * kTile + 2 * 64 * 4;
 
 struct Stage {
@@ -47,7 +50,7 @@ struct Smem {
   unsigned char v[2 * kTile];
   Stage ring[kStages];
   unsigned long long ring_full[kStages], ring_empty[kStages];
-  unsigned long long kv_full, kv_empty, s_full, sdp_free, p_full, pv_done;
+  unsigned long long kv_full, kv_empty, s_full[2], sdp_free[2], p_full[2], pv_done[2], acc_done, acc_free;
   unsigned long long list_full[kLists], list_empty[kLists];
   uint32_t tmem_base;
   int abort;
@@ -160,20 +163,24 @@ __global__ void __launch_bounds__(kThreads, 1)
     for (int s = 0; s < kStages; ++s) { mbar_init(s32(&sm.ring_full[s]), 1); mbar_init(s32(&sm.ring_empty[s]), 1); }
     mbar_init(s32(&sm.kv_full), 1);
     mbar_init(s32(&sm.kv_empty), 1);
-    mbar_init(s32(&sm.s_full), 1);
-    mbar_init(s32(&sm.sdp_free), 256);
-    mbar_init(s32(&sm.p_full), 256);
-    mbar_init(s32(&sm.pv_done), 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(s32(&sm.s_full[b]), 1);
+      mbar_init(s32(&sm.sdp_free[b]), 32 * kGroupWarps);
+      mbar_init(s32(&sm.p_full[b]), 32 * kGroupWarps);
+      mbar_init(s32(&sm.pv_done[b]), 1);
+    }
+    mbar_init(s32(&sm.acc_done), 1);
+    mbar_init(s32(&sm.acc_free), kRowWarps);
     for (int i = 0; i < kLists; ++i) {
       mbar_init(s32(&sm.list_full[i]), 1);
-      mbar_init(s32(&sm.list_empty[i]), 11);  // 8 row-thread warps + 2 MMA issuers + TMA producer
+      mbar_init(s32(&sm.list_empty[i]), kRowWarps + 3);  // row-thread warps + 2 MMA issuers + TMA producer
     }
     sm.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   __syncthreads();
-  if (warp == 9) {
+  if (warp == kWMma0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(&sm.tmem_base)),
                  "r"(kTmemCols)
                  : "memory");
@@ -186,9 +193,9 @@ __global__ void __launch_bounds__(kThreads, 1)
   const uint32_t tmem = sm.tmem_base;
   volatile int* abort = &sm.abort;
 
-  if (warp == 11) {
+  if (warp == kWPlan) {
     planner_kv_loop(sm, g, csr_off, csr_q, work_counter, ipu, total_items, lane, abort, status);
-  } else if (warp == 8) {
+  } else if (warp == kWProd) {
     // ------------------------------------------------------------- TMA producer
     if (lane == 0) {
       long long step = 0;  // query-side chunks issued so far (ring position)
@@ -243,15 +250,15 @@ __global__ void __launch_bounds__(kThreads, 1)
           if (!mbar_wait(s32(&sm.ring_empty[s % kStages]), (uint32_t)((s / kStages) & 1), abort, status)) break;
       }
     }
-  } else if (warp == 9) {
+  } else if (warp == kWMma0) {
     // ------------------------------------------------------------- issuer of S^T = K Q^T and dP^T = V dO^T (one thread)
-    // A thread issues an N = 64 product no faster than one in about 50 cycles; the sixteen products of a step are
-    // split over two issuing threads (this one and warp 10), which are ordered by barriers only.
+    // Product n goes to buffer n & 1.  A buffer may be overwritten once its row threads hold the product before
+    // last in registers, so this thread runs up to two products ahead of the row threads.
     if (lane == 0) {
       constexpr uint32_t idesc_nt = make_idesc(false);
       const uint64_t kdesc = smem_desc(s32(sm.k)), vdesc = smem_desc(s32(sm.v));
       long long step = 0;   // ring position
-      uint32_t nt = 0;      // products started so far (phase of the per-product barriers)
+      uint32_t nt = 0;      // products started so far (buffer and phase of the per-product barriers)
       int items = 0;
       bool ok = true, fresh = true;
       for (int lb = 0; ok; ++lb) {
@@ -270,17 +277,19 @@ __global__ void __launch_bounds__(kThreads, 1)
         for (int e = 0; e < n && ok; ++e) {
           for (int c = 0; c < g.cpb && ok; ++c, ++step) {
             const int st = (int)(step % kStages);
+            const uint32_t b = nt & 1, j = nt >> 1;
             ok = mbar_wait(s32(&sm.ring_full[st]), (uint32_t)((step / kStages) & 1), abort, status);
-            // S^T and dP^T may be overwritten once the row threads hold the previous product in registers
-            if (ok && nt > 0) ok = mbar_wait(s32(&sm.sdp_free), (nt - 1) & 1, abort, status);
+            if (ok && j > 0) ok = mbar_wait(s32(&sm.sdp_free[b]), (j - 1) & 1, abort, status);
             if (!ok) break;
             tc_fence_after();
             const uint64_t qdesc = smem_desc(s32(sm.ring[st].q)), dodesc = smem_desc(s32(sm.ring[st].d_o));
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) umma_ss(tmem + kColS, kdesc + 2 * kk, qdesc + 2 * kk, idesc_nt, kk > 0);
+            for (int kk = 0; kk < 4; ++kk)
+              umma_ss(tmem + kColS + 64 * b, kdesc + 2 * kk, qdesc + 2 * kk, idesc_nt, kk > 0);
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) umma_ss(tmem + kColDP, vdesc + 2 * kk, dodesc + 2 * kk, idesc_nt, kk > 0);
-            tc_commit(s32(&sm.s_full));
+            for (int kk = 0; kk < 4; ++kk)
+              umma_ss(tmem + kColDP + 64 * b, vdesc + 2 * kk, dodesc + 2 * kk, idesc_nt, kk > 0);
+            tc_commit(s32(&sm.s_full[b]));
             ++nt;
           }
         }
@@ -289,12 +298,13 @@ __global__ void __launch_bounds__(kThreads, 1)
         if (ok) mbar_arrive(s32(&sm.list_empty[buf]));
       }
     }
-  } else if (warp == 10) {
+  } else if (warp == kWMma1) {
     // ------------------------------------------------------------- issuer of dV += P^T dO and dK += dS^T Q (one thread)
     if (lane == 0) {
       constexpr uint32_t idesc_nn = make_idesc(true);
       long long step = 0;
       uint32_t nt = 0;
+      uint32_t items = 0;   // items whose accumulators have been handed to the row threads
       bool ok = true, first = true;
       for (int lb = 0; ok; ++lb) {
         const int buf = lb % kLists;
@@ -306,43 +316,57 @@ __global__ void __launch_bounds__(kThreads, 1)
         for (int e = 0; e < n && ok; ++e) {
           for (int c = 0; c < g.cpb && ok; ++c, ++step) {
             const int st = (int)(step % kStages);
+            const uint32_t b = nt & 1, j = nt >> 1;
             // the stage landed before S^T could be produced; this wait makes the copied Q and dO visible here too
             ok = mbar_wait(s32(&sm.ring_full[st]), (uint32_t)((step / kStages) & 1), abort, status);
-            if (ok) ok = mbar_wait(s32(&sm.p_full), nt & 1, abort, status);
+            if (ok) ok = mbar_wait(s32(&sm.p_full[b]), j & 1, abort, status);
+            // a new accumulation overwrites dK and dV: every row thread must have read the previous item's
+            if (ok && first && items > 0) ok = mbar_wait(s32(&sm.acc_free), (items - 1) & 1, abort, status);
             if (!ok) break;
             tc_fence_after();
             const uint64_t qmn = smem_desc(s32(sm.ring[st].q)), domn = smem_desc(s32(sm.ring[st].d_o));
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)
-              umma_ts(tmem + kColDV, tmem + kColP + 8 * kk, domn + (uint64_t)((2048 * kk) >> 4), idesc_nn,
+              umma_ts(tmem + kColDV, tmem + kColP + 32 * b + 8 * kk, domn + (uint64_t)((2048 * kk) >> 4), idesc_nn,
                       (!first || kk > 0));
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)
-              umma_ts(tmem + kColDK, tmem + kColDS + 8 * kk, qmn + (uint64_t)((2048 * kk) >> 4), idesc_nn,
+              umma_ts(tmem + kColDK, tmem + kColDS + 32 * b + 8 * kk, qmn + (uint64_t)((2048 * kk) >> 4), idesc_nn,
                       (!first || kk > 0));
             // the stage's S^T and dP^T completed before P^T could be formed, so this thread's completion frees it
             tc_commit(s32(&sm.ring_empty[st]));
-            tc_commit(s32(&sm.pv_done));
+            tc_commit(s32(&sm.pv_done[b]));
             first = false;
             ++nt;
           }
         }
-        if (!more) first = true;  // the next list buffer starts a new item: new accumulation
+        if (ok && !more && !first) {  // the item's accumulators are complete behind this commit
+          tc_commit(s32(&sm.acc_done));
+          ++items;
+          first = true;
+        }
         if (ok) mbar_arrive(s32(&sm.list_empty[buf]));
       }
     }
-  } else if (warp < 8) {
+  } else if (warp < kRowWarps) {
     // ------------------------------------------------------------- row threads (TMEM lane = key row)
-    const int ch = warp >> 2;        // half of the query columns (and of the output channels) this thread owns
-    const int quad = warp & 3;       // TMEM lane quadrant
-    const int hh = quad >> 1;        // 64-row half of the tile this warp's rows belong to
+    // Two groups of eight warps take the products in turn (product n: group and buffer n & 1), so one group's
+    // waits and TMEM traffic fall into the other's arithmetic.  Inside a group two threads share a key row, each
+    // with half of the query columns.
+    const int grp = warp >> 3;        // products this thread works on: those with n & 1 == grp
+    const int ch = (warp >> 2) & 1;   // half of the query columns
+    const int cq = warp >> 2;         // quarter of the output channels (epilogue)
+    const int quad = warp & 3;        // TMEM lane quadrant
+    const int hh = quad >> 1;         // 64-row half of the tile this warp's rows belong to
     const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
     const uint32_t tb = tmem + lane_off;
     const uint32_t hbit = 1u << hh;
     const uint64_t scale2 = pack2(g.scale_log2, g.scale_log2);
-    uint32_t nt = 0;
+    const uint32_t col_s = kColS + 64 * grp + 32 * ch, col_dp = kColDP + 64 * grp + 32 * ch;
+    const uint32_t col_p = kColP + 32 * grp + 16 * ch, col_ds = kColDS + 32 * grp + 16 * ch;
+    uint32_t nt = 0;     // products seen so far (both groups)
     long long step = 0;  // ring position, to find the stage that holds the query rows' -LSE and -D
-    uint32_t item_done = 0;
+    uint32_t item_steps = 0, items = 0;
     bool ok = true;
     for (int lb = 0; ok; ++lb) {
       const int buf = lb % kLists;
@@ -354,8 +378,10 @@ __global__ void __launch_bounds__(kThreads, 1)
       const bool more = sm.info[buf].more != 0;
       for (int e = 0; e < n && ok; ++e) {
         const bool connected = (sm.mask[buf][e] & hbit) != 0;
-        for (int c = 0; c < g.cpb; ++c, ++step) {
-          ok = mbar_wait(s32(&sm.s_full), nt & 1, abort, status);
+        for (int c = 0; c < g.cpb; ++c, ++step, ++nt, ++item_steps) {
+          if ((int)(nt & 1) != grp) continue;
+          const uint32_t j = nt >> 1;
+          ok = mbar_wait(s32(&sm.s_full[grp]), j & 1, abort, status);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
@@ -369,11 +395,11 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (!ok) break;
             const Stage& sg = sm.ring[st];
             uint32_t sv[32], dp[32];
-            tmem_ld32(tb + kColS + 32 * ch, sv);
-            tmem_ld32(tb + kColDP + 32 * ch, dp);
+            tmem_ld32(tb + col_s, sv);
+            tmem_ld32(tb + col_dp, dp);
             tmem_wait_ld();
             tc_fence_before();
-            mbar_arrive(s32(&sm.sdp_free));  // S^T and dP^T go back to the tensor core
+            mbar_arrive(s32(&sm.sdp_free[grp]));  // S^T and dP^T go back to the tensor core
 #pragma unroll
             for (int i = 0; i < 32; i += 4) {
               // -LSE*log2(e) and -D of four query columns (the same for every thread: broadcast loads)
@@ -394,30 +420,28 @@ __global__ void __launch_bounds__(kThreads, 1)
             }
           } else {
             tc_fence_before();
-            mbar_arrive(s32(&sm.sdp_free));
+            mbar_arrive(s32(&sm.sdp_free[grp]));
 #pragma unroll
             for (int i = 0; i < 16; ++i) { pp[i] = 0u; ds[i] = 0u; }
           }
-          // P^T and dS^T have one buffer each: the previous product's dV / dK updates must have consumed them
-          if (item_done > 0) {
-            ok = mbar_wait(s32(&sm.pv_done), (nt - 1) & 1, abort, status);
+          // this group's P^T and dS^T buffer: its previous dV / dK updates must have consumed it
+          if (j > 0) {
+            ok = mbar_wait(s32(&sm.pv_done[grp]), (j - 1) & 1, abort, status);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
           }
-          tmem_st16(tb + kColP + 16 * ch, pp);
-          tmem_st16(tb + kColDS + 16 * ch, ds);
+          tmem_st16(tb + col_p, pp);
+          tmem_st16(tb + col_ds, ds);
           tmem_wait_st();
           tc_fence_before();
-          mbar_arrive(s32(&sm.p_full));
-          ++nt;
-          ++item_done;
+          mbar_arrive(s32(&sm.p_full[grp]));
         }
       }
       if (!ok) break;
       if (!more) {
-        if (item_done > 0) {
-          ok = mbar_wait(s32(&sm.pv_done), (nt - 1) & 1, abort, status);
+        if (item_steps > 0) {
+          ok = mbar_wait(s32(&sm.acc_done), items & 1, abort, status);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
@@ -426,21 +450,26 @@ __global__ void __launch_bounds__(kThreads, 1)
                                   chunk_token(g, sm.info[buf].hb[hh], sm.info[buf].hc[hh], (quad & 1) * 32 + lane);
 #pragma unroll
             for (int which = 0; which < 2; ++which) {  // 0: dK (scaled), 1: dV
-              uint4* dst = reinterpret_cast<uint4*>((which ? dv : dk) + tok * kD + 32 * ch);
+              uint4* dst = reinterpret_cast<uint4*>((which ? dv : dk) + tok * kD + 16 * cq);
               const float f = which ? 1.f : g.scale;
-              uint32_t ov[32];
-              tmem_ld32(tb + (which ? kColDV : kColDK) + 32 * ch, ov);
+              uint32_t ov[16];
+              tmem_ld16(tb + (which ? kColDV : kColDK) + 16 * cq, ov);
               tmem_wait_ld();
-              uint32_t w[16];
+              uint32_t w[8];
 #pragma unroll
-              for (int i = 0; i < 16; ++i)
+              for (int i = 0; i < 8; ++i)
                 w[i] = bf16x2(__uint_as_float(ov[2 * i]) * f, __uint_as_float(ov[2 * i + 1]) * f);
-#pragma unroll
-              for (int i = 0; i < 4; ++i) dst[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+              dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+              dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
             }
           }
+          // the accumulators may be overwritten by the next item's first products
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(s32(&sm.acc_free));
+          ++items;
         }
-        item_done = 0;
+        item_steps = 0;
       }
       tc_fence_before();
       __syncwarp();
@@ -449,7 +478,7 @@ __global__ void __launch_bounds__(kThreads, 1)
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 9) {
+  if (warp == kWMma0) {
     tc_fence_after();
     __syncwarp();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");

@@ -10,12 +10,14 @@
 // Key/value-stationary: a persistent CTA per SM draws items of 128 KEY rows (one tile = two 64-row halves,
 // each half one 64-token chunk of a key block; tile t of the 256-row items the other kernels use).  The K
 // and V tiles stay in shared memory; query-side chunks (Q, dO, and per query row -LSE*log2(e) and -D)
-// stream through a ring.  Per product:  S^T = K Q^T and dP^T = V dO^T (eight MMAs into two 64-column TMEM
-// buffers); the row threads (TMEM lane = key row, four threads per row, each a quarter of the query columns; the
-// backward has no reduction along a row, so they never talk) pull their share into registers and hand the
-// buffers back at once, so the next product's S^T and dP^T are computed while they form P^T and dS^T (bf16,
-// own TMEM columns); then dV += P^T dO and dK += dS^T Q (TMEM A operands, the staged dO and Q chunks as
-// MN-major B operands), issued one product behind.
+// stream through a ring of slots, two chunks (a pair of products) per slot.  Per pair:  S^T = K Q^T and
+// dP^T = V dO^T for both chunks at once (eight MMAs with N = 128: the two chunks' Q tiles lie back to back in
+// the slot, their S^T buffers side by side in TMEM); two groups of row threads (TMEM lane = key row, two threads
+// per row and group, each half of the query columns; the backward has no reduction along a row, so they never
+// talk), one group per chunk, pull their share into registers and hand the buffers back at once, so the next
+// pair's S^T and dP^T are computed while they form P^T and dS^T (bf16, own TMEM columns per group); then
+// dV += P^T dO and dK += dS^T Q (TMEM A operands, the staged dO and Q chunks as MN-major B operands), issued by
+// a second thread as each group finishes.  A list with an odd number of chunks ends in a pair of one.
 // Lists: the planner merges the local neighbourhoods of the tile's key blocks (entries carry a mask of the
 // halves they are connected to) and appends each block's CSR list; a list longer than a list buffer
 // continues in the next buffer (ItemInfo::more).  The order of a list is a function of the pattern alone,
@@ -27,30 +29,30 @@ namespace mosaic {
 
 namespace {
 
-constexpr int kStages = 6;       // ring depth of query-side chunks
+constexpr int kSlots = 4;        // ring depth in pairs of query-side chunks
 constexpr int kRowWarps = 16;    // two groups of eight: two threads per key row in each
+constexpr int kGroupWarps = kRowWarps / 2;
 constexpr int kThreads = 32 * (kRowWarps + 4);  // row threads, then TMA producer, two MMA issuers, planner
 constexpr int kWProd = kRowWarps, kWMma0 = kRowWarps + 1, kWMma1 = kRowWarps + 2, kWPlan = kRowWarps + 3;
-constexpr int kGroupWarps = kRowWarps / 2;  // row-thread warps of one group (products alternate between two groups)
 constexpr uint32_t kTmemCols = 512;
-// dK, dV accumulators; two buffers each of S^T and dP^T (fp32, 64 columns) and of P^T and dS^T (bf16 pairs, 32 columns)
+// dK, dV accumulators; per chunk of a pair S^T and dP^T (fp32, 64 columns) and P^T and dS^T (bf16 pairs, 32 columns)
 constexpr uint32_t kColDK = 0, kColDV = 64, kColS = 128, kColDP = 256, kColP = 384, kColDS = 448;
-constexpr uint32_t kStageBytes = 2 * kTile + 2 * 64 * 4;
+constexpr uint32_t kChunkBytes = 2 * kTile + 2 * 64 * 4;
 
-struct Stage {
-  unsigned char q[kTile];     // 64 query rows x 128 B, swizzled
-  unsigned char d_o[kTile];
-  float neg_lse2[64];         // -LSE * log2(e) of the chunk's query rows
-  float neg_d[64];            // -D of the chunk's query rows
-  unsigned char pad[1024 - 512];
+struct Slot {
+  unsigned char q[2][kTile];     // per chunk 64 query rows x 128 B, swizzled; the two tiles form one 128-row operand
+  unsigned char d_o[2][kTile];
+  float neg_lse2[2][64];         // -LSE * log2(e) of the chunks' query rows
+  float neg_d[2][64];            // -D of the chunks' query rows
 };
+static_assert(sizeof(Slot) % 1024 == 0, "slots keep the 1024-byte alignment of the swizzled tiles");
 
 struct Smem {
   unsigned char k[2 * kTile];              // 128 key rows x 128 B
   unsigned char v[2 * kTile];
-  Stage ring[kStages];
-  unsigned long long ring_full[kStages], ring_empty[kStages];
-  unsigned long long kv_full, kv_empty, s_full[2], sdp_free[2], p_full[2], pv_done[2], acc_done, acc_free;
+  Slot ring[kSlots];
+  unsigned long long ring_full[kSlots], ring_empty[kSlots];
+  unsigned long long kv_full, kv_empty, s_full, sdp_free, p_full[2], pv_done, acc_done, acc_free;
   unsigned long long list_full[kLists], list_empty[kLists];
   uint32_t tmem_base;
   int abort;
@@ -160,15 +162,14 @@ __global__ void __launch_bounds__(kThreads, 1)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(s32(&sm.ring_full[s]), 1); mbar_init(s32(&sm.ring_empty[s]), 1); }
+    for (int s = 0; s < kSlots; ++s) { mbar_init(s32(&sm.ring_full[s]), 1); mbar_init(s32(&sm.ring_empty[s]), 1); }
     mbar_init(s32(&sm.kv_full), 1);
     mbar_init(s32(&sm.kv_empty), 1);
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(s32(&sm.s_full[b]), 1);
-      mbar_init(s32(&sm.sdp_free[b]), 32 * kGroupWarps);
-      mbar_init(s32(&sm.p_full[b]), 32 * kGroupWarps);
-      mbar_init(s32(&sm.pv_done[b]), 1);
-    }
+    mbar_init(s32(&sm.s_full), 1);
+    mbar_init(s32(&sm.sdp_free), 32 * kRowWarps);
+    mbar_init(s32(&sm.p_full[0]), 32 * kGroupWarps);
+    mbar_init(s32(&sm.p_full[1]), 32 * kGroupWarps);
+    mbar_init(s32(&sm.pv_done), 1);
     mbar_init(s32(&sm.acc_done), 1);
     mbar_init(s32(&sm.acc_free), kRowWarps);
     for (int i = 0; i < kLists; ++i) {
@@ -193,12 +194,14 @@ __global__ void __launch_bounds__(kThreads, 1)
   const uint32_t tmem = sm.tmem_base;
   volatile int* abort = &sm.abort;
 
+  // Every role walks the same sequence: list buffers, and inside a buffer its n * cpb chunks two at a time.
+  // `pr` counts pairs (ring slot pr % kSlots, phase of the per-pair barriers).
   if (warp == kWPlan) {
     planner_kv_loop(sm, g, csr_off, csr_q, work_counter, ipu, total_items, lane, abort, status);
   } else if (warp == kWProd) {
     // ------------------------------------------------------------- TMA producer
     if (lane == 0) {
-      long long step = 0;  // query-side chunks issued so far (ring position)
+      long long pr = 0;
       int items = 0;       // items started so far (phase of kv_full / kv_empty)
       bool ok = true, fresh = true;  // fresh: the next list buffer starts a new item
       for (int lb = 0; ok; ++lb) {
@@ -223,20 +226,22 @@ __global__ void __launch_bounds__(kThreads, 1)
           ++items;
         }
         fresh = inf.more == 0;
-        for (int e = 0; e < n && ok; ++e) {
-          const int i = sm.ids[buf][e], by = i / g.nbw, bx = i - by * g.nbw;
-          for (int c = 0; c < g.cpb; ++c, ++step) {
-            const int st = (int)(step % kStages);
-            ok = mbar_wait(s32(&sm.ring_empty[st]), (uint32_t)((step / kStages) & 1) ^ 1, abort, status);
-            if (!ok) break;
-            Stage& sg = sm.ring[st];
-            const uint32_t bar = s32(&sm.ring_full[st]);
+        const int chunks = n * g.cpb;
+        for (int p0 = 0; p0 < chunks && ok; p0 += 2, ++pr) {
+          const int slot = (int)(pr % kSlots), np = min(2, chunks - p0);
+          ok = mbar_wait(s32(&sm.ring_empty[slot]), (uint32_t)((pr / kSlots) & 1) ^ 1, abort, status);
+          if (!ok) break;
+          Slot& sl = sm.ring[slot];
+          const uint32_t bar = s32(&sm.ring_full[slot]);
+          mbar_expect_tx(bar, np * kChunkBytes);
+          for (int h = 0; h < np; ++h) {
+            const int e = (p0 + h) / g.cpb, c = (p0 + h) - e * g.cpb;
+            const int i = sm.ids[buf][e], by = i / g.nbw, bx = i - by * g.nbw;
             const int x0 = bx * g.bw, y0 = by * g.bh + c * g.crows;
-            mbar_expect_tx(bar, kStageBytes);
-            tma_load_4d(s32(sg.q), &map_q, bar, 0, x0, y0, u);
-            tma_load_4d(s32(sg.d_o), &map_do, bar, 0, x0, y0, u);
-            tma_load_3d(s32(sg.neg_lse2), &map_nlse, bar, x0, y0, u);
-            tma_load_3d(s32(sg.neg_d), &map_nd, bar, x0, y0, u);
+            tma_load_4d(s32(sl.q[h]), &map_q, bar, 0, x0, y0, u);
+            tma_load_4d(s32(sl.d_o[h]), &map_do, bar, 0, x0, y0, u);
+            tma_load_3d(s32(sl.neg_lse2[h]), &map_nlse, bar, x0, y0, u);
+            tma_load_3d(s32(sl.neg_d[h]), &map_nd, bar, x0, y0, u);
           }
         }
         if (ok) mbar_arrive(s32(&sm.list_empty[buf]));
@@ -244,21 +249,20 @@ __global__ void __launch_bounds__(kThreads, 1)
       if (*abort) {  // give copies in flight time to land before the CTA's memory is released
         const long long t0 = clock64();
         while (clock64() - t0 < 400000) {}
-      } else {       // drain: the last uses of every ring stage have been released
-        const long long first = step > kStages ? step - kStages : 0;
-        for (long long s = first; s < step; ++s)
-          if (!mbar_wait(s32(&sm.ring_empty[s % kStages]), (uint32_t)((s / kStages) & 1), abort, status)) break;
+      } else {       // drain: the last uses of every ring slot have been released
+        const long long first = pr > kSlots ? pr - kSlots : 0;
+        for (long long s = first; s < pr; ++s)
+          if (!mbar_wait(s32(&sm.ring_empty[s % kSlots]), (uint32_t)((s / kSlots) & 1), abort, status)) break;
       }
     }
   } else if (warp == kWMma0) {
     // ------------------------------------------------------------- issuer of S^T = K Q^T and dP^T = V dO^T (one thread)
-    // Product n goes to buffer n & 1.  A buffer may be overwritten once its row threads hold the product before
-    // last in registers, so this thread runs up to two products ahead of the row threads.
+    // The buffers may be overwritten once the row threads hold the previous pair in registers, so this thread runs
+    // one pair ahead of their arithmetic.
     if (lane == 0) {
-      constexpr uint32_t idesc_nt = make_idesc(false);
+      constexpr uint32_t idesc1 = make_idesc(false, 64u), idesc2 = make_idesc(false, 128u);
       const uint64_t kdesc = smem_desc(s32(sm.k)), vdesc = smem_desc(s32(sm.v));
-      long long step = 0;   // ring position
-      uint32_t nt = 0;      // products started so far (buffer and phase of the per-product barriers)
+      long long pr = 0;
       int items = 0;
       bool ok = true, fresh = true;
       for (int lb = 0; ok; ++lb) {
@@ -274,24 +278,20 @@ __global__ void __launch_bounds__(kThreads, 1)
           ++items;
         }
         fresh = !more;
-        for (int e = 0; e < n && ok; ++e) {
-          for (int c = 0; c < g.cpb && ok; ++c, ++step) {
-            const int st = (int)(step % kStages);
-            const uint32_t b = nt & 1, j = nt >> 1;
-            ok = mbar_wait(s32(&sm.ring_full[st]), (uint32_t)((step / kStages) & 1), abort, status);
-            if (ok && j > 0) ok = mbar_wait(s32(&sm.sdp_free[b]), (j - 1) & 1, abort, status);
-            if (!ok) break;
-            tc_fence_after();
-            const uint64_t qdesc = smem_desc(s32(sm.ring[st].q)), dodesc = smem_desc(s32(sm.ring[st].d_o));
+        const int chunks = n * g.cpb;
+        for (int p0 = 0; p0 < chunks && ok; p0 += 2, ++pr) {
+          const int slot = (int)(pr % kSlots);
+          ok = mbar_wait(s32(&sm.ring_full[slot]), (uint32_t)((pr / kSlots) & 1), abort, status);
+          if (ok && pr > 0) ok = mbar_wait(s32(&sm.sdp_free), (uint32_t)((pr - 1) & 1), abort, status);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t idesc = chunks - p0 >= 2 ? idesc2 : idesc1;
+          const uint64_t qdesc = smem_desc(s32(sm.ring[slot].q[0])), dodesc = smem_desc(s32(sm.ring[slot].d_o[0]));
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-              umma_ss(tmem + kColS + 64 * b, kdesc + 2 * kk, qdesc + 2 * kk, idesc_nt, kk > 0);
+          for (int kk = 0; kk < 4; ++kk) umma_ss(tmem + kColS, kdesc + 2 * kk, qdesc + 2 * kk, idesc, kk > 0);
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-              umma_ss(tmem + kColDP + 64 * b, vdesc + 2 * kk, dodesc + 2 * kk, idesc_nt, kk > 0);
-            tc_commit(s32(&sm.s_full[b]));
-            ++nt;
-          }
+          for (int kk = 0; kk < 4; ++kk) umma_ss(tmem + kColDP, vdesc + 2 * kk, dodesc + 2 * kk, idesc, kk > 0);
+          tc_commit(s32(&sm.s_full));
         }
         // the K and V tiles are read by this thread's products only: all of the item's are behind this commit
         if (ok && !more) tc_commit(s32(&sm.kv_empty));
@@ -302,9 +302,9 @@ __global__ void __launch_bounds__(kThreads, 1)
     // ------------------------------------------------------------- issuer of dV += P^T dO and dK += dS^T Q (one thread)
     if (lane == 0) {
       constexpr uint32_t idesc_nn = make_idesc(true);
-      long long step = 0;
-      uint32_t nt = 0;
-      uint32_t items = 0;   // items whose accumulators have been handed to the row threads
+      long long pr = 0;
+      uint32_t jg[2] = {0u, 0u};  // products each group of row threads has handed over (phase of p_full)
+      uint32_t items = 0;         // items whose accumulators have been handed to the row threads
       bool ok = true, first = true;
       for (int lb = 0; ok; ++lb) {
         const int buf = lb % kLists;
@@ -313,32 +313,33 @@ __global__ void __launch_bounds__(kThreads, 1)
         const int n = sm.info[buf].n;
         if (n < 0) break;
         const bool more = sm.info[buf].more != 0;
-        for (int e = 0; e < n && ok; ++e) {
-          for (int c = 0; c < g.cpb && ok; ++c, ++step) {
-            const int st = (int)(step % kStages);
-            const uint32_t b = nt & 1, j = nt >> 1;
-            // the stage landed before S^T could be produced; this wait makes the copied Q and dO visible here too
-            ok = mbar_wait(s32(&sm.ring_full[st]), (uint32_t)((step / kStages) & 1), abort, status);
-            if (ok) ok = mbar_wait(s32(&sm.p_full[b]), j & 1, abort, status);
+        const int chunks = n * g.cpb;
+        for (int p0 = 0; p0 < chunks && ok; p0 += 2, ++pr) {
+          const int slot = (int)(pr % kSlots), np = min(2, chunks - p0);
+          // the slot landed before S^T could be produced; this wait makes the copied Q and dO visible here too
+          ok = mbar_wait(s32(&sm.ring_full[slot]), (uint32_t)((pr / kSlots) & 1), abort, status);
+          for (int h = 0; h < np && ok; ++h) {
+            ok = mbar_wait(s32(&sm.p_full[h]), jg[h] & 1, abort, status);
             // a new accumulation overwrites dK and dV: every row thread must have read the previous item's
             if (ok && first && items > 0) ok = mbar_wait(s32(&sm.acc_free), (items - 1) & 1, abort, status);
             if (!ok) break;
+            ++jg[h];
             tc_fence_after();
-            const uint64_t qmn = smem_desc(s32(sm.ring[st].q)), domn = smem_desc(s32(sm.ring[st].d_o));
+            const uint64_t qmn = smem_desc(s32(sm.ring[slot].q[h])), domn = smem_desc(s32(sm.ring[slot].d_o[h]));
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)
-              umma_ts(tmem + kColDV, tmem + kColP + 32 * b + 8 * kk, domn + (uint64_t)((2048 * kk) >> 4), idesc_nn,
+              umma_ts(tmem + kColDV, tmem + kColP + 32 * h + 8 * kk, domn + (uint64_t)((2048 * kk) >> 4), idesc_nn,
                       (!first || kk > 0));
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)
-              umma_ts(tmem + kColDK, tmem + kColDS + 32 * b + 8 * kk, qmn + (uint64_t)((2048 * kk) >> 4), idesc_nn,
+              umma_ts(tmem + kColDK, tmem + kColDS + 32 * h + 8 * kk, qmn + (uint64_t)((2048 * kk) >> 4), idesc_nn,
                       (!first || kk > 0));
-            // the stage's S^T and dP^T completed before P^T could be formed, so this thread's completion frees it
-            tc_commit(s32(&sm.ring_empty[st]));
-            tc_commit(s32(&sm.pv_done[b]));
             first = false;
-            ++nt;
           }
+          if (!ok) break;
+          // the pair's S^T and dP^T completed before P^T could be formed, so this thread's completion frees the slot
+          tc_commit(s32(&sm.ring_empty[slot]));
+          tc_commit(s32(&sm.pv_done));
         }
         if (ok && !more && !first) {  // the item's accumulators are complete behind this commit
           tc_commit(s32(&sm.acc_done));
@@ -350,10 +351,9 @@ __global__ void __launch_bounds__(kThreads, 1)
     }
   } else if (warp < kRowWarps) {
     // ------------------------------------------------------------- row threads (TMEM lane = key row)
-    // Two groups of eight warps take the products in turn (product n: group and buffer n & 1), so one group's
-    // waits and TMEM traffic fall into the other's arithmetic.  Inside a group two threads share a key row, each
-    // with half of the query columns.
-    const int grp = warp >> 3;        // products this thread works on: those with n & 1 == grp
+    // Group 0 takes the first chunk of every pair, group 1 the second, so the two work side by side.  Inside a
+    // group two threads share a key row, each with half of the query columns.
+    const int grp = warp >> 3;        // chunk of a pair this thread works on
     const int ch = (warp >> 2) & 1;   // half of the query columns
     const int cq = warp >> 2;         // quarter of the output channels (epilogue)
     const int quad = warp & 3;        // TMEM lane quadrant
@@ -364,9 +364,8 @@ __global__ void __launch_bounds__(kThreads, 1)
     const uint64_t scale2 = pack2(g.scale_log2, g.scale_log2);
     const uint32_t col_s = kColS + 64 * grp + 32 * ch, col_dp = kColDP + 64 * grp + 32 * ch;
     const uint32_t col_p = kColP + 32 * grp + 16 * ch, col_ds = kColDS + 32 * grp + 16 * ch;
-    uint32_t nt = 0;     // products seen so far (both groups)
-    long long step = 0;  // ring position, to find the stage that holds the query rows' -LSE and -D
-    uint32_t item_steps = 0, items = 0;
+    long long pr = 0;    // pairs seen so far
+    uint32_t item_chunks = 0, items = 0;
     bool ok = true;
     for (int lb = 0; ok; ++lb) {
       const int buf = lb % kLists;
@@ -376,71 +375,75 @@ __global__ void __launch_bounds__(kThreads, 1)
       const int n = sm.info[buf].n;
       if (n < 0) break;
       const bool more = sm.info[buf].more != 0;
-      for (int e = 0; e < n && ok; ++e) {
-        const bool connected = (sm.mask[buf][e] & hbit) != 0;
-        for (int c = 0; c < g.cpb; ++c, ++step, ++nt, ++item_steps) {
-          if ((int)(nt & 1) != grp) continue;
-          const uint32_t j = nt >> 1;
-          ok = mbar_wait(s32(&sm.s_full[grp]), j & 1, abort, status);
+      const int chunks = n * g.cpb;
+      item_chunks += (uint32_t)chunks;
+      for (int p0 = 0; p0 < chunks; p0 += 2, ++pr) {
+        ok = mbar_wait(s32(&sm.s_full), (uint32_t)(pr & 1), abort, status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        const int p = p0 + grp;
+        if (p >= chunks) {  // a pair of one: nothing for group 1, the buffers go back at once
+          tc_fence_before();
+          mbar_arrive(s32(&sm.sdp_free));
+          continue;
+        }
+        const bool connected = (sm.mask[buf][p / g.cpb] & hbit) != 0;
+        uint32_t pp[16], ds[16];
+        if (connected) {
+          const int slot = (int)(pr % kSlots);
+          // the slot landed before the MMA warp could produce this S^T; waiting on its barrier here as well
+          // makes the copied -LSE and -D visible to this thread
+          ok = mbar_wait(s32(&sm.ring_full[slot]), (uint32_t)((pr / kSlots) & 1), abort, status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          const Slot& sl = sm.ring[slot];
+          uint32_t sv[32], dp[32];
+          tmem_ld32(tb + col_s, sv);
+          tmem_ld32(tb + col_dp, dp);
+          tmem_wait_ld();
+          tc_fence_before();
+          mbar_arrive(s32(&sm.sdp_free));  // S^T and dP^T go back to the tensor core
+#pragma unroll
+          for (int i = 0; i < 32; i += 4) {
+            // -LSE*log2(e) and -D of four query columns (the same for every thread: broadcast loads)
+            const float4 nl = *reinterpret_cast<const float4*>(&sl.neg_lse2[grp][32 * ch + i]);
+            const float4 nd = *reinterpret_cast<const float4*>(&sl.neg_d[grp][32 * ch + i]);
+            float x0, x1, x2, x3, d0, d1, d2, d3;
+            unpack2(fma2(pack2(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])), scale2, pack2(nl.x, nl.y)), x0, x1);
+            unpack2(fma2(pack2(__uint_as_float(sv[i + 2]), __uint_as_float(sv[i + 3])), scale2, pack2(nl.z, nl.w)), x2, x3);
+            const float e0 = ex2(x0), e1 = ex2(x1), e2 = ex2(x2), e3 = ex2(x3);
+            const uint64_t t01 = add2(pack2(__uint_as_float(dp[i]), __uint_as_float(dp[i + 1])), pack2(nd.x, nd.y));
+            const uint64_t t23 = add2(pack2(__uint_as_float(dp[i + 2]), __uint_as_float(dp[i + 3])), pack2(nd.z, nd.w));
+            unpack2(mul2(pack2(e0, e1), t01), d0, d1);
+            unpack2(mul2(pack2(e2, e3), t23), d2, d3);
+            pp[i >> 1] = bf16x2(e0, e1);
+            pp[(i >> 1) + 1] = bf16x2(e2, e3);
+            ds[i >> 1] = bf16x2(d0, d1);
+            ds[(i >> 1) + 1] = bf16x2(d2, d3);
+          }
+        } else {
+          tc_fence_before();
+          mbar_arrive(s32(&sm.sdp_free));
+#pragma unroll
+          for (int i = 0; i < 16; ++i) { pp[i] = 0u; ds[i] = 0u; }
+        }
+        // P^T and dS^T have one buffer per group: the previous pair's dV / dK updates must have consumed them
+        if (pr > 0) {
+          ok = mbar_wait(s32(&sm.pv_done), (uint32_t)((pr - 1) & 1), abort, status);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
-          uint32_t pp[16], ds[16];
-          if (connected) {
-            const int st = (int)(step % kStages);
-            // the stage landed before the MMA warp could produce this S^T; waiting on its barrier here as well
-            // makes the copied -LSE and -D visible to this thread
-            ok = mbar_wait(s32(&sm.ring_full[st]), (uint32_t)((step / kStages) & 1), abort, status);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            const Stage& sg = sm.ring[st];
-            uint32_t sv[32], dp[32];
-            tmem_ld32(tb + col_s, sv);
-            tmem_ld32(tb + col_dp, dp);
-            tmem_wait_ld();
-            tc_fence_before();
-            mbar_arrive(s32(&sm.sdp_free[grp]));  // S^T and dP^T go back to the tensor core
-#pragma unroll
-            for (int i = 0; i < 32; i += 4) {
-              // -LSE*log2(e) and -D of four query columns (the same for every thread: broadcast loads)
-              const float4 nl = *reinterpret_cast<const float4*>(&sg.neg_lse2[32 * ch + i]);
-              const float4 nd = *reinterpret_cast<const float4*>(&sg.neg_d[32 * ch + i]);
-              float x0, x1, x2, x3, d0, d1, d2, d3;
-              unpack2(fma2(pack2(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])), scale2, pack2(nl.x, nl.y)), x0, x1);
-              unpack2(fma2(pack2(__uint_as_float(sv[i + 2]), __uint_as_float(sv[i + 3])), scale2, pack2(nl.z, nl.w)), x2, x3);
-              const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
-              const uint64_t t01 = add2(pack2(__uint_as_float(dp[i]), __uint_as_float(dp[i + 1])), pack2(nd.x, nd.y));
-              const uint64_t t23 = add2(pack2(__uint_as_float(dp[i + 2]), __uint_as_float(dp[i + 3])), pack2(nd.z, nd.w));
-              unpack2(mul2(pack2(p0, p1), t01), d0, d1);
-              unpack2(mul2(pack2(p2, p3), t23), d2, d3);
-              pp[i >> 1] = bf16x2(p0, p1);
-              pp[(i >> 1) + 1] = bf16x2(p2, p3);
-              ds[i >> 1] = bf16x2(d0, d1);
-              ds[(i >> 1) + 1] = bf16x2(d2, d3);
-            }
-          } else {
-            tc_fence_before();
-            mbar_arrive(s32(&sm.sdp_free[grp]));
-#pragma unroll
-            for (int i = 0; i < 16; ++i) { pp[i] = 0u; ds[i] = 0u; }
-          }
-          // this group's P^T and dS^T buffer: its previous dV / dK updates must have consumed it
-          if (j > 0) {
-            ok = mbar_wait(s32(&sm.pv_done[grp]), (j - 1) & 1, abort, status);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after();
-          }
-          tmem_st16(tb + col_p, pp);
-          tmem_st16(tb + col_ds, ds);
-          tmem_wait_st();
-          tc_fence_before();
-          mbar_arrive(s32(&sm.p_full[grp]));
         }
+        tmem_st16(tb + col_p, pp);
+        tmem_st16(tb + col_ds, ds);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(s32(&sm.p_full[grp]));
       }
       if (!ok) break;
       if (!more) {
-        if (item_steps > 0) {
+        if (item_chunks > 0) {
           ok = mbar_wait(s32(&sm.acc_done), items & 1, abort, status);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
@@ -469,7 +472,7 @@ __global__ void __launch_bounds__(kThreads, 1)
           if (lane == 0) mbar_arrive(s32(&sm.acc_free));
           ++items;
         }
-        item_steps = 0;
+        item_chunks = 0;
       }
       tc_fence_before();
       __syncwarp();

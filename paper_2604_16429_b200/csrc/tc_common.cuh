@@ -254,9 +254,9 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
   d |= (uint64_t)2 << 61;               // SWIZZLE_128B
   return d;
 }
-// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 64.
-__host__ __device__ constexpr uint32_t make_idesc(bool b_mn_major) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((64u >> 3) << 17) |
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 64 unless given.
+__host__ __device__ constexpr uint32_t make_idesc(bool b_mn_major, uint32_t n = 64u) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((n >> 3) << 17) |
          ((128u >> 4) << 24);
 }
 

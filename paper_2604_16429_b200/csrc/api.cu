@@ -75,7 +75,7 @@ BranchWs branch_layout(const Geo& g) {
 
 namespace {
 
-struct BwdWs { size_t D, negD, nlse2, off, q, total; };
+struct BwdWs { size_t D, negD, nlse2, off, q, order, total; };
 BwdWs bwd_layout(const Geo& g) {
   BwdWs w;
   size_t at = kStatusBytes;
@@ -84,6 +84,8 @@ BwdWs bwd_layout(const Geo& g) {
   w.nlse2 = at; at = align256(at + sizeof(float) * (size_t)g.U * g.N);
   w.off = at; at = align256(at + sizeof(int32_t) * (size_t)g.U * (g.m + 1));
   w.q = at; at = align256(at + sizeof(int32_t) * (size_t)g.U * g.m * (g.topk > 0 ? g.topk : 1));
+  // dK/dV items (two 128-row tiles per 256-row item of a key/value unit), longest first, and their cost classes
+  w.order = at; at = align256(at + 2 * sizeof(int32_t) * 2 * (size_t)g.Ukv * items_per_unit(g));
   w.total = at;
   return w;
 }
@@ -216,7 +218,7 @@ int mosaic_bsa_bwd(const mosaic_bsa_params* p, const void* q, const void* k, con
   char* base = (char*)ws;
   return launch_bwd(c, q, k, v, o, lse, d_o, block_idx, dq, dk, dv, (float*)(base + w.D),
                     (float*)(base + w.negD), (float*)(base + w.nlse2), (int32_t*)(base + w.off),
-                    (int32_t*)(base + w.q));
+                    (int32_t*)(base + w.q), (int32_t*)(base + w.order));
 }
 
 int mosaic_bsa_last_status(const void* ws, void* cuda_stream) {

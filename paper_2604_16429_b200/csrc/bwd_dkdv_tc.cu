@@ -64,12 +64,16 @@ struct Smem {
 // Planner of the key-stationary kernel: per item (tile), the merged local neighbourhoods of its key blocks,
 // then each block's list of selecting query blocks, cut into list buffers.
 __device__ __forceinline__ void planner_kv_loop(Smem& sm, const Geo& g, const int32_t* __restrict__ csr_off,
-                                                const int32_t* __restrict__ csr_q, int* work_counter, int ipu,
+                                                const int32_t* __restrict__ csr_q,
+                                                const int32_t* __restrict__ order, int* work_counter, int ipu,
                                                 int total_items, int lane, volatile int* abort, int* status) {
   int lb = 0;  // list buffers handed out so far
   for (int it = 0;; ++it) {
     int item = 0;
-    if (lane == 0) item = it == 0 ? (int)blockIdx.x : atomicAdd(work_counter, 1) + (int)gridDim.x;
+    if (lane == 0) {  // the queue hands out positions of the longest-first order
+      const int pos = it == 0 ? (int)blockIdx.x : atomicAdd(work_counter, 1) + (int)gridDim.x;
+      item = pos < total_items ? __ldg(order + pos) : total_items;
+    }
     item = __shfl_sync(0xffffffffu, item, 0);
     bool ok = true;
     auto acquire = [&]() {  // wait until list buffer lb % kLists is free
@@ -150,12 +154,67 @@ __device__ __forceinline__ void planner_kv_loop(Smem& sm, const Geo& g, const in
 
 }  // namespace
 
+// The items' lists differ in length (a key block that many query blocks selected has a long one), and a long item
+// drawn late leaves the other SMs idle at the end.  This kernel orders the items by the number of selecting query
+// blocks, longest first, inside windows of consecutive key/value units (the windows keep their order, so that items
+// in flight at the same time read the same few units; a window holds at least sixteen items per SM).  One CTA per
+// window, counting sort; the place inside a class of equal length is arbitrary, which changes no result: an item
+// writes only its own tile, in the order of its own list.
+constexpr int kCostBins = 2048;
+__global__ void __launch_bounds__(1024) dkdv_order_kernel(const Geo g, const int32_t* __restrict__ csr_off, int ipu,
+                                                          int total_items, int window_items,
+                                                          int32_t* __restrict__ order, int32_t* __restrict__ bins) {
+  __shared__ int hist[kCostBins];
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int first_item = (int)blockIdx.x * window_items;
+  const int end_item = min(total_items, first_item + window_items);
+  for (int i = tid; i < kCostBins; i += (int)blockDim.x) hist[i] = 0;
+  __syncthreads();
+  const int ratio = g.H / g.Hkv;
+  for (int item = first_item + tid; item < end_item; item += (int)blockDim.x) {
+    const int i256 = item >> 1, t = item & 1, u = i256 / ipu;
+    int hb4[4], hc4[4];
+    const int valid = (item_halves(g, i256 - u * ipu, hb4, hc4) >> (2 * t)) & 3;
+    const int b0 = hb4[2 * t], b1 = hb4[2 * t + 1];
+    const bool use0 = (valid & 1) != 0, use1 = (valid & 2) != 0 && !(valid == 3 && b0 == b1);
+    const int qu0 = (u / g.Hkv) * g.H + (u - (u / g.Hkv) * g.Hkv) * ratio;
+    int cost = 0;
+    for (int r = 0; r < ratio; ++r) {
+      const int32_t* off = csr_off + (long long)(qu0 + r) * (g.m + 1);
+      if (use0) cost += __ldg(off + b0 + 1) - __ldg(off + b0);
+      if (use1) cost += __ldg(off + b1 + 1) - __ldg(off + b1);
+    }
+    const int bin = cost < 0 ? 0 : (cost < kCostBins ? cost : kCostBins - 1);
+    bins[item] = bin;
+    atomicAdd(&hist[bin], 1);
+  }
+  __syncthreads();
+  if (tid < 32) {  // first place of each class, classes in descending order
+    int carry = 0;
+    for (int base = kCostBins - 32; base >= 0; base -= 32) {
+      const int b = base + 31 - lane;  // lane 0 takes the highest class of the chunk
+      const int v = hist[b];
+      int incl = v;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int nb = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += nb;
+      }
+      hist[b] = carry + incl - v;
+      carry += __shfl_sync(0xffffffffu, incl, 31);
+    }
+  }
+  __syncthreads();
+  for (int item = first_item + tid; item < end_item; item += (int)blockDim.x)
+    order[first_item + atomicAdd(&hist[bins[item]], 1)] = item;
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
     dkdv_tc_kernel(const Geo g, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_do,
                    const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                    const __grid_constant__ CUtensorMap map_nlse, const __grid_constant__ CUtensorMap map_nd,
                    const int32_t* __restrict__ csr_off, const int32_t* __restrict__ csr_q,
-                   __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv, int* status, int* work_counter,
+                   const int32_t* __restrict__ order, __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv, int* status, int* work_counter,
                    int ipu, int total_items) {
   extern __shared__ unsigned char smem_raw[];
   Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -197,7 +256,7 @@ __global__ void __launch_bounds__(kThreads, 1)
   // Every role walks the same sequence: list buffers, and inside a buffer its n * cpb chunks two at a time.
   // `pr` counts pairs (ring slot pr % kSlots, phase of the per-pair barriers).
   if (warp == kWPlan) {
-    planner_kv_loop(sm, g, csr_off, csr_q, work_counter, ipu, total_items, lane, abort, status);
+    planner_kv_loop(sm, g, csr_off, csr_q, order, work_counter, ipu, total_items, lane, abort, status);
   } else if (warp == kWProd) {
     // ------------------------------------------------------------- TMA producer
     if (lane == 0) {
@@ -491,7 +550,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 // `work_counter` must be zero when the kernel starts (a word of the workspace status block).
 int launch_dkdv_tc(const HostCtx& c, const void* q, const void* k, const void* v, const void* d_o,
                    const float* neg_lse2, const float* neg_d, const int32_t* csr_off, const int32_t* csr_q, void* dk,
-                   void* dv, int* work_counter) {
+                   void* dv, int* work_counter, int32_t* order) {
   const Geo& g = c.g;
   CUtensorMap mq, mdo, mk, mv, mnl, mnd;
   if (!make_map(&mq, q, g, g.U) || !make_map(&mdo, d_o, g, g.U) || !make_map(&mk, k, g, g.Ukv) || !make_map(&mv, v, g, g.Ukv) ||
@@ -505,7 +564,17 @@ int launch_dkdv_tc(const HostCtx& c, const void* q, const void* k, const void* v
   const long long total = 2ll * g.Ukv * ipu;  // one item per 128-row tile of a key/value unit
   if (total > 0x7fffff00ll) return MOSAIC_E_UNSUPPORTED;
   const long long grid = total < (long long)sms ? total : (long long)sms;
-  dkdv_tc_kernel<<<(unsigned)grid, kThreads, smem, c.stream>>>(g, mq, mdo, mk, mv, mnl, mnd, csr_off, csr_q,
+  // window: the key/value units whose Q and dO (all query heads of the group) take about 48 MB, widened to
+  // sixteen items per SM
+  const size_t unit_bytes = (size_t)(g.H / g.Hkv) * g.N * kD * 2 * 2;
+  long long win_units = unit_bytes >= (48u << 20) ? 1 : (long long)((48u << 20) / unit_bytes);
+  const long long min_units = (16ll * sms + 2 * ipu - 1) / (2 * ipu);
+  if (win_units < min_units) win_units = min_units;
+  const long long win_items = win_units * 2 * ipu;
+  dkdv_order_kernel<<<(unsigned)((total + win_items - 1) / win_items), 1024, 0, c.stream>>>(
+      g, csr_off, ipu, (int)total, (int)win_items, order, order + total);
+  if (cudaGetLastError() != cudaSuccess) return MOSAIC_E_CUDA;
+  dkdv_tc_kernel<<<(unsigned)grid, kThreads, smem, c.stream>>>(g, mq, mdo, mk, mv, mnl, mnd, csr_off, csr_q, order,
                                                                (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, c.status,
                                                                work_counter, ipu, (int)total);
   return cudaGetLastError() == cudaSuccess ? MOSAIC_OK : MOSAIC_E_CUDA;

@@ -83,6 +83,13 @@ __device__ __forceinline__ long long chunk_token(const Geo& g, int j, int c, int
   return chunk_row_token(g, j, c, r) + (e - r * g.bw);
 }
 
+// Work items of 256 rows (four 64-row halves) per unit, as the tensor-core kernels cut a unit's blocks.
+__host__ __device__ inline int items_per_unit(const Geo& g) {
+  if (g.cpb == 1) return (g.nbh >> 1) * ((g.nbw + 1) >> 1) + (g.nbh & 1) * ((g.nbw + 3) >> 2);
+  if (g.cpb == 2) return g.nbw > 1 ? g.nbh * ((g.nbw + 1) >> 1) : (g.nbh + 1) >> 1;
+  return g.m * ((g.cpb + 3) >> 2);
+}
+
 // ---- host side ---------------------------------------------------------------------------
 struct HostCtx {
   Geo g;
@@ -112,9 +119,9 @@ int launch_dq_tc(const HostCtx& c, const void* q, const void* k, const void* v, 
                  const float* D, const int32_t* block_idx, void* dq, int* work_counter);
 int launch_dkdv_tc(const HostCtx& c, const void* q, const void* k, const void* v, const void* d_o,
                    const float* neg_lse2, const float* neg_d, const int32_t* csr_off, const int32_t* csr_q, void* dk,
-                   void* dv, int* work_counter);
+                   void* dv, int* work_counter, int32_t* order);
 int launch_bwd(const HostCtx& c, const void* q, const void* k, const void* v, const void* o, const float* lse,
                const void* d_o, const int32_t* block_idx, void* dq, void* dk, void* dv, float* Dbuf, float* neg_d,
-               float* neg_lse2, int32_t* csr_off, int32_t* csr_q);
+               float* neg_lse2, int32_t* csr_off, int32_t* csr_q, int32_t* order);
 
 }  // namespace mosaic

@@ -318,12 +318,6 @@ __device__ __forceinline__ int item_halves(const Geo& g, int it, int (&hb)[4], i
   return valid;
 }
 
-__host__ __device__ inline int items_per_unit(const Geo& g) {
-  if (g.cpb == 1) return (g.nbh >> 1) * ((g.nbw + 1) >> 1) + (g.nbh & 1) * ((g.nbw + 3) >> 2);
-  if (g.cpb == 2) return g.nbw > 1 ? g.nbh * ((g.nbw + 1) >> 1) : (g.nbh + 1) >> 1;
-  return g.m * ((g.cpb + 3) >> 2);
-}
-
 // Warp-cooperative attended list of query block i (local set, then valid selected ids) written to
 // ids[n0..); returns the new count.  `j` is this lane's entry of the block's row of block_idx (-1 beyond top-k).
 __device__ __forceinline__ int warp_attended(const Geo& g, int j, int i, int* ids, int n0, int lane, int* status) {

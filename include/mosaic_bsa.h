@@ -72,7 +72,8 @@ typedef struct mosaic_bsa_params {
  * blocks of 1024 tokens -- is nlat = N/16, nlon = 16, bh = 8, bw = 16, rlat = 8, rlon = 1 with this flag. */
 #define MOSAIC_FLAG_LOCAL_GROUPS 1u
 
-enum { MOSAIC_OP_SELECT = 0, MOSAIC_OP_FWD = 1, MOSAIC_OP_BWD = 2, MOSAIC_OP_FWD_BRANCHES = 3 };
+enum { MOSAIC_OP_SELECT = 0, MOSAIC_OP_FWD = 1, MOSAIC_OP_BWD = 2, MOSAIC_OP_FWD_BRANCHES = 3,
+       MOSAIC_OP_BWD_BRANCHES = 4 };
 
 enum {
   MOSAIC_OK = 0,
@@ -155,6 +156,28 @@ int mosaic_bsa_fwd_branches(const mosaic_bsa_params *p, const void *q, const voi
 int mosaic_bsa_bwd(const mosaic_bsa_params *p, const void *q, const void *k, const void *v,
                    const void *o, const float *lse, const void *d_o, const int32_t *block_idx,
                    void *dq, void *dk, void *dv, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Backward of the three-branch form (gradient of mosaic_bsa_fwd_branches with the selection held constant).
+ * Each attention branch is a softmax attention of its own, so each takes the attention backward with dO
+ * scaled by its gate; the compression branch is differentiated on the block level (softmax backward on the
+ * mean-pooled vectors; a mean spreads its gradient evenly over the block's tokens), which is the only path by
+ * which gradient reaches the block-level (routing) scores (the paper's ablation appendix: the routing scores
+ * are trained through the compression branch).  The forward's intermediates are recomputed, so nothing of the
+ * forward call has to be kept.
+ *   q                in   [B,H,N,d] bf16;  k, v in [B,Hkv,N,d] bf16
+ *   block_idx        in   [B,H,m,topk] int32, same rules as mosaic_bsa_fwd
+ *   gates            in   [B,H,N,3] fp32, order (compression, selection, local)
+ *   d_o              in   [B,H,N,d] bf16, gradient of the forward's o
+ *   dq               out  [B,H,N,d] bf16;  dk, dv out [B,Hkv,N,d] bf16
+ *   dgates           out  [B,H,N,3] fp32, dgates[l][x] = <d_o_l, branch output x of token l>
+ * Workspace: mosaic_bsa_workspace_bytes(p, MOSAIC_OP_BWD_BRANCHES) (about ten tensors of the size of q).
+ * Results are deterministic.  Errors as for mosaic_bsa_bwd.
+ */
+int mosaic_bsa_bwd_branches(const mosaic_bsa_params *p, const void *q, const void *k, const void *v,
+                            const int32_t *block_idx, const float *gates, const void *d_o, void *dq,
+                            void *dk, void *dv, float *dgates, void *ws, size_t ws_bytes,
+                            void *cuda_stream);
 
 /*
  * Selection for callers that cannot allocate device memory.  (The paper has no counterpart of this

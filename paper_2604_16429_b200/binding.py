@@ -17,10 +17,10 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmosaic_bsa.so")
 _lib = None
 
-OP_SELECT, OP_FWD, OP_BWD, OP_FWD_BRANCHES = 0, 1, 2, 3
+OP_SELECT, OP_FWD, OP_BWD, OP_FWD_BRANCHES, OP_BWD_BRANCHES = 0, 1, 2, 3, 4
 EXPORTS = ("mosaic_bsa_workspace_bytes", "mosaic_bsa_select", "mosaic_bsa_fwd", "mosaic_bsa_bwd",
            "mosaic_bsa_last_status", "mosaic_bsa_strerror", "mosaic_bsa_select_static",
-           "mosaic_bsa_descriptor_encodes", "mosaic_bsa_fwd_branches")
+           "mosaic_bsa_descriptor_encodes", "mosaic_bsa_fwd_branches", "mosaic_bsa_bwd_branches")
 STATIC_SCRATCH_BYTES = 4 << 20
 FLAG_LOCAL_GROUPS = 1
 
@@ -95,6 +95,8 @@ def lib():
         L.mosaic_bsa_fwd.argtypes = [pp, vp, vp, vp, i32p, vp, fp, vp, ctypes.c_size_t, vp]
         L.mosaic_bsa_fwd_branches.restype = ctypes.c_int
         L.mosaic_bsa_fwd_branches.argtypes = [pp, vp, vp, vp, i32p, fp, vp, fp, fp, vp, ctypes.c_size_t, vp]
+        L.mosaic_bsa_bwd_branches.restype = ctypes.c_int
+        L.mosaic_bsa_bwd_branches.argtypes = [pp, vp, vp, vp, i32p, fp, vp, vp, vp, vp, fp, vp, ctypes.c_size_t, vp]
         L.mosaic_bsa_bwd.restype = ctypes.c_int
         L.mosaic_bsa_bwd.argtypes = [pp, vp, vp, vp, vp, fp, vp, i32p, vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.mosaic_bsa_last_status.restype = ctypes.c_int
@@ -219,6 +221,27 @@ def mosaic_bsa_bwd(p: Params, q, k, v, o, lse, d_o, block_idx, dq=None, dk=None,
     if rc:
         raise MosaicError(rc, "mosaic_bsa_bwd")
     return dq, dk, dv
+
+
+def mosaic_bsa_bwd_branches(p: Params, q, k, v, block_idx, gates, d_o, dq=None, dk=None, dv=None, dgates=None, ws=None,
+                            stream=None):
+    """Backward of the three-branch form.  Returns (dq, dk, dv, dgates); dgates is [B, H, N, 3] fp32."""
+    _chk_qkv(p, q, d_o)
+    _chk_qkv(p, k, v, heads=p.kv_heads)
+    if gates.dtype != torch.float32 or not gates.is_contiguous() or tuple(gates.shape) != (p.B, p.H, p.N, 3):
+        raise ValueError(f"expected contiguous cuda fp32 gates [{p.B},{p.H},{p.N},3]")
+    dq = torch.empty_like(q) if dq is None else dq
+    dk = torch.empty_like(k) if dk is None else dk
+    dv = torch.empty_like(k) if dv is None else dv
+    dgates = torch.empty_like(gates) if dgates is None else dgates
+    if ws is None:
+        ws = alloc_workspace(p, OP_BWD_BRANCHES, q.device)
+    pc = p.c()
+    rc = lib().mosaic_bsa_bwd_branches(ctypes.byref(pc), _ptr(q), _ptr(k), _ptr(v), _ptr(block_idx), _ptr(gates), _ptr(d_o),
+                                       _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dgates), _ptr(ws), ws.numel(), _stream(stream))
+    if rc:
+        raise MosaicError(rc, "mosaic_bsa_bwd_branches")
+    return dq, dk, dv, dgates
 
 
 def mosaic_bsa_last_status(ws, stream=None) -> int:

@@ -89,6 +89,34 @@ BwdWs bwd_layout(const Geo& g) {
   w.total = at;
   return w;
 }
+// Scratch of the three-branch backward: the forward's (pooled sums, obar, both branch outputs), the branch
+// log-sum-exps, the block-level backward's vectors, the gated copies of dO, the branch gradients, and the
+// attention backward's own scratch (used by the two passes in turn).
+struct BwdBranchWs {
+  BranchWs f;
+  size_t lse_fg, lse_l, lse_cg, delta, dob, dqm, dkm, dvm, do_fg, do_l, dq_fg, dq_l, dk_fg, dk_l, dv_fg, dv_l, inner, total;
+};
+BwdBranchWs bwd_branch_layout(const Geo& g) {
+  BwdBranchWs w;
+  w.f = branch_layout(g);
+  const size_t pooled = align256(sizeof(float) * (size_t)g.U * g.m * kD), rows = align256(sizeof(float) * (size_t)g.U * g.N);
+  const size_t blocks = align256(sizeof(float) * (size_t)g.U * g.m);
+  const size_t full = align256(2 * (size_t)g.U * g.N * kD);
+  size_t at = w.f.total;
+  w.lse_fg = at; at += rows;
+  w.lse_l = at; at += rows;
+  w.lse_cg = at; at += blocks;
+  w.delta = at; at += blocks;
+  w.dob = at; at += pooled;
+  w.dqm = at; at += pooled;
+  w.dkm = at; at += pooled;
+  w.dvm = at; at += pooled;
+  size_t* fulls[] = {&w.do_fg, &w.do_l, &w.dq_fg, &w.dq_l, &w.dk_fg, &w.dk_l, &w.dv_fg, &w.dv_l};
+  for (size_t* f : fulls) { *f = at; at += full; }
+  w.inner = at;  // the attention backward's layout starts with a status block of its own (unused here)
+  w.total = at + bwd_layout(g).total;
+  return w;
+}
 size_t select_total(const Geo& g) { return select_layout(g).total; }
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
@@ -132,6 +160,7 @@ size_t mosaic_bsa_workspace_bytes(const mosaic_bsa_params* p, int op) {
     case MOSAIC_OP_FWD: return kStatusBytes;
     case MOSAIC_OP_BWD: return bwd_layout(g).total;
     case MOSAIC_OP_FWD_BRANCHES: return branch_layout(g).total;
+    case MOSAIC_OP_BWD_BRANCHES: return bwd_branch_layout(g).total;
     default: return 0;
   }
 }
@@ -187,7 +216,7 @@ int mosaic_bsa_fwd_branches(const mosaic_bsa_params* p, const void* q, const voi
   cp.g.topk = 0;  // pooling only
   if ((rc = launch_select(cp, q, k, nullptr, pq, pk, nrm, nrm + (size_t)g.U * g.m))) return rc;
   if ((rc = launch_pool_one(c, v, pv, nrm, g.Ukv))) return rc;
-  if ((rc = launch_compress(c, pq, pk, pv, ocg))) return rc;
+  if ((rc = launch_compress(c, pq, pk, pv, ocg, nullptr))) return rc;
   // local branch: the neighbourhood only (no selected blocks); work queue in the second word of the status block
   HostCtx cl = c;
   cl.g.topk = 0;
@@ -218,7 +247,70 @@ int mosaic_bsa_bwd(const mosaic_bsa_params* p, const void* q, const void* k, con
   char* base = (char*)ws;
   return launch_bwd(c, q, k, v, o, lse, d_o, block_idx, dq, dk, dv, (float*)(base + w.D),
                     (float*)(base + w.negD), (float*)(base + w.nlse2), (int32_t*)(base + w.off),
-                    (int32_t*)(base + w.q), (int32_t*)(base + w.order));
+                    (int32_t*)(base + w.q), (int32_t*)(base + w.order), c.status + 1);
+}
+
+int mosaic_bsa_bwd_branches(const mosaic_bsa_params* p, const void* q, const void* k, const void* v,
+                            const int32_t* block_idx, const float* gates, const void* d_o, void* dq, void* dk,
+                            void* dv, float* dgates, void* ws, size_t ws_bytes, void* cuda_stream) {
+  HostCtx c;
+  Geo g;
+  int rc = validate(p, &g);
+  if (rc) return rc;
+  if (!q || !k || !v || !gates || !d_o || !dq || !dk || !dv || !dgates || (!block_idx && g.topk > 0))
+    return MOSAIC_E_INVALID_ARG;
+  const void* ptrs[] = {q, k, v, d_o, dq, dk, dv};
+  for (const void* x : ptrs)
+    if (!aligned(x, 16)) return MOSAIC_E_MISALIGNED;
+  if (!aligned(gates, 4) || !aligned(dgates, 4) || !aligned(block_idx, 4)) return MOSAIC_E_MISALIGNED;
+  if (2 * (size_t)g.m * sizeof(int) + (size_t)g.m * g.topk / 8 + 8 > 200 * 1024) return MOSAIC_E_UNSUPPORTED;  // transposed-pattern kernel
+  const BwdBranchWs w = bwd_branch_layout(g);
+  if ((rc = begin(p, ws, ws_bytes, w.total, cuda_stream, &c))) return rc;
+  char* base = (char*)ws;
+  auto F = [&](size_t off) { return (float*)(base + off); };
+  float *pq = F(w.f.pq), *pk = F(w.f.pk), *pv = F(w.f.pv), *nrm = F(w.f.nrm), *ocg = F(w.f.ocg);
+  void *ofg = base + w.f.ofg, *ol = base + w.f.ol;
+  // the forward again: pooled sums, block-level attention (with its log-sum-exp), both attention branches
+  HostCtx cp = c;
+  cp.g.topk = 0;  // pooling only
+  if ((rc = launch_select(cp, q, k, nullptr, pq, pk, nrm, nrm + (size_t)g.U * g.m))) return rc;
+  if ((rc = launch_pool_one(c, v, pv, nrm, g.Ukv))) return rc;
+  if ((rc = launch_compress(c, pq, pk, pv, ocg, F(w.lse_cg)))) return rc;
+  HostCtx cl = c;
+  cl.g.topk = 0;          // local branch: the neighbourhood only
+  HostCtx cs = c;
+  cs.g.local_off = 1;     // selection branch: the selected blocks only
+  const bool sel = g.topk > 0;
+  if ((rc = launch_fwd_tc(cl, q, k, v, nullptr, ol, F(w.lse_l), c.status + 1))) return rc;
+  if (sel) {
+    if ((rc = launch_fwd_tc(cs, q, k, v, block_idx, ofg, F(w.lse_fg), c.status + 2))) return rc;
+  } else if (cudaMemsetAsync(ofg, 0, 2 * (size_t)g.U * g.N * kD, c.stream) != cudaSuccess) {
+    return MOSAIC_E_CUDA;
+  }
+  // gate gradients, gated copies of dO, gated block sums of dO
+  if ((rc = launch_gate(c, d_o, ofg, ol, ocg, gates, dgates, base + w.do_fg, base + w.do_l, F(w.dob)))) return rc;
+  // compression branch on the block level
+  if ((rc = launch_compress_bwd(c, pq, pk, pv, F(w.dob), ocg, F(w.lse_cg), F(w.delta), F(w.dqm), F(w.dkm), F(w.dvm))))
+    return rc;
+  // the two attention branches, one after the other on the same scratch
+  const BwdWs bw = bwd_layout(g);
+  char* in = base + w.inner;
+  auto attention_bwd = [&](const HostCtx& cx, const void* o_x, const float* lse_x, const void* do_x, const int32_t* idx,
+                           void* dq_x, void* dk_x, void* dv_x, int* counters) {
+    return launch_bwd(cx, q, k, v, o_x, lse_x, do_x, idx, dq_x, dk_x, dv_x, (float*)(in + bw.D), (float*)(in + bw.negD),
+                      (float*)(in + bw.nlse2), (int32_t*)(in + bw.off), (int32_t*)(in + bw.q), (int32_t*)(in + bw.order),
+                      counters);
+  };
+  if ((rc = attention_bwd(cl, ol, F(w.lse_l), base + w.do_l, nullptr, base + w.dq_l, base + w.dk_l, base + w.dv_l,
+                          c.status + 3)))
+    return rc;
+  if (sel && (rc = attention_bwd(cs, ofg, F(w.lse_fg), base + w.do_fg, block_idx, base + w.dq_fg, base + w.dk_fg,
+                                 base + w.dv_fg, c.status + 5)))
+    return rc;
+  // sums: both attention branches plus what the compression branch gives every token of a block
+  if ((rc = launch_grad_sum(c, g.U, base + w.dq_l, sel ? base + w.dq_fg : nullptr, F(w.dqm), dq))) return rc;
+  if ((rc = launch_grad_sum(c, g.Ukv, base + w.dk_l, sel ? base + w.dk_fg : nullptr, F(w.dkm), dk))) return rc;
+  return launch_grad_sum(c, g.Ukv, base + w.dv_l, sel ? base + w.dv_fg : nullptr, F(w.dvm), dv);
 }
 
 int mosaic_bsa_last_status(const void* ws, void* cuda_stream) {

@@ -35,7 +35,7 @@ struct CompressSmem {
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kCW * 32) compress_kernel(Geo g, const float* __restrict__ pq,
                                                             const float* __restrict__ pk, const float* __restrict__ pv,
-                                                            float* __restrict__ ocg) {
+                                                            float* __restrict__ ocg, float* __restrict__ lse2) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   CompressSmem& sm = *reinterpret_cast<CompressSmem*>(smem_raw);
   constexpr int TI = kCW * kCR, NT = kCW * 32;
@@ -125,6 +125,8 @@ __global__ void __launch_bounds__(kCW * 32) compress_kernel(Geo g, const float* 
     if (i < g.m) {
       const float f = inv_b / zz;
       *reinterpret_cast<float2*>(ocg + ((long long)u * g.m + i) * kD + 2 * lane) = make_float2(acc[a][0] * f, acc[a][1] * f);
+      // base-2 log-sum-exp of the row's block-level logits, for the backward (which recomputes abar from it)
+      if (lse2 && lane == 0) lse2[(long long)u * g.m + i] = mx[a] + log2f(zz);
     }
   }
 }
@@ -163,7 +165,8 @@ __global__ void __launch_bounds__(256) combine_kernel(Geo g, const float* __rest
 
 }  // namespace
 
-int launch_compress(const HostCtx& c, const float* pooled_q, const float* pooled_k, const float* pooled_v, float* ocg) {
+int launch_compress(const HostCtx& c, const float* pooled_q, const float* pooled_k, const float* pooled_v, float* ocg,
+                    float* lse2) {
   const Geo& g = c.g;
   const size_t smem = sizeof(CompressSmem);
   static unsigned long long configured = 0;  // devices on which the kernel's shared-memory opt-in is set
@@ -176,7 +179,7 @@ int launch_compress(const HostCtx& c, const float* pooled_q, const float* pooled
     configured |= 1ull << dev;
   }
   const int tiles = (g.m + kCW * kCR - 1) / (kCW * kCR);
-  compress_kernel<<<(unsigned)(g.U * tiles), kCW * 32, smem, c.stream>>>(g, pooled_q, pooled_k, pooled_v, ocg);
+  compress_kernel<<<(unsigned)(g.U * tiles), kCW * 32, smem, c.stream>>>(g, pooled_q, pooled_k, pooled_v, ocg, lse2);
   return cudaGetLastError() == cudaSuccess ? MOSAIC_OK : MOSAIC_E_CUDA;
 }
 

@@ -147,7 +147,7 @@ static int csr_segments(const Geo& g, size_t* smem) {
 int launch_bwd(const HostCtx& c, const void* q, const void* k, const void* v, const void* o, const float* lse,
                const void* d_o, const int32_t* block_idx, void* dq, void* dk, void* dv, float* Dbuf, float* neg_d,
                float* neg_lse2,
-               int32_t* csr_off, int32_t* csr_q, int32_t* order) {
+               int32_t* csr_off, int32_t* csr_q, int32_t* order, int* counters) {
   const Geo& g = c.g;
   const long long tokens = (long long)g.U * g.N;
   {
@@ -175,14 +175,13 @@ int launch_bwd(const HostCtx& c, const void* q, const void* k, const void* v, co
   }
   if (cudaGetLastError() != cudaSuccess) return MOSAIC_E_CUDA;
   {
-    // dQ on the tcgen05 path; its work queue counts in the second word of the status block (zeroed when the
-    // op started)
-    const int rc = launch_dq_tc(c, q, k, v, d_o, lse, Dbuf, block_idx, dq, c.status + 1);
+    // dQ on the tcgen05 path; its work queue counts in a word of the status block (zeroed when the op started)
+    const int rc = launch_dq_tc(c, q, k, v, d_o, lse, Dbuf, block_idx, dq, counters);
     if (rc) return rc;
   }
   {
-    // dK, dV on the tcgen05 path; its work queue counts in the third word of the status block
-    const int rc = launch_dkdv_tc(c, q, k, v, d_o, neg_lse2, neg_d, csr_off, csr_q, dk, dv, c.status + 2, order);
+    // dK, dV on the tcgen05 path; its work queue counts in the next word
+    const int rc = launch_dkdv_tc(c, q, k, v, d_o, neg_lse2, neg_d, csr_off, csr_q, dk, dv, counters + 1, order);
     if (rc) return rc;
   }
   return MOSAIC_OK;

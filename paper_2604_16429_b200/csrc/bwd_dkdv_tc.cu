@@ -530,6 +530,15 @@ __global__ void __launch_bounds__(kThreads, 1)
           __syncwarp();
           if (lane == 0) mbar_arrive(s32(&sm.acc_free));
           ++items;
+        } else if ((sm.info[buf].hvalid >> hh) & 1) {
+          // a tile that no query block is connected to (possible when the local set is switched off): zero gradients
+          const long long tok = (long long)sm.info[buf].kvunit * g.N +
+                                chunk_token(g, sm.info[buf].hb[hh], sm.info[buf].hc[hh], (quad & 1) * 32 + lane);
+          const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+          uint4* dst_k = reinterpret_cast<uint4*>(dk + tok * kD + 16 * cq);
+          uint4* dst_v = reinterpret_cast<uint4*>(dv + tok * kD + 16 * cq);
+          dst_k[0] = zero; dst_k[1] = zero;
+          dst_v[0] = zero; dst_v[1] = zero;
         }
         item_chunks = 0;
       }

@@ -314,6 +314,11 @@ __global__ void __launch_bounds__(kThreads, 1)
               dst[part * 4 + i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
           }
         }
+      } else if (valid) {
+        // a tile whose rows attend nothing (possible when the local set is switched off): zero gradient
+        uint4* dst = reinterpret_cast<uint4*>(dq + tok * kD);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) dst[i] = make_uint4(0u, 0u, 0u, 0u);
       }
       tc_fence_before();
       __syncwarp();

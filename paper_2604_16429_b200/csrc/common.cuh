@@ -113,7 +113,15 @@ int launch_fwd_tc(const HostCtx& c, const void* q, const void* k, const void* v,
 struct BranchWs { size_t pq, pk, pv, nrm, ocg, ofg, ol, total; };
 BranchWs branch_layout(const Geo& g);
 int launch_pool_one(const HostCtx& c, const void* x, float* pooled, float* norm, int units);
-int launch_compress(const HostCtx& c, const float* pooled_q, const float* pooled_k, const float* pooled_v, float* ocg);
+// `lse2` (may be null): base-2 log-sum-exp of every query block's block-level logits, [U, m]
+int launch_compress(const HostCtx& c, const float* pooled_q, const float* pooled_k, const float* pooled_v, float* ocg,
+                    float* lse2);
+// backward of the three-branch form (branches_bwd.cu)
+int launch_gate(const HostCtx& c, const void* d_o, const void* o_fg, const void* o_l, const float* ocg,
+                const float* gates, float* dgates, void* do_fg, void* do_l, float* dob);
+int launch_compress_bwd(const HostCtx& c, const float* pq, const float* pk, const float* pv, const float* dob,
+                        const float* ocg, const float* lse2, float* delta, float* dqm, float* dkm, float* dvm);
+int launch_grad_sum(const HostCtx& c, int units, const void* x_l, const void* x_fg, const float* xm, void* out);
 int launch_combine(const HostCtx& c, const float* ocg, const void* o_fg, const void* o_l, const float* gates, void* o);
 int launch_dq_tc(const HostCtx& c, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
                  const float* D, const int32_t* block_idx, void* dq, int* work_counter);
@@ -122,6 +130,6 @@ int launch_dkdv_tc(const HostCtx& c, const void* q, const void* k, const void* v
                    void* dv, int* work_counter, int32_t* order);
 int launch_bwd(const HostCtx& c, const void* q, const void* k, const void* v, const void* o, const float* lse,
                const void* d_o, const int32_t* block_idx, void* dq, void* dk, void* dv, float* Dbuf, float* neg_d,
-               float* neg_lse2, int32_t* csr_off, int32_t* csr_q, int32_t* order);
+               float* neg_lse2, int32_t* csr_off, int32_t* csr_q, int32_t* order, int* counters);
 
 }  // namespace mosaic

@@ -101,3 +101,89 @@ def test_three_branch_at_the_1p5_degree_size_sampled_units():
         bound = G.FWD_MAX_ABS * np.maximum(1.0, np.abs(gates[0, h]).sum(axis=1, keepdims=True))
         assert (np.abs(o[0, h] - r["o"]) <= bound).all()
         assert np.abs(lf[0, h] - r["lse_fg"]).max() <= G.LSE_ABS and np.abs(ll[0, h] - r["lse_l"]).max() <= G.LSE_ABS
+
+
+# ---------------------------------------------------------------------------------------------------------
+# Backward of the three-branch form against the oracle's `bwd3`.
+# Tolerances: dQ, dK, dV are sums of two bf16 branch gradients and the compression branch's fp32 share, rounded to
+# bf16 once more: three roundings of 2^-9 relative on values of a few units, on top of the attention backward's own
+# error, so the bound is the attention backward's (5e-2) plus 2^-8 of the largest reference magnitude.  The gate
+# gradients are dot products of dO with bf16 branch outputs whose own error is bounded by the forward tolerance:
+# |error| <= sum_c |dO_c| * err_c, taken here as FWD_MEAN_ABS * sum_c |dO_c| * 4 (errors do not add coherently).
+BWD3_CASES = [
+    synth.small_case(32, 64, 8, 8, 4, B=1, H=2, seed=91, backward=True),
+    synth.small_case(40, 56, 8, 8, 5, B=1, H=1, kind="smooth", seed=92, backward=True),       # odd block grid
+    synth.small_case(32, 64, 16, 16, 3, B=1, H=1, kind="smooth", seed=93, backward=True),     # 16x16 blocks
+    synth.small_case(256, 16, 8, 16, 3, B=1, H=4, kind="smooth", seed=94, rlat=8, rlon=1, backward=True,
+                     local_groups=True, Hkv=2),                                               # the paper's layout, GQA
+]
+
+
+def _run_bwd3(w, x, idx, gates):
+    p = mb.Params.from_workload(w)
+    dx = G.device_inputs(x)
+    ws = G.Guarded((mb.workspace_bytes(p, mb.OP_BWD_BRANCHES),), torch.uint8)
+    dq = G.Guarded(tuple(dx["q"].shape), torch.bfloat16, fill=float("nan"))
+    dk = G.Guarded(tuple(dx["k"].shape), torch.bfloat16, fill=float("nan"))
+    dv = G.Guarded(tuple(dx["k"].shape), torch.bfloat16, fill=float("nan"))
+    dg = G.Guarded((w.B, w.H, w.N, 3), torch.float32, fill=float("nan"))
+    gt = torch.from_numpy(gates.astype(np.float32)).cuda().contiguous()
+    mb.mosaic_bsa_bwd_branches(p, dx["q"], dx["k"], dx["v"], idx, gt, dx["do"], dq=dq.t, dk=dk.t, dv=dv.t, dgates=dg.t, ws=ws.t)
+    mb.check_status(ws.t, "bwd_branches")
+    for b_, n_ in ((ws, "workspace"), (dq, "dq"), (dk, "dk"), (dv, "dv"), (dg, "dgates")):
+        b_.check(n_)
+    return [t.t.float().cpu().numpy().astype(np.float64) for t in (dq, dk, dv, dg)]
+
+
+def _compare_bwd3(w, x, idx_h, gates, got):
+    dq, dk, dv, dg = got
+    g = G.geom_of(w)
+    r = w.H // w.kv_heads
+    do_abs = np.abs(synth.bf16_bits_to_f32(x["do"]).astype(np.float64)).sum(axis=-1)     # [B, H, N]
+    for b in range(w.B):
+        for hk in range(w.kv_heads):
+            dK_sum, dV_sum = np.zeros((w.N, w.d)), np.zeros((w.N, w.d))
+            for h in range(hk * r, (hk + 1) * r):
+                gq = gates[b, h].astype(np.float32).astype(np.float64)
+                dQ, dK, dV, dG = oracle.bwd3(g, x["q"][b, h], x["k"][b, hk], x["v"][b, hk], x["do"][b, h], idx_h[b, h], gq)
+                tol = G.BWD_MAX_ABS + 2.0 ** -8 * np.abs(dQ).max()
+                assert np.isfinite(dq[b, h]).all() and np.abs(dq[b, h] - dQ).max() <= tol, (h, np.abs(dq[b, h] - dQ).max(), tol)
+                bound = 4 * G.FWD_MEAN_ABS * do_abs[b, h][:, None] + 1e-3
+                assert np.isfinite(dg[b, h]).all() and (np.abs(dg[b, h] - dG) <= bound).all(), (h, np.abs(dg[b, h] - dG).max())
+                dK_sum += dK
+                dV_sum += dV
+            for name, a, ref in (("dK", dk[b, hk], dK_sum), ("dV", dv[b, hk], dV_sum)):
+                tol = G.BWD_MAX_ABS + 2.0 ** -8 * np.abs(ref).max()
+                assert np.isfinite(a).all() and np.abs(a - ref).max() <= tol, (name, hk, np.abs(a - ref).max(), tol)
+
+
+@pytest.mark.parametrize("w", BWD3_CASES, ids=lambda w: w.name)
+def test_three_branch_backward_matches_oracle(w):
+    x = synth.make_inputs(w)
+    idx = G.gpu_select(w, G.device_inputs(x))
+    gates = np.random.default_rng(w.cfg).standard_normal((w.B, w.H, w.N, 3))
+    _compare_bwd3(w, x, idx.cpu().numpy(), gates, _run_bwd3(w, x, idx, gates))
+
+
+def test_three_branch_backward_one_branch_at_a_time_and_empty_rows():
+    """Each gate alone isolates one branch (the compression branch alone reaches every key and value of the unit);
+    a query block that selects nothing and key blocks nobody selected get zero from the selection branch."""
+    w = synth.small_case(32, 64, 8, 8, 4, B=1, H=1, seed=95, backward=True)
+    x = synth.make_inputs(w)
+    idx = G.gpu_select(w, G.device_inputs(x))
+    idx[0, 0, 5, :] = -1
+    idx[0, 0, 6, 1:] = -1
+    j0 = int(idx[0, 0, 0, 0])
+    idx[idx == j0] = -1                                    # a key block that nobody selects
+    idx_h = idx.cpu().numpy()
+    for col in range(3):
+        gates = np.zeros((1, 1, w.N, 3)); gates[..., col] = 1.0
+        got = _run_bwd3(w, x, idx, gates)
+        _compare_bwd3(w, x, idx_h, gates, got)
+        if col == 0:
+            assert (np.abs(got[1][0, 0]).max(axis=1) > 0).all() and (np.abs(got[2][0, 0]).max(axis=1) > 0).all()
+        if col == 1:
+            tok5 = oracle.block_tokens(G.geom_of(w), 5)
+            assert np.all(got[0][0, 0][tok5] == 0)
+            tu = oracle.block_tokens(G.geom_of(w), j0)
+            assert np.all(got[1][0, 0][tu] == 0) and np.all(got[2][0, 0][tu] == 0)

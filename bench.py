@@ -374,7 +374,23 @@ def run_ours(args, w):
     torch.cuda.synchronize()
     mb.check_status(ws3, "three-branch forward")
     t_br = sum(e[0].elapsed_time(e[1]) for e in ev3) / k3
-    del ws3, gates, lse_fg, lse_l
+    del ws3, lse_fg, lse_l
+    # and its backward (recomputes the forward's intermediates; gradient of the gates included)
+    ws3b = torch.empty(mb.workspace_bytes(p, mb.OP_BWD_BRANCHES), dtype=torch.uint8, device=dev)
+    dgates = torch.empty_like(gates)
+    k3b = min(K, 20)
+    ev3b = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(k3b)]
+    for s in range(k3b + 2):
+        flush_buf.zero_()
+        if s >= 2:
+            ev3b[s - 2][0].record(stream)
+        mb.mosaic_bsa_bwd_branches(p, dx["q"], dx["k"], dx["v"], idx, gates, dx["do"], dq=dq, dk=dk, dv=dv, dgates=dgates, ws=ws3b)
+        if s >= 2:
+            ev3b[s - 2][1].record(stream)
+    torch.cuda.synchronize()
+    mb.check_status(ws3b, "three-branch backward")
+    t_brb = sum(e[0].elapsed_time(e[1]) for e in ev3b) / k3b
+    del ws3b, gates, dgates
 
     # end to end: pinned host -> device, step, device -> pinned host
     ke = min(K, 20)
@@ -419,7 +435,7 @@ def run_ours(args, w):
                      "traffic": traffic, "traffic_source": traffic_source, "peak_source": peaks["source"] + " (burst)",
                      "frac_of_nominal_2250": fwd_tflops / NOMINAL_BF16_TFLOPS, "ms": t_fwd},
         "stages": {"select_ms": t_sel, "fwd_ms": t_fwd, "bwd_ms": t_bwd, "ms_layer_fwd": t_step,
-                   "fwd_three_branch_ms": t_br,
+                   "fwd_three_branch_ms": t_br, "bwd_three_branch_ms": t_brb,
                    "fwd_tflops": fwd_tflops, "bwd_tflops": flops.bwd_flops(w) / (t_bwd * 1e-3) / 1e12,
                    "select_pool_gbs_lower_bound": pool_bytes / (t_sel * 1e-3) / 1e9,
                    "pct_of_nominal_peak": 100 * fwd_tflops / NOMINAL_BF16_TFLOPS,

@@ -53,6 +53,7 @@ struct Smem {
   Slot ring[kSlots];
   unsigned long long ring_full[kSlots], ring_empty[kSlots];
   unsigned long long kv_full, kv_empty, s_full, sdp_free, p_full[2], pv_done, acc_done, acc_free;
+  unsigned long long mma_drain_bar[2];  // abort path: completion of each issuer's outstanding products
   unsigned long long list_full[kLists], list_empty[kLists];
   uint32_t tmem_base;
   int abort;
@@ -231,6 +232,8 @@ __global__ void __launch_bounds__(kThreads, 1)
     mbar_init(s32(&sm.pv_done), 1);
     mbar_init(s32(&sm.acc_done), 1);
     mbar_init(s32(&sm.acc_free), kRowWarps);
+    mbar_init(s32(&sm.mma_drain_bar[0]), 1);
+    mbar_init(s32(&sm.mma_drain_bar[1]), 1);
     for (int i = 0; i < kLists; ++i) {
       mbar_init(s32(&sm.list_full[i]), 1);
       mbar_init(s32(&sm.list_empty[i]), kRowWarps + 3);  // row-thread warps + 2 MMA issuers + TMA producer
@@ -305,9 +308,10 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
         if (ok) mbar_arrive(s32(&sm.list_empty[buf]));
       }
-      if (*abort) {  // give copies in flight time to land before the CTA's memory is released
-        const long long t0 = clock64();
-        while (clock64() - t0 < 400000) {}
+      if (*abort) {  // copies this thread issued must land before the CTA's memory is released
+        const long long first = pr > kSlots ? pr - kSlots : 0;
+        for (long long s = first; s < pr; ++s) mbar_drain(s32(&sm.ring_full[s % kSlots]), (uint32_t)((s / kSlots) & 1));
+        if (items > 0) mbar_drain(s32(&sm.kv_full), (uint32_t)((items - 1) & 1));
       } else {       // drain: the last uses of every ring slot have been released
         const long long first = pr > kSlots ? pr - kSlots : 0;
         for (long long s = first; s < pr; ++s)
@@ -356,6 +360,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         if (ok && !more) tc_commit(s32(&sm.kv_empty));
         if (ok) mbar_arrive(s32(&sm.list_empty[buf]));
       }
+      if (*abort) mma_drain(s32(&sm.mma_drain_bar[0]));  // products already issued must finish before the release
     }
   } else if (warp == kWMma1) {
     // ------------------------------------------------------------- issuer of dV += P^T dO and dK += dS^T Q (one thread)
@@ -407,6 +412,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
         if (ok) mbar_arrive(s32(&sm.list_empty[buf]));
       }
+      if (*abort) mma_drain(s32(&sm.mma_drain_bar[1]));
     }
   } else if (warp < kRowWarps) {
     // ------------------------------------------------------------- row threads (TMEM lane = key row)

@@ -33,6 +33,7 @@ struct Smem {
   unsigned char kv[kStages][2][kTile];     // [stage][K, V]
   unsigned long long kv_full[kStages], kv_empty[kStages];
   unsigned long long q_full[2], q_empty[2], s_full[2], sdp_free[2], p_full[2], pv_done[2];  // [tile]
+  unsigned long long mma_drain_bar[2];  // abort path: completion of each issuer's outstanding products
   unsigned long long list_full[kLists], list_empty[kLists];
   uint32_t tmem_base;
   int abort;
@@ -59,6 +60,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     for (int t = 0; t < 2; ++t) {
       mbar_init(s32(&sm.q_full[t]), 1);
       mbar_init(s32(&sm.q_empty[t]), 1);
+      mbar_init(s32(&sm.mma_drain_bar[t]), 1);
       mbar_init(s32(&sm.s_full[t]), 1);
       mbar_init(s32(&sm.sdp_free[t]), 128);
       mbar_init(s32(&sm.p_full[t]), 128);
@@ -92,6 +94,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     // ------------------------------------------------------------- TMA producer
     if (lane == 0) {
       long long step = 0;  // key/value chunks issued so far (ring position)
+      int q_armed[2] = {-1, -1};  // phase parity of the last load into each tile's Q / dO buffer
       bool ok = true;
       for (int it = 0; ok; ++it) {
         const int buf = it % kLists;
@@ -106,6 +109,7 @@ __global__ void __launch_bounds__(kThreads, 1)
           ok = mbar_wait(s32(&sm.q_empty[t]), (it & 1) ^ 1, abort, status);
           if (!ok) break;
           mbar_expect_tx(s32(&sm.q_full[t]), 4 * kTile);
+          q_armed[t] = it & 1;
           for (int hh = 0; hh < 2; ++hh) {
             const int h = 2 * t + hh, by = inf.hb[h] / g.nbw, bx = inf.hb[h] - by * g.nbw;
             tma_load_4d(s32(sm.q[t] + hh * kTile), &map_q, s32(&sm.q_full[t]), 0, bx * g.bw,
@@ -127,9 +131,11 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
         if (ok) mbar_arrive(s32(&sm.list_empty[buf]));
       }
-      if (*abort) {  // give copies in flight time to land before the CTA's memory is released
-        const long long t0 = clock64();
-        while (clock64() - t0 < 400000) {}
+      if (*abort) {  // copies this thread issued must land before the CTA's memory is released
+        const long long first = step > kStages ? step - kStages : 0;
+        for (long long s = first; s < step; ++s) mbar_drain(s32(&sm.kv_full[s % kStages]), (uint32_t)((s / kStages) & 1));
+        for (int t = 0; t < 2; ++t)
+          if (q_armed[t] >= 0) mbar_drain(s32(&sm.q_full[t]), (uint32_t)q_armed[t]);
       } else {       // drain: the last uses of every ring stage have been released by both tiles
         const long long first = step > kStages ? step - kStages : 0;
         for (long long s = first; s < step; ++s)
@@ -215,6 +221,10 @@ __global__ void __launch_bounds__(kThreads, 1)
       }
       if (ok && pend) issue_dq(pend_st, pend_first);  // the item's last product
       if (ok && elect_one()) mbar_arrive(s32(&sm.list_empty[buf]));
+    }
+    if (*abort) {  // products already issued must finish before TMEM and shared memory are released
+      if (elect_one()) mma_drain(s32(&sm.mma_drain_bar[t]));
+      __syncwarp();
     }
   } else {
     // ------------------------------------------------------------- row threads of tile t: S, dP -> dS; then epilogue

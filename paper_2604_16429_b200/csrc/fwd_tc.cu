@@ -55,6 +55,7 @@ struct Smem {
   unsigned char kv[kStages][2][kTile];     // [stage][K, V]
   unsigned long long kv_full[kStages], kv_empty[kStages];
   unsigned long long q_full[2][2], q_empty[2][2];  // [item parity][tile]
+  unsigned long long mma_drain_bar[2];             // abort path: completion of each issuer's outstanding products
   unsigned long long q_ready[2];                   // [tile]: the item's query rows are in TMEM
   unsigned long long s_full[2][2], p_full[2][2], pv_done[2][2];  // [tile][S buffer]
   unsigned long long list_full[kLists], list_empty[kLists];
@@ -83,6 +84,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     for (int t = 0; t < 2; ++t) {
       for (int b = 0; b < 2; ++b) {
         mbar_init(s32(&sm.q_full[b][t]), 1);
+        if (t == 0) mbar_init(s32(&sm.mma_drain_bar[b]), 1);
         mbar_init(s32(&sm.q_empty[b][t]), 128);
       }
       mbar_init(s32(&sm.q_ready[t]), 128);
@@ -120,6 +122,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     // ------------------------------------------------------------- TMA producer
     if (lane == 0) {
       long long step = 0;  // key/value chunks issued so far (ring position)
+      int q_armed[2][2] = {{-1, -1}, {-1, -1}};  // phase parity of the last load into each query-tile buffer
       bool ok = true;
       for (int it = 0; ok; ++it) {
         const int buf = it % kLists, qb = it & 1;
@@ -135,6 +138,7 @@ __global__ void __launch_bounds__(kThreads, 1)
           ok = mbar_wait(s32(&sm.q_empty[qb][t]), ((it >> 1) & 1) ^ 1, abort, status);
           if (!ok) break;
           mbar_expect_tx(s32(&sm.q_full[qb][t]), 2 * kTile);
+          q_armed[qb][t] = (it >> 1) & 1;
           for (int hh = 0; hh < 2; ++hh) {
             const int h = 2 * t + hh, by = inf.hb[h] / g.nbw, bx = inf.hb[h] - by * g.nbw;
             tma_load_4d(s32(sm.q[qb][t] + hh * kTile), &map_q, s32(&sm.q_full[qb][t]), 0, bx * g.bw,
@@ -159,9 +163,11 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
         if (ok) mbar_arrive(s32(&sm.list_empty[buf]));
       }
-      if (*abort) {  // give copies in flight time to land before the CTA's memory is released
-        const long long t0 = clock64();
-        while (clock64() - t0 < 400000) {}
+      if (*abort) {  // copies this thread issued must land before the CTA's memory is released
+        const long long first = step > kStages ? step - kStages : 0;
+        for (long long s = first; s < step; ++s) mbar_drain(s32(&sm.kv_full[s % kStages]), (uint32_t)((s / kStages) & 1));
+        for (int i = 0; i < 4; ++i)
+          if (q_armed[i >> 1][i & 1] >= 0) mbar_drain(s32(&sm.q_full[i >> 1][i & 1]), (uint32_t)q_armed[i >> 1][i & 1]);
       } else {       // drain: the last uses of every ring stage have been released by both tiles
         const long long first = step > kStages ? step - kStages : 0;
         for (long long s = first; s < step; ++s)
@@ -238,6 +244,10 @@ __global__ void __launch_bounds__(kThreads, 1)
       }
       if (ok && pend) issue_pv(pend_n, pend_st, pend_first);  // the item's last product
       if (ok && elect_one()) mbar_arrive(s32(&sm.list_empty[buf]));
+    }
+    if (*abort) {  // products already issued must finish before TMEM and shared memory are released
+      if (elect_one()) mma_drain(s32(&sm.mma_drain_bar[t]));
+      __syncwarp();
     }
   } else {
     // ------------------------------------------------------------- softmax of tile t, then epilogue

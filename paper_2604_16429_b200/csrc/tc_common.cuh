@@ -85,6 +85,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   return mbar_wait_slow(bar, parity, abort, status);
 }
 
+// Abort path only: a bounded wait for phase `parity` of `bar` that records nothing.  After a failed wait the roles
+// leave their loops with copies and tensor-core work possibly still in flight; the producer waits on the barriers it
+// armed and each MMA issuer commits and waits once more, so that shared memory and TMEM are released only after
+// everything that was issued has landed or run out of this (second, shorter) bound.
+constexpr long long kDrainCycles = 4000000;  // about 2 ms per barrier
+__device__ __forceinline__ bool mbar_drain(uint32_t bar, uint32_t parity) {
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity))
+    if (clock64() - t0 > kDrainCycles) return false;
+  return true;
+}
 // Warp-wide wait: lane 0 polls, the warp learns the outcome and synchronises (polls by all 32 lanes serialise on the
 // barrier word and cost several times as much).  What lane 0 acquired is visible to the warp after the barrier.
 __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort, int* status, int lane) {
@@ -115,6 +126,12 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// One thread's tensor-core work issued so far has completed (or the bound ran out): commit to a barrier of its
+// own (count 1, never used before) and wait for it.
+__device__ __forceinline__ void mma_drain(uint32_t bar) {
+  tc_commit(bar);
+  mbar_drain(bar, 0);
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }

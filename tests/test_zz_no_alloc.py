@@ -45,3 +45,20 @@ def test_static_scratch_rejects_problems_beyond_its_size():
     pc = p.c()
     rc = mb.lib().mosaic_bsa_select_static(ctypes.byref(pc), 256, 256, 256, None)   # never dereferenced: the size check comes first
     assert rc == -3 and "workspace" in mb.strerror(rc)
+
+
+def test_static_scratch_selection_takes_no_device_memory():
+    """Free device memory as the driver reports it is the same before and after a call that has run once before
+    (the first call may load the library's module; the caller's tensors exist before the measurement)."""
+    w = synth.small_case(32, 64, 8, 8, 4, B=1, H=3, seed=63)
+    x = synth.make_inputs(w)
+    q, k = mb.from_bits(x["q"]), mb.from_bits(x["k"])
+    p = mb.Params.from_workload(w)
+    out = torch.empty((w.B, w.H, w.m, w.topk), dtype=torch.int32, device="cuda")
+    mb.mosaic_bsa_select_static(p, q, k, block_idx=out)
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    mb.mosaic_bsa_select_static(p, q, k, block_idx=out)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before

@@ -227,6 +227,21 @@ def bwd3(g: Geom, q, k, v, d_o, idx, gates):
     return dQ, dK, dV, dG
 
 
+def rope(g: Geom, x, pos, theta=10000.0):
+    """2-D rotary position embedding of one [N, d] tensor (bf16 bits); pos is [N, 2] = (longitude, latitude) in
+    radians.  Returns (fp64 unrounded [N, d], bf16 bits [N, d])."""
+    x = _u16(x, g)
+    pos = np.ascontiguousarray(pos, np.float64)
+    assert pos.shape == (g.N, 2)
+    out = np.zeros((g.N, g.d))
+    bits = np.zeros((g.N, g.d), np.uint16)
+    gc = g.c()
+    rc = _load().mo_rope_unit(ctypes.byref(gc), _p(x, ctypes.c_uint16), _p(pos, ctypes.c_double), ctypes.c_double(theta),
+                              _p(out, ctypes.c_double), _p(bits, ctypes.c_uint16))
+    assert rc == 0
+    return out, bits
+
+
 def block_tokens(g: Geom, j: int) -> np.ndarray:
     """Token ids of block j in row-major order inside the block (layout helper)."""
     by, bx = divmod(j, g.nbw)

@@ -757,3 +757,42 @@ int mo_bwd3_unit(const mo_geom *g, const uint16_t *q, const uint16_t *k, const u
   free(dob); free(dqm); free(dkm); free(dvm);
   return 0;
 }
+
+/*
+ * Two-dimensional rotary position embedding of one [N, d] tensor ("Overall architecture" paragraph: RoPE on
+ * queries and keys encodes longitude and latitude, the head dimension split equally between the two
+ * coordinates, each half a standard RoPE of its angle in radians; architecture table: theta = 10000).
+ * Reading: channels [0, d/2) belong to the longitude, [d/2, d) to the latitude; inside a half of width
+ * D = d/2 the pair (2i, 2i+1), i < D/2, turns by the angle  pos * theta^(-2i/D):
+ *     y_2i = x_2i cos a - x_2i+1 sin a ,   y_2i+1 = x_2i sin a + x_2i+1 cos a .
+ * pos: [N, 2] = (longitude, latitude) of every token in radians.  out: fp64, unrounded (may be NULL);
+ * out_bits: the same rounded to bf16, nearest even (may be NULL).
+ */
+static uint16_t bf16_round(double x) {
+  float f = (float)x; /* double -> float -> bf16: the float has 24 bits, bf16 keeps 8; ties of the second step are
+                         decided on the float, which is what a device that computes in fp32 does too */
+  uint32_t u;
+  memcpy(&u, &f, sizeof u);
+  if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x40u); /* NaN stays NaN */
+  u += 0x7fffu + ((u >> 16) & 1u);
+  return (uint16_t)(u >> 16);
+}
+
+int mo_rope_unit(const mo_geom *g, const uint16_t *x, const double *pos, double theta, double *out, uint16_t *out_bits) {
+  if (!g_ok(g) || g->d % 4 || theta <= 0.0) return -1;
+  int d = g->d, D = d / 2;
+  int64_t N = (int64_t)g->nlat * g->nlon;
+#pragma omp parallel for schedule(static)
+  for (int64_t t = 0; t < N; ++t)
+    for (int half = 0; half < 2; ++half)
+      for (int i = 0; i < D / 2; ++i) {
+        double a = pos[t * 2 + half] * pow(theta, -2.0 * i / D);
+        double c = cos(a), s = sin(a);
+        int64_t e = t * d + half * D + 2 * i;
+        double x0 = bf16_widen(x[e]), x1 = bf16_widen(x[e + 1]);
+        double y0 = x0 * c - x1 * s, y1 = x0 * s + x1 * c;
+        if (out) { out[e] = y0; out[e + 1] = y1; }
+        if (out_bits) { out_bits[e] = bf16_round(y0); out_bits[e + 1] = bf16_round(y1); }
+      }
+  return 0;
+}

@@ -392,6 +392,23 @@ def run_ours(args, w):
     t_brb = sum(e[0].elapsed_time(e[1]) for e in ev3b) / k3b
     del ws3b, gates, dgates
 
+    # 2-D rotary position embedding of Q and K (the paper applies it before the operator): an HBM-bound pass
+    pos = torch.rand((w.N, 2), dtype=torch.float32, device=dev)
+    q_r, k_r = torch.empty_like(dx["q"]), torch.empty_like(dx["k"])
+    kr = min(K, 20)
+    evr = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(kr)]
+    for s in range(kr + 2):
+        flush_buf.zero_()
+        if s >= 2:
+            evr[s - 2][0].record(stream)
+        mb.mosaic_bsa_rope(p, dx["q"], dx["k"], pos, q_out=q_r, k_out=k_r)
+        if s >= 2:
+            evr[s - 2][1].record(stream)
+    torch.cuda.synchronize()
+    t_rope = sum(e[0].elapsed_time(e[1]) for e in evr) / kr
+    rope_gbs = 2 * (dx["q"].numel() + dx["k"].numel()) * 2 / (t_rope * 1e-3) / 1e9
+    del pos, q_r, k_r
+
     # end to end: pinned host -> device, step, device -> pinned host
     ke = min(K, 20)
     o_host = torch.empty(o.shape, dtype=torch.int16).pin_memory()
@@ -435,7 +452,7 @@ def run_ours(args, w):
                      "traffic": traffic, "traffic_source": traffic_source, "peak_source": peaks["source"] + " (burst)",
                      "frac_of_nominal_2250": fwd_tflops / NOMINAL_BF16_TFLOPS, "ms": t_fwd},
         "stages": {"select_ms": t_sel, "fwd_ms": t_fwd, "bwd_ms": t_bwd, "ms_layer_fwd": t_step,
-                   "fwd_three_branch_ms": t_br, "bwd_three_branch_ms": t_brb,
+                   "fwd_three_branch_ms": t_br, "bwd_three_branch_ms": t_brb, "rope_ms": t_rope, "rope_gbs": rope_gbs,
                    "fwd_tflops": fwd_tflops, "bwd_tflops": flops.bwd_flops(w) / (t_bwd * 1e-3) / 1e12,
                    "select_pool_gbs_lower_bound": pool_bytes / (t_sel * 1e-3) / 1e9,
                    "pct_of_nominal_peak": 100 * fwd_tflops / NOMINAL_BF16_TFLOPS,

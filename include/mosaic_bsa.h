@@ -180,6 +180,22 @@ int mosaic_bsa_bwd_branches(const mosaic_bsa_params *p, const void *q, const voi
                             void *cuda_stream);
 
 /*
+ * Two-dimensional rotary position embedding of queries and keys ("Overall architecture" paragraph: RoPE encodes
+ * longitude and latitude, the head dimension split equally between the two coordinates, each half a standard
+ * RoPE of its angle in radians; architecture table: theta = 10000).  Channels [0, d/2) turn with the longitude,
+ * [d/2, d) with the latitude; inside a half of width D = d/2 the pair (2i, 2i+1) turns by pos * theta^(-2i/D).
+ * The paper applies it before the attention operator; the other entry points take what this one writes.
+ *   q        in   [B,H,N,d] bf16;  k  in  [B,Hkv,N,d] bf16
+ *   pos      in   [N,2] fp32, (longitude, latitude) of every token in radians (the same for all units)
+ *   theta    in   base of the frequencies (> 0)
+ *   q_out, k_out  out  same shapes as q, k (may be q, k themselves: every element is read once, then written)
+ * No workspace and no status word; errors are the host-side codes only.  The other fields of `p` than B, H, Hkv and
+ * the grid must still describe a valid problem.
+ */
+int mosaic_bsa_rope(const mosaic_bsa_params *p, const void *q, const void *k, const float *pos, float theta,
+                    void *q_out, void *k_out, void *cuda_stream);
+
+/*
  * Selection for callers that cannot allocate device memory.  (The paper has no counterpart of this
  * entry point: it computes exactly what mosaic_bsa_select computes, with the same arguments minus the
  * workspace.)

@@ -20,7 +20,7 @@ _lib = None
 OP_SELECT, OP_FWD, OP_BWD, OP_FWD_BRANCHES, OP_BWD_BRANCHES = 0, 1, 2, 3, 4
 EXPORTS = ("mosaic_bsa_workspace_bytes", "mosaic_bsa_select", "mosaic_bsa_fwd", "mosaic_bsa_bwd",
            "mosaic_bsa_last_status", "mosaic_bsa_strerror", "mosaic_bsa_select_static",
-           "mosaic_bsa_descriptor_encodes", "mosaic_bsa_fwd_branches", "mosaic_bsa_bwd_branches")
+           "mosaic_bsa_descriptor_encodes", "mosaic_bsa_fwd_branches", "mosaic_bsa_bwd_branches", "mosaic_bsa_rope")
 STATIC_SCRATCH_BYTES = 4 << 20
 FLAG_LOCAL_GROUPS = 1
 
@@ -97,6 +97,8 @@ def lib():
         L.mosaic_bsa_fwd_branches.argtypes = [pp, vp, vp, vp, i32p, fp, vp, fp, fp, vp, ctypes.c_size_t, vp]
         L.mosaic_bsa_bwd_branches.restype = ctypes.c_int
         L.mosaic_bsa_bwd_branches.argtypes = [pp, vp, vp, vp, i32p, fp, vp, vp, vp, vp, fp, vp, ctypes.c_size_t, vp]
+        L.mosaic_bsa_rope.restype = ctypes.c_int
+        L.mosaic_bsa_rope.argtypes = [pp, vp, vp, fp, ctypes.c_float, vp, vp, vp]
         L.mosaic_bsa_bwd.restype = ctypes.c_int
         L.mosaic_bsa_bwd.argtypes = [pp, vp, vp, vp, vp, fp, vp, i32p, vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.mosaic_bsa_last_status.restype = ctypes.c_int
@@ -242,6 +244,23 @@ def mosaic_bsa_bwd_branches(p: Params, q, k, v, block_idx, gates, d_o, dq=None, 
     if rc:
         raise MosaicError(rc, "mosaic_bsa_bwd_branches")
     return dq, dk, dv, dgates
+
+
+def mosaic_bsa_rope(p: Params, q, k, pos, theta=10000.0, q_out=None, k_out=None, stream=None):
+    """2-D rotary position embedding of q and k; pos is [N, 2] fp32 (longitude, latitude in radians).
+    Returns (q_out, k_out)."""
+    _chk_qkv(p, q)
+    _chk_qkv(p, k, heads=p.kv_heads)
+    if pos.dtype != torch.float32 or not pos.is_cuda or not pos.is_contiguous() or tuple(pos.shape) != (p.N, 2):
+        raise ValueError(f"expected contiguous cuda fp32 positions [{p.N},2]")
+    q_out = torch.empty_like(q) if q_out is None else q_out
+    k_out = torch.empty_like(k) if k_out is None else k_out
+    pc = p.c()
+    rc = lib().mosaic_bsa_rope(ctypes.byref(pc), _ptr(q), _ptr(k), _ptr(pos), float(theta), _ptr(q_out), _ptr(k_out),
+                               _stream(stream))
+    if rc:
+        raise MosaicError(rc, "mosaic_bsa_rope")
+    return q_out, k_out
 
 
 def mosaic_bsa_last_status(ws, stream=None) -> int:

@@ -313,6 +313,20 @@ int mosaic_bsa_bwd_branches(const mosaic_bsa_params* p, const void* q, const voi
   return launch_grad_sum(c, g.Ukv, base + w.dv_l, sel ? base + w.dv_fg : nullptr, F(w.dvm), dv);
 }
 
+int mosaic_bsa_rope(const mosaic_bsa_params* p, const void* q, const void* k, const float* pos, float theta, void* q_out,
+                    void* k_out, void* cuda_stream) {
+  HostCtx c;
+  int rc = validate(p, &c.g);
+  if (rc) return rc;
+  if (!q || !k || !pos || !q_out || !k_out || !(theta > 0.f)) return MOSAIC_E_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(k, 16) || !aligned(q_out, 16) || !aligned(k_out, 16) || !aligned(pos, 4))
+    return MOSAIC_E_MISALIGNED;
+  if ((rc = device_ok())) return rc;
+  c.stream = (cudaStream_t)cuda_stream;
+  c.status = nullptr;
+  return launch_rope(c, q, k, pos, (double)theta, q_out, k_out);
+}
+
 int mosaic_bsa_last_status(const void* ws, void* cuda_stream) {
   if (!ws) return MOSAIC_E_INVALID_ARG;
   if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess) return MOSAIC_E_CUDA;

@@ -121,6 +121,7 @@ int launch_gate(const HostCtx& c, const void* d_o, const void* o_fg, const void*
                 const float* gates, float* dgates, void* do_fg, void* do_l, float* dob);
 int launch_compress_bwd(const HostCtx& c, const float* pq, const float* pk, const float* pv, const float* dob,
                         const float* ocg, const float* lse2, float* delta, float* dqm, float* dkm, float* dvm);
+int launch_rope(const HostCtx& c, const void* q, const void* k, const float* pos, double theta, void* q_out, void* k_out);
 int launch_grad_sum(const HostCtx& c, int units, const void* x_l, const void* x_fg, const float* xm, void* out);
 int launch_combine(const HostCtx& c, const float* ocg, const void* o_fg, const void* o_l, const float* gates, void* o);
 int launch_dq_tc(const HostCtx& c, const void* q, const void* k, const void* v, const void* d_o, const float* lse,

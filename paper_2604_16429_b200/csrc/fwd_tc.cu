@@ -99,21 +99,9 @@ __global__ void __launch_bounds__(kThreads, 1)
       mbar_init(s32(&sm.list_empty[i]), 11);  // 8 softmax warps + 2 MMA warps + TMA producer
     }
     sm.abort = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    cta_publish_barriers();
   }
-  __syncthreads();
-  if (warp == 9) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(&sm.tmem_base)),
-                 "r"(kTmemCols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-
-  const uint32_t tmem = sm.tmem_base;
+  const uint32_t tmem = cta_tmem_alloc(warp == 9, &sm.tmem_base, kTmemCols);
   volatile int* abort = &sm.abort;
 
   if (warp == 11) {
@@ -448,13 +436,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       n = n_next;
     }
   }
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 9) {
-    tc_fence_after();
-    __syncwarp();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
-  }
+  cta_tmem_free(warp == 9, tmem, kTmemCols);
 }
 
 // ---------------------------------------------------------------------------------------------

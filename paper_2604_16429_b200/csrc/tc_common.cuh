@@ -133,6 +133,34 @@ __device__ __forceinline__ void mma_drain(uint32_t bar) {
   tc_commit(bar);
   mbar_drain(bar, 0);
 }
+// CTA prologue and epilogue that the tensor-core kernels share.  After the barriers are initialised (by one thread,
+// followed by `cta_publish_barriers`), `alloc_warp` takes the whole of the SM's tensor memory and every thread
+// reads its base address; at the end the same warp gives it back once every role has left its loop.
+__device__ __forceinline__ void cta_publish_barriers() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cta_tmem_alloc(bool alloc_warp, uint32_t* slot, uint32_t cols) {
+  __syncthreads();  // barrier initialisation is visible to every thread
+  if (alloc_warp) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(slot)), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  return *slot;
+}
+__device__ __forceinline__ void cta_tmem_free(bool alloc_warp, uint32_t tmem, uint32_t cols) {
+  tc_fence_before();
+  __syncthreads();
+  if (alloc_warp) {
+    tc_fence_after();
+    __syncwarp();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(cols) : "memory");
+  }
+}
+
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 

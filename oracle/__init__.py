@@ -39,6 +39,7 @@ class _Geom(ctypes.Structure):
         ("topk", ctypes.c_int32),
         ("scale", ctypes.c_double),
         ("local_groups", ctypes.c_int32),
+        ("f16", ctypes.c_int32),
     ]
 
 
@@ -54,6 +55,7 @@ class Geom:
     topk: int = 0
     scale: float = 0.0
     local_groups: bool = False
+    f16: bool = False          # the 16-bit inputs are IEEE binary16 instead of bf16
 
     @property
     def N(self): return self.nlat * self.nlon
@@ -68,7 +70,7 @@ class Geom:
 
     def c(self):
         return _Geom(self.nlat, self.nlon, self.d, self.bh, self.bw, self.rlat, self.rlon,
-                     self.topk, float(self.scale), int(self.local_groups))
+                     self.topk, float(self.scale), int(self.local_groups), int(self.f16))
 
 
 def _load():
@@ -240,6 +242,16 @@ def rope(g: Geom, x, pos, theta=10000.0):
                               _p(out, ctypes.c_double), _p(bits, ctypes.c_uint16))
     assert rc == 0
     return out, bits
+
+
+def widen16(g: Geom, bits) -> np.ndarray:
+    """The 16-bit storage type's values as fp64 (bf16, or binary16 when g.f16)."""
+    bits = np.ascontiguousarray(bits, np.uint16)
+    out = np.zeros(bits.shape)
+    gc = g.c()
+    rc = _load().mo_widen16(ctypes.byref(gc), _p(bits, ctypes.c_uint16), ctypes.c_int64(bits.size), _p(out, ctypes.c_double))
+    assert rc == 0
+    return out
 
 
 def block_tokens(g: Geom, j: int) -> np.ndarray:

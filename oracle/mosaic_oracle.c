@@ -10,7 +10,7 @@
  * every equation of the method is per head and per sample):
  *   grid nlat x nlon, token t = lat*nlon + lon, head dim d;
  *   block (by,bx) holds tokens (by*bh + r, bx*bw + c), r < bh, c < bw; id j = by*nbw + bx;
- *   inputs are bf16 bit patterns (uint16), widened exactly to double.
+ *   inputs are bf16 bit patterns (uint16), or IEEE binary16 when the geometry says so, widened exactly to double.
  *
  * Steps and where the paper defines them:
  *   pooling      -- "Compression" paragraph of the Block-Sparse Attention section
@@ -58,6 +58,8 @@ typedef struct mo_geom {
   int32_t local_groups; /* 0: local set = sliding neighbourhood of radius (rlat, rlon);
                            1: local set = the aligned group of rlat x rlon blocks that holds the block
                               (the paper's "Local Attention": dense attention inside large blocks) */
+  int32_t f16;          /* 0: the 16-bit inputs are bf16 bit patterns; 1: IEEE binary16 (the paper trains in fp16,
+                           "Training details" paragraph) */
 } mo_geom;
 
 #define MO_MAX_LOCAL 256
@@ -83,6 +85,17 @@ static double bf16_widen(uint16_t h) {
   memcpy(&f, &u, sizeof f);
   return (double)f;
 }
+/* IEEE binary16: 1 sign, 5 exponent (bias 15), 10 fraction bits; exact in double */
+static double f16_widen(uint16_t h) {
+  int sign = h >> 15, ex = (h >> 10) & 31, fr = h & 1023;
+  double v;
+  if (ex == 0) v = ldexp((double)fr, -24);                 /* zero and subnormals */
+  else if (ex == 31) v = fr ? NAN : INFINITY;
+  else v = ldexp((double)(1024 + fr), ex - 25);
+  return sign ? -v : v;
+}
+/* a 16-bit input element in the problem's storage type */
+static double w16(const mo_geom *g, uint16_t h) { return g->f16 ? f16_widen(h) : bf16_widen(h); }
 
 /* token index of element e (row-major inside the block) of block j */
 static int64_t block_token(const mo_geom *g, int j, int e) {
@@ -138,7 +151,7 @@ int mo_pool_unit(const mo_geom *g, const uint16_t *x, float *pooled /* [m,d] */)
   for (int j = 0; j < m; ++j) {
     for (int c = 0; c < d; ++c) {
       double acc = 0.0;
-      for (int e = 0; e < b; ++e) acc += bf16_widen(x[block_token(g, j, e) * d + c]);
+      for (int e = 0; e < b; ++e) acc += w16(g, x[block_token(g, j, e) * d + c]);
       pooled[(size_t)j * d + c] = (float)acc;
     }
   }
@@ -221,7 +234,7 @@ static void row_logits(const mo_geom *g, const uint16_t *q, const uint16_t *k, i
     for (int e = 0; e < b; ++e) {
       int64_t t = block_token(g, att[a], e);
       double s = 0.0;
-      for (int c = 0; c < d; ++c) s += bf16_widen(q[l * d + c]) * bf16_widen(k[t * d + c]);
+      for (int c = 0; c < d; ++c) s += w16(g, q[l * d + c]) * w16(g, k[t * d + c]);
       x[(size_t)a * b + e] = sc * s;
     }
 }
@@ -276,7 +289,7 @@ int mo_fwd_unit(const mo_geom *g, const uint16_t *q, const uint16_t *k, const ui
           for (int e2 = 0; e2 < b; ++e2) {
             double w = exp(x[(size_t)a * b + e2] - M) / Z;
             int64_t t = block_token(g, att[a], e2);
-            for (int c = 0; c < d; ++c) o[c] += w * bf16_widen(v[t * d + c]);
+            for (int c = 0; c < d; ++c) o[c] += w * w16(g, v[t * d + c]);
           }
         LSE[(size_t)n * b + e] = M + log(Z);
       }
@@ -313,7 +326,7 @@ int mo_bwd_unit(const mo_geom *g, const uint16_t *q, const uint16_t *k, const ui
       double acc = 0.0;
       for (int c = 0; c < d; ++c) {
         double o = Ob[((size_t)i * b + e) * d + c];
-        acc += bf16_widen(d_o[l * d + c]) * o;
+        acc += w16(g, d_o[l * d + c]) * o;
         if (O_out) O_out[l * d + c] = o;
       }
       D[l] = acc;
@@ -338,9 +351,9 @@ int mo_bwd_unit(const mo_geom *g, const uint16_t *q, const uint16_t *k, const ui
             int64_t t = block_token(g, att[a], e2);
             double w = exp(x[(size_t)a * b + e2] - LSE[l]);
             double dP = 0.0;
-            for (int c = 0; c < d; ++c) dP += bf16_widen(d_o[l * d + c]) * bf16_widen(v[t * d + c]);
+            for (int c = 0; c < d; ++c) dP += w16(g, d_o[l * d + c]) * w16(g, v[t * d + c]);
             double dS = w * (dP - D[l]);
-            for (int c = 0; c < d; ++c) dq[c] += sc * dS * bf16_widen(k[t * d + c]);
+            for (int c = 0; c < d; ++c) dq[c] += sc * dS * w16(g, k[t * d + c]);
           }
       }
     }
@@ -367,14 +380,14 @@ int mo_bwd_unit(const mo_geom *g, const uint16_t *q, const uint16_t *k, const ui
             int64_t t = block_token(g, j, e2);
             double s = 0.0, dP = 0.0;
             for (int c = 0; c < d; ++c) {
-              s += bf16_widen(q[l * d + c]) * bf16_widen(k[t * d + c]);
-              dP += bf16_widen(d_o[l * d + c]) * bf16_widen(v[t * d + c]);
+              s += w16(g, q[l * d + c]) * w16(g, k[t * d + c]);
+              dP += w16(g, d_o[l * d + c]) * w16(g, v[t * d + c]);
             }
             double w = exp(sc * s - LSE[l]);
             double dS = w * (dP - D[l]);
             for (int c = 0; c < d; ++c) {
-              dV[t * d + c] += w * bf16_widen(d_o[l * d + c]);
-              dK[t * d + c] += sc * dS * bf16_widen(q[l * d + c]);
+              dV[t * d + c] += w * w16(g, d_o[l * d + c]);
+              dK[t * d + c] += sc * dS * w16(g, q[l * d + c]);
             }
           }
         }
@@ -432,7 +445,7 @@ int mo_bwd_blocks(const mo_geom *g, const uint16_t *q, const uint16_t *k, const 
     for (int e = 0; e < b; ++e) {
       int64_t l = block_token(g, list[n], e);
       double acc = 0.0;
-      for (int c = 0; c < d; ++c) acc += bf16_widen(d_o[l * d + c]) * Ob[((size_t)n * b + e) * d + c];
+      for (int c = 0; c < d; ++c) acc += w16(g, d_o[l * d + c]) * Ob[((size_t)n * b + e) * d + c];
       D[l] = acc;
       LSE[l] = Lb[(size_t)n * b + e];
     }
@@ -455,9 +468,9 @@ int mo_bwd_blocks(const mo_geom *g, const uint16_t *q, const uint16_t *k, const 
             int64_t t = block_token(g, att[a], e2);
             double w = exp(x[(size_t)a * b + e2] - LSE[l]);
             double dP = 0.0;
-            for (int c = 0; c < d; ++c) dP += bf16_widen(d_o[l * d + c]) * bf16_widen(v[t * d + c]);
+            for (int c = 0; c < d; ++c) dP += w16(g, d_o[l * d + c]) * w16(g, v[t * d + c]);
             double dS = w * (dP - D[l]);
-            for (int c = 0; c < d; ++c) dq[c] += sc * dS * bf16_widen(k[t * d + c]);
+            for (int c = 0; c < d; ++c) dq[c] += sc * dS * w16(g, k[t * d + c]);
           }
       }
     }
@@ -487,14 +500,14 @@ int mo_bwd_blocks(const mo_geom *g, const uint16_t *q, const uint16_t *k, const 
           int64_t l = block_token(g, conn[ci], e);
           double s = 0.0, dP = 0.0;
           for (int c = 0; c < d; ++c) {
-            s += bf16_widen(q[l * d + c]) * bf16_widen(k[t * d + c]);
-            dP += bf16_widen(d_o[l * d + c]) * bf16_widen(v[t * d + c]);
+            s += w16(g, q[l * d + c]) * w16(g, k[t * d + c]);
+            dP += w16(g, d_o[l * d + c]) * w16(g, v[t * d + c]);
           }
           double w = exp(sc * s - LSE[l]);
           double dS = w * (dP - D[l]);
           for (int c = 0; c < d; ++c) {
-            dv[c] += w * bf16_widen(d_o[l * d + c]);
-            dk[c] += sc * dS * bf16_widen(q[l * d + c]);
+            dv[c] += w * w16(g, d_o[l * d + c]);
+            dk[c] += sc * dS * w16(g, q[l * d + c]);
           }
         }
     }
@@ -532,7 +545,7 @@ static double branch_row(const mo_geom *g, const uint16_t *q, const uint16_t *k,
     for (int e2 = 0; e2 < b; ++e2) {
       double w = exp(x[(size_t)a * b + e2] - M) / Z;
       int64_t t = block_token(g, blk[a], e2);
-      for (int c = 0; c < d; ++c) o[c] += w * bf16_widen(v[t * d + c]);
+      for (int c = 0; c < d; ++c) o[c] += w * w16(g, v[t * d + c]);
     }
   return M + log(Z);
 }
@@ -656,7 +669,7 @@ int mo_bwd3_unit(const mo_geom *g, const uint16_t *q, const uint16_t *k, const u
       int64_t l = block_token(g, i, e);
       double gc = 0.0, gf = 0.0, gl = 0.0;
       for (int c = 0; c < d; ++c) {
-        double go = bf16_widen(d_o[l * d + c]);
+        double go = w16(g, d_o[l * d + c]);
         gc += go * OCG[l * d + c];
         gf += go * OFG[l * d + c];
         gl += go * OL[l * d + c];
@@ -705,15 +718,15 @@ int mo_bwd3_unit(const mo_geom *g, const uint16_t *q, const uint16_t *k, const u
         for (int e = 0; e < b; ++e) {
           int64_t l = block_token(g, i, e);
           double gate = gates[l * 3 + br], D = 0.0;
-          for (int c = 0; c < d; ++c) D += gate * bf16_widen(d_o[l * d + c]) * OB[l * d + c];
+          for (int c = 0; c < d; ++c) D += gate * w16(g, d_o[l * d + c]) * OB[l * d + c];
           row_logits(g, q, k, l, blk, nb, x);
           for (int a = 0; a < nb; ++a)
             for (int e2 = 0; e2 < b; ++e2) {
               int64_t t = block_token(g, blk[a], e2);
               double w = exp(x[(size_t)a * b + e2] - LSE[l]), dP = 0.0;
-              for (int c = 0; c < d; ++c) dP += gate * bf16_widen(d_o[l * d + c]) * bf16_widen(v[t * d + c]);
+              for (int c = 0; c < d; ++c) dP += gate * w16(g, d_o[l * d + c]) * w16(g, v[t * d + c]);
               double dS = w * (dP - D);
-              for (int c = 0; c < d; ++c) dQ[l * d + c] += sc * dS * bf16_widen(k[t * d + c]);
+              for (int c = 0; c < d; ++c) dQ[l * d + c] += sc * dS * w16(g, k[t * d + c]);
             }
         }
       }
@@ -735,18 +748,18 @@ int mo_bwd3_unit(const mo_geom *g, const uint16_t *q, const uint16_t *k, const u
           for (int e = 0; e < b; ++e) {
             int64_t l = block_token(g, i, e);
             double gate = gates[l * 3 + br], D = 0.0;
-            for (int c = 0; c < d; ++c) D += gate * bf16_widen(d_o[l * d + c]) * OB[l * d + c];
+            for (int c = 0; c < d; ++c) D += gate * w16(g, d_o[l * d + c]) * OB[l * d + c];
             for (int e2 = 0; e2 < b; ++e2) {
               int64_t t = block_token(g, j, e2);
               double s = 0.0, dP = 0.0;
               for (int c = 0; c < d; ++c) {
-                s += bf16_widen(q[l * d + c]) * bf16_widen(k[t * d + c]);
-                dP += gate * bf16_widen(d_o[l * d + c]) * bf16_widen(v[t * d + c]);
+                s += w16(g, q[l * d + c]) * w16(g, k[t * d + c]);
+                dP += gate * w16(g, d_o[l * d + c]) * w16(g, v[t * d + c]);
               }
               double w = exp(sc * s - LSE[l]), dS = w * (dP - D);
               for (int c = 0; c < d; ++c) {
-                dV[t * d + c] += w * gate * bf16_widen(d_o[l * d + c]);
-                dK[t * d + c] += sc * dS * bf16_widen(q[l * d + c]);
+                dV[t * d + c] += w * gate * w16(g, d_o[l * d + c]);
+                dK[t * d + c] += sc * dS * w16(g, q[l * d + c]);
               }
             }
           }
@@ -778,6 +791,25 @@ static uint16_t bf16_round(double x) {
   return (uint16_t)(u >> 16);
 }
 
+/* double -> float -> binary16, both steps to nearest even */
+static uint16_t f16_round(double x) {
+  float f = (float)x;
+  uint32_t u;
+  memcpy(&u, &f, sizeof u);
+  uint16_t sign = (uint16_t)((u >> 16) & 0x8000u);
+  uint32_t a = u & 0x7fffffffu;
+  if (a > 0x7f800000u) return (uint16_t)(sign | 0x7e00u);                 /* NaN */
+  if (a >= 0x47800000u) return (uint16_t)(sign | 0x7c00u);                /* >= 65536 (or inf): inf; [65520, 65536) rounds below */
+  if (a < 0x33000000u) return sign;                                       /* below half the smallest subnormal (2^-25): zero */
+  int e = (int)(a >> 23) - 127;                                           /* unbiased exponent of the float */
+  uint32_t man = (a & 0x7fffffu) | 0x800000u;                             /* 24-bit significand */
+  int shift = e >= -14 ? 13 : 13 + (-14 - e);                             /* bits dropped (more for subnormal results) */
+  uint32_t kept = man >> shift, rem = man & ((1u << shift) - 1u), half = 1u << (shift - 1);
+  if (rem > half || (rem == half && (kept & 1u))) ++kept;
+  uint32_t out = e >= -14 ? (((uint32_t)(e + 15) << 10) + (kept - 0x400u)) : kept;   /* a carry moves into the exponent */
+  return (uint16_t)(sign | out);
+}
+
 int mo_rope_unit(const mo_geom *g, const uint16_t *x, const double *pos, double theta, double *out, uint16_t *out_bits) {
   if (!g_ok(g) || g->d % 4 || theta <= 0.0) return -1;
   int d = g->d, D = d / 2;
@@ -789,10 +821,20 @@ int mo_rope_unit(const mo_geom *g, const uint16_t *x, const double *pos, double 
         double a = pos[t * 2 + half] * pow(theta, -2.0 * i / D);
         double c = cos(a), s = sin(a);
         int64_t e = t * d + half * D + 2 * i;
-        double x0 = bf16_widen(x[e]), x1 = bf16_widen(x[e + 1]);
+        double x0 = w16(g, x[e]), x1 = w16(g, x[e + 1]);
         double y0 = x0 * c - x1 * s, y1 = x0 * s + x1 * c;
         if (out) { out[e] = y0; out[e + 1] = y1; }
-        if (out_bits) { out_bits[e] = bf16_round(y0); out_bits[e + 1] = bf16_round(y1); }
+        if (out_bits) {
+          out_bits[e] = g->f16 ? f16_round(y0) : bf16_round(y0);
+          out_bits[e + 1] = g->f16 ? f16_round(y1) : bf16_round(y1);
+        }
       }
+  return 0;
+}
+
+/* The storage type's decoding on its own (for the tests that pin it against a library's conversion). */
+int mo_widen16(const mo_geom *g, const uint16_t *x, int64_t n, double *out) {
+  if (!g) return -1;
+  for (int64_t i = 0; i < n; ++i) out[i] = w16(g, x[i]);
   return 0;
 }

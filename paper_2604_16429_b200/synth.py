@@ -45,6 +45,7 @@ class Workload:
     rlon: int = 1
     local_groups: bool = False   # local set = aligned group of rlat x rlon blocks (the paper's large local blocks)
     Hkv: int = 0                 # heads of K and V (grouped-query attention); 0 = H
+    f16: bool = False            # 16-bit tensors are IEEE binary16 instead of bf16 (the same values, rounded to that type)
 
     @property
     def N(self): return self.nlat * self.nlon
@@ -86,6 +87,15 @@ def bf16_bits_to_f32(h: np.ndarray) -> np.ndarray:
     return (h.astype(np.uint32) << np.uint32(16)).view(np.float32)
 
 
+def to_f16_bits(x: np.ndarray) -> np.ndarray:
+    """float32 -> IEEE binary16 bit patterns, round to nearest even."""
+    return np.ascontiguousarray(x, np.float32).astype(np.float16).view(np.uint16)
+
+
+def f16_bits_to_f32(h: np.ndarray) -> np.ndarray:
+    return np.ascontiguousarray(h, np.uint16).view(np.float16).astype(np.float32)
+
+
 def iid_normal(B, H, N, d, seed) -> np.ndarray:
     rng = np.random.Generator(np.random.PCG64(seed))
     return to_bf16_bits(rng.standard_normal((B, H, N, d), dtype=np.float32))
@@ -122,11 +132,14 @@ def make_inputs(w: Workload, with_do: bool | None = None) -> dict:
     out = {"q": gen(base + 0), "k": gen(base + 1, w.kv_heads), "v": gen(base + 2, w.kv_heads)}   # K, V: [B, Hkv, N, d]
     if w.backward if with_do is None else with_do:
         out["do"] = iid_normal(w.B, w.H, w.N, w.d, base + 3)
+    if w.f16:   # the same draws, stored as binary16 (a bf16 value of this range is exact in binary16 bar underflow)
+        out = {k: to_f16_bits(bf16_bits_to_f32(v)) for k, v in out.items()}
     return out
 
 
 def small_case(nlat, nlon, bh, bw, topk, B=1, H=1, d=64, kind="iid", seed=7, rlat=1, rlon=1, backward=False,
-               local_groups=False, Hkv=0):
+               local_groups=False, Hkv=0, f16=False):
     """A free-form small workload for tests (cfg number = seed)."""
-    return Workload(f"small_{nlat}x{nlon}_{bh}x{bw}_k{topk}" + ("_groups" if local_groups else "") + (f"_kv{Hkv}" if Hkv else ""),
-                    seed, B, H, nlat, nlon, bh, bw, topk, kind, backward, d, rlat, rlon, local_groups, Hkv)
+    return Workload(f"small_{nlat}x{nlon}_{bh}x{bw}_k{topk}" + ("_groups" if local_groups else "") + (f"_kv{Hkv}" if Hkv else "")
+                    + ("_f16" if f16 else ""),
+                    seed, B, H, nlat, nlon, bh, bw, topk, kind, backward, d, rlat, rlon, local_groups, Hkv, f16)

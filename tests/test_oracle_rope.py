@@ -63,3 +63,25 @@ def test_inner_products_depend_on_the_position_difference_only():
     rd, _ = oracle.rope(g, q, pa - pb)
     kf = synth.bf16_bits_to_f32(k).astype(np.float64)
     assert np.abs((rq * rk).sum(1) - (rd * kf).sum(1)).max() < 1e-11
+
+
+def test_binary16_storage_decoding_and_rounding_against_numpy():
+    """Every binary16 bit pattern decodes as numpy's float16 does, the identity rotation returns the same bits, and
+    rotated values round as numpy rounds float32 -> float16."""
+    g16 = Geom(8, 16, d=64, bh=8, bw=8, topk=0, f16=True)
+    allbits = np.arange(65536, dtype=np.uint16)
+    want = allbits.view(np.float16).astype(np.float64)
+    got = oracle.widen16(g16, allbits)
+    assert np.array_equal(np.isnan(got), np.isnan(want)) and np.array_equal(got[~np.isnan(want)], want[~np.isnan(want)])
+    some = allbits[:0x7F80:7]                                             # finite bf16 patterns
+    assert np.array_equal(oracle.widen16(Geom(8, 16), some), synth.bf16_bits_to_f32(some).astype(np.float64))
+    finite = allbits[np.isfinite(want)]
+    x = np.resize(finite, (g16.N, g16.d)).astype(np.uint16)
+    _, same = oracle.rope(g16, x, np.zeros((g16.N, 2)))
+    assert np.array_equal(same & 0x7FFF, x & 0x7FFF) and np.array_equal(same[(x & 0x7FFF) != 0], x[(x & 0x7FFF) != 0])
+    rng = np.random.default_rng(5)
+    xs = synth.to_f16_bits((rng.standard_normal((g16.N, g16.d)) * 10.0 ** rng.integers(-7, 5, (g16.N, 1))).astype(np.float32))
+    pos = rng.uniform(-3, 3, (g16.N, 2))
+    out, bits = oracle.rope(g16, xs, pos)
+    with np.errstate(over="ignore"):
+        assert np.array_equal(bits, out.astype(np.float32).astype(np.float16).view(np.uint16))

@@ -60,7 +60,7 @@ typedef struct mosaic_bsa_params {
                          MOSAIC_FLAG_LOCAL_GROUPS: height and width of the local group    */
   int32_t topk;       /* selected non-local blocks per query block, >= 0               */
   float scale;        /* softmax scale; <= 0 means 1/sqrt(d)                           */
-  uint32_t flags;     /* 0 or MOSAIC_FLAG_LOCAL_GROUPS                                 */
+  uint32_t flags;     /* 0 or a sum of MOSAIC_FLAG_LOCAL_GROUPS, MOSAIC_FLAG_FP16      */
   int32_t Hkv;        /* heads of K and V (grouped-query attention, the paper's GQA ratio
                          H / Hkv); 0 means H; H % Hkv == 0                                */
 } mosaic_bsa_params;
@@ -71,6 +71,11 @@ typedef struct mosaic_bsa_params {
  * of a row or column may be ragged).  The paper's HEALPix layout -- 128 contiguous tokens per block, local
  * blocks of 1024 tokens -- is nlat = N/16, nlon = 16, bh = 8, bw = 16, rlat = 8, rlon = 1 with this flag. */
 #define MOSAIC_FLAG_LOCAL_GROUPS 1u
+/* The 16-bit tensors (q, k, v, o, d_o, dq, dk, dv and the rotated q, k) are IEEE binary16 instead of bf16
+ * wherever a comment says "bf16" (appendix, "Distributed training" paragraph: the paper trains entirely in
+ * float16).  Arithmetic is unchanged: tensor-core products of 16-bit operands with fp32 accumulation, fp32
+ * softmax, selection on the exactly widened values. */
+#define MOSAIC_FLAG_FP16 2u
 
 enum { MOSAIC_OP_SELECT = 0, MOSAIC_OP_FWD = 1, MOSAIC_OP_BWD = 2, MOSAIC_OP_FWD_BRANCHES = 3,
        MOSAIC_OP_BWD_BRANCHES = 4 };

@@ -59,7 +59,7 @@ typedef struct mo_geom {
                            1: local set = the aligned group of rlat x rlon blocks that holds the block
                               (the paper's "Local Attention": dense attention inside large blocks) */
   int32_t f16;          /* 0: the 16-bit inputs are bf16 bit patterns; 1: IEEE binary16 (the paper trains in fp16,
-                           "Training details" paragraph) */
+                           appendix, "Distributed training" paragraph) */
 } mo_geom;
 
 #define MO_MAX_LOCAL 256

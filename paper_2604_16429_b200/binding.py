@@ -23,6 +23,7 @@ EXPORTS = ("mosaic_bsa_workspace_bytes", "mosaic_bsa_select", "mosaic_bsa_fwd", 
            "mosaic_bsa_descriptor_encodes", "mosaic_bsa_fwd_branches", "mosaic_bsa_bwd_branches", "mosaic_bsa_rope")
 STATIC_SCRATCH_BYTES = 4 << 20
 FLAG_LOCAL_GROUPS = 1
+FLAG_FP16 = 2
 
 
 class MosaicError(RuntimeError):
@@ -70,7 +71,8 @@ class Params:
     @staticmethod
     def from_workload(w, **over):
         kw = dict(B=w.B, H=w.H, nlat=w.nlat, nlon=w.nlon, d=w.d, bh=w.bh, bw=w.bw, rlat=w.rlat, rlon=w.rlon,
-                  topk=w.topk, flags=FLAG_LOCAL_GROUPS if getattr(w, "local_groups", False) else 0,
+                  topk=w.topk, flags=(FLAG_LOCAL_GROUPS if getattr(w, "local_groups", False) else 0)
+                  | (FLAG_FP16 if getattr(w, "f16", False) else 0),
                   Hkv=getattr(w, "Hkv", 0))
         kw.update(over)
         return Params(**kw)
@@ -131,9 +133,10 @@ def _ptr(t) -> int:
 
 def _chk_qkv(p: Params, *ts, heads=None):
     h = p.H if heads is None else heads
+    dt = torch.float16 if p.flags & FLAG_FP16 else torch.bfloat16
     for t in ts:
-        if t.dtype != torch.bfloat16 or not t.is_cuda or not t.is_contiguous() or tuple(t.shape) != (p.B, h, p.N, p.d):
-            raise ValueError(f"expected contiguous cuda bf16 [{p.B},{h},{p.N},{p.d}], got {t.dtype} {tuple(t.shape)}")
+        if t.dtype != dt or not t.is_cuda or not t.is_contiguous() or tuple(t.shape) != (p.B, h, p.N, p.d):
+            raise ValueError(f"expected contiguous cuda {dt} [{p.B},{h},{p.N},{p.d}], got {t.dtype} {tuple(t.shape)}")
 
 
 def alloc_workspace(p: Params, op: int, device="cuda") -> torch.Tensor:
@@ -277,11 +280,11 @@ def check_status(ws, where: str, stream=None):
         raise MosaicError(st, where + " (device status)")
 
 
-def from_bits(bits, device="cuda") -> torch.Tensor:
-    """uint16 bf16 bit patterns (numpy) -> bf16 tensor on `device`, bit for bit."""
+def from_bits(bits, device="cuda", f16=False) -> torch.Tensor:
+    """uint16 bit patterns (numpy) -> bf16 (or, with f16, float16) tensor on `device`, bit for bit."""
     import numpy as np
     t = torch.from_numpy(np.ascontiguousarray(bits).view(np.int16))
-    return t.to(device).view(torch.bfloat16)
+    return t.to(device).view(torch.float16 if f16 else torch.bfloat16)
 
 
 def default_scale(d: int) -> float:

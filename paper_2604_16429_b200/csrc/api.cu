@@ -12,7 +12,7 @@ size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 int validate(const mosaic_bsa_params* p, Geo* g) {
   if (!p) return MOSAIC_E_INVALID_ARG;
   if (p->B <= 0 || p->H <= 0 || p->nlat <= 0 || p->nlon <= 0 || p->bh <= 0 || p->bw <= 0 || p->topk < 0 ||
-      p->rlat < 0 || p->rlon < 0 || (p->flags & ~MOSAIC_FLAG_LOCAL_GROUPS) != 0)
+      p->rlat < 0 || p->rlon < 0 || (p->flags & ~(MOSAIC_FLAG_LOCAL_GROUPS | MOSAIC_FLAG_FP16)) != 0)
     return MOSAIC_E_INVALID_ARG;
   if (p->nlat % p->bh || p->nlon % p->bw) return MOSAIC_E_INVALID_ARG;
   if (!(p->scale == p->scale) || isinf(p->scale)) return MOSAIC_E_INVALID_ARG;
@@ -41,6 +41,7 @@ int validate(const mosaic_bsa_params* p, Geo* g) {
   g->rlat = p->rlat; g->rlon = p->rlon; g->topk = p->topk;
   g->local_off = 0;
   g->local_groups = groups ? 1 : 0;
+  g->f16 = (p->flags & MOSAIC_FLAG_FP16) ? 1 : 0;
   g->scale = p->scale > 0.f ? p->scale : 1.0f / sqrtf((float)p->d);
   g->scale_log2 = g->scale * 1.4426950408889634f;
   g->N = N;

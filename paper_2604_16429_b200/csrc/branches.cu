@@ -155,10 +155,10 @@ __global__ void __launch_bounds__(256) combine_kernel(Geo g, const float* __rest
   uint32_t r[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    const float lo = gc * cgv[2 * i] + gf * __uint_as_float(av[i] << 16) + gl * __uint_as_float(bv[i] << 16);
-    const float hi = gc * cgv[2 * i + 1] + gf * __uint_as_float(av[i] & 0xffff0000u) + gl * __uint_as_float(bv[i] & 0xffff0000u);
-    const __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
-    r[i] = *reinterpret_cast<const uint32_t*>(&p);
+    float a0, a1, b0, b1;
+    unpack16x2(av[i], g.f16 != 0, a0, a1);
+    unpack16x2(bv[i], g.f16 != 0, b0, b1);
+    r[i] = pack16x2(gc * cgv[2 * i] + gf * a0 + gl * b0, gc * cgv[2 * i + 1] + gf * a1 + gl * b1, g.f16 != 0);
   }
   o[x * 8 + part] = make_uint4(r[0], r[1], r[2], r[3]);
 }

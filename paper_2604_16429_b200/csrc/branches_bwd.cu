@@ -24,21 +24,15 @@ __device__ __forceinline__ int token_block(const Geo& g, long long t) {
   const int lat = (int)(t / g.nlon), lon = (int)(t - (long long)lat * g.nlon);
   return (lat / g.bh) * g.nbw + lon / g.bw;
 }
-__device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
+__device__ __forceinline__ void unpack8(const Geo& g, const uint4& v, float (&f)[8]) {
   const uint32_t x[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    f[2 * i] = __uint_as_float(x[i] << 16);
-    f[2 * i + 1] = __uint_as_float(x[i] & 0xffff0000u);
-  }
+  for (int i = 0; i < 4; ++i) unpack16x2(x[i], g.f16 != 0, f[2 * i], f[2 * i + 1]);
 }
-__device__ __forceinline__ uint4 pack8(const float (&f)[8]) {
+__device__ __forceinline__ uint4 pack8(const Geo& g, const float (&f)[8]) {
   uint32_t r[4];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const __nv_bfloat162 p = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
-    r[i] = *reinterpret_cast<const uint32_t*>(&p);
-  }
+  for (int i = 0; i < 4; ++i) r[i] = pack16x2(f[2 * i], f[2 * i + 1], g.f16 != 0);
   return make_uint4(r[0], r[1], r[2], r[3]);
 }
 
@@ -63,9 +57,9 @@ __global__ void __launch_bounds__(256) gate_kernel(Geo g, const uint4* __restric
     const float4 c0 = __ldg(cg), c1 = __ldg(cg + 1);
     const float cgv[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
     float go[8], a[8], b[8], sf[8], sl[8];
-    unpack8(__ldg(d_o + x * 8 + part), go);
-    unpack8(__ldg(o_fg + x * 8 + part), a);
-    unpack8(__ldg(o_l + x * 8 + part), b);
+    unpack8(g, __ldg(d_o + x * 8 + part), go);
+    unpack8(g, __ldg(o_fg + x * 8 + part), a);
+    unpack8(g, __ldg(o_l + x * 8 + part), b);
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       dc = fmaf(go[i], cgv[i], dc);
@@ -74,8 +68,8 @@ __global__ void __launch_bounds__(256) gate_kernel(Geo g, const uint4* __restric
       sf[i] = gf * go[i];
       sl[i] = gl * go[i];
     }
-    do_fg[x * 8 + part] = pack8(sf);
-    do_l[x * 8 + part] = pack8(sl);
+    do_fg[x * 8 + part] = pack8(g, sf);
+    do_l[x * 8 + part] = pack8(g, sl);
   }
 #pragma unroll
   for (int o = 1; o < 8; o <<= 1) {
@@ -108,7 +102,7 @@ __global__ void __launch_bounds__(256) gated_pool_kernel(Geo g, const uint4* __r
     const long long t0 = (long long)u * g.N + (long long)(by * g.bh + r) * g.nlon + bx * g.bw;
     for (int c = 0; c < g.bw; ++c) {
       float go[8];
-      unpack8(__ldg(d_o + (t0 + c) * 8 + sub), go);
+      unpack8(g, __ldg(d_o + (t0 + c) * 8 + sub), go);
       const float gc = __ldg(gates + (t0 + c) * 3);
 #pragma unroll
       for (int e = 0; e < 8; ++e) acc[e] = fmaf(gc, go[e], acc[e]);
@@ -303,11 +297,11 @@ __global__ void __launch_bounds__(256) sum_kernel(Geo g, long long tokens, const
   const float4 c0 = __ldg(cm), c1 = __ldg(cm + 1);
   const float cv[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
   float a[8], b[8], r[8];
-  unpack8(__ldg(x_l + x * 8 + part), a);
-  if (x_fg) unpack8(__ldg(x_fg + x * 8 + part), b);
+  unpack8(g, __ldg(x_l + x * 8 + part), a);
+  if (x_fg) unpack8(g, __ldg(x_fg + x * 8 + part), b);
 #pragma unroll
   for (int i = 0; i < 8; ++i) r[i] = a[i] + (x_fg ? b[i] : 0.f) + cv[i];
-  out[x * 8 + part] = pack8(r);
+  out[x * 8 + part] = pack8(g, r);
 }
 
 }  // namespace

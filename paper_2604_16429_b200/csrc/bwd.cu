@@ -25,7 +25,7 @@ constexpr float kLog2e = 1.4426950408889634f;
 __global__ void __launch_bounds__(256) rowdot_kernel(long long tokens, const uint4* __restrict__ o,
                                                      const uint4* __restrict__ d_o, const float* __restrict__ lse,
                                                      float* __restrict__ D, float* __restrict__ neg_d,
-                                                     float* __restrict__ neg_lse2) {
+                                                     float* __restrict__ neg_lse2, bool f16) {
   long long t = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 3;
   int part = threadIdx.x & 7;
   float acc = 0.f;
@@ -34,8 +34,11 @@ __global__ void __launch_bounds__(256) rowdot_kernel(long long tokens, const uin
     const uint32_t av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      acc += __uint_as_float(av[i] << 16) * __uint_as_float(bv[i] << 16);
-      acc += __uint_as_float(av[i] & 0xffff0000u) * __uint_as_float(bv[i] & 0xffff0000u);
+      float a0, a1, b0, b1;
+      unpack16x2(av[i], f16, a0, a1);
+      unpack16x2(bv[i], f16, b0, b1);
+      acc += a0 * b0;
+      acc += a1 * b1;
     }
   }
   acc += __shfl_xor_sync(0xffffffffu, acc, 1);
@@ -153,7 +156,7 @@ int launch_bwd(const HostCtx& c, const void* q, const void* k, const void* v, co
   {
     long long threads = tokens * 8;
     rowdot_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, c.stream>>>(tokens, (const uint4*)o,
-                                                                           (const uint4*)d_o, lse, Dbuf, neg_d, neg_lse2);
+                                                                           (const uint4*)d_o, lse, Dbuf, neg_d, neg_lse2, g.f16 != 0);
     if (cudaGetLastError() != cudaSuccess) return MOSAIC_E_CUDA;
   }
   if (g.topk > 0) {

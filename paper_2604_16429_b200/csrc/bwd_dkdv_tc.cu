@@ -210,6 +210,7 @@ __global__ void __launch_bounds__(1024) dkdv_order_kernel(const Geo g, const int
     order[first_item + atomicAdd(&hist[bins[item]], 1)] = item;
 }
 
+template <bool F16>
 __global__ void __launch_bounds__(kThreads, 1)
     dkdv_tc_kernel(const Geo g, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_do,
                    const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
@@ -311,7 +312,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     // The buffers may be overwritten once the row threads hold the previous pair in registers, so this thread runs
     // one pair ahead of their arithmetic.
     if (lane == 0) {
-      constexpr uint32_t idesc1 = make_idesc(false, 64u), idesc2 = make_idesc(false, 128u);
+      constexpr uint32_t idesc1 = make_idesc(false, 64u, F16), idesc2 = make_idesc(false, 128u, F16);
       const uint64_t kdesc = smem_desc(s32(sm.k)), vdesc = smem_desc(s32(sm.v));
       long long pr = 0;
       int items = 0;
@@ -353,7 +354,7 @@ __global__ void __launch_bounds__(kThreads, 1)
   } else if (warp == kWMma1) {
     // ------------------------------------------------------------- issuer of dV += P^T dO and dK += dS^T Q (one thread)
     if (lane == 0) {
-      constexpr uint32_t idesc_nn = make_idesc(true);
+      constexpr uint32_t idesc_nn = make_idesc(true, 64u, F16);
       long long pr = 0;
       uint32_t jg[2] = {0u, 0u};  // products each group of row threads has handed over (phase of p_full)
       uint32_t items = 0;         // items whose accumulators have been handed to the row threads
@@ -470,10 +471,10 @@ __global__ void __launch_bounds__(kThreads, 1)
             const uint64_t t23 = add2(pack2(__uint_as_float(dp[i + 2]), __uint_as_float(dp[i + 3])), pack2(nd.z, nd.w));
             unpack2(mul2(pack2(e0, e1), t01), d0, d1);
             unpack2(mul2(pack2(e2, e3), t23), d2, d3);
-            pp[i >> 1] = bf16x2(e0, e1);
-            pp[(i >> 1) + 1] = bf16x2(e2, e3);
-            ds[i >> 1] = bf16x2(d0, d1);
-            ds[(i >> 1) + 1] = bf16x2(d2, d3);
+            pp[i >> 1] = pack2<F16>(e0, e1);
+            pp[(i >> 1) + 1] = pack2<F16>(e2, e3);
+            ds[i >> 1] = pack2<F16>(d0, d1);
+            ds[(i >> 1) + 1] = pack2<F16>(d2, d3);
           }
         } else {
           tc_fence_before();
@@ -514,7 +515,7 @@ __global__ void __launch_bounds__(kThreads, 1)
               uint32_t w[8];
 #pragma unroll
               for (int i = 0; i < 8; ++i)
-                w[i] = bf16x2(__uint_as_float(ov[2 * i]) * f, __uint_as_float(ov[2 * i + 1]) * f);
+                w[i] = pack2<F16>(__uint_as_float(ov[2 * i]) * f, __uint_as_float(ov[2 * i + 1]) * f);
               dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
               dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
             }
@@ -545,7 +546,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 }
 
 // `work_counter` must be zero when the kernel starts (a word of the workspace status block).
-int launch_dkdv_tc(const HostCtx& c, const void* q, const void* k, const void* v, const void* d_o,
+template <bool F16>
+static int launch_dkdv_tc_t(const HostCtx& c, const void* q, const void* k, const void* v, const void* d_o,
                    const float* neg_lse2, const float* neg_d, const int32_t* csr_off, const int32_t* csr_q, void* dk,
                    void* dv, int* work_counter, int32_t* order) {
   const Geo& g = c.g;
@@ -556,7 +558,7 @@ int launch_dkdv_tc(const HostCtx& c, const void* q, const void* k, const void* v
   const size_t smem = sizeof(Smem) + 1024;
   static unsigned long long configured = 0;  // devices on which the kernel's shared-memory opt-in is set
   int sms = 0;
-  if (const int rc = launch_setup(reinterpret_cast<const void*>(dkdv_tc_kernel), smem, &configured, &sms)) return rc;
+  if (const int rc = launch_setup(reinterpret_cast<const void*>(dkdv_tc_kernel<F16>), smem, &configured, &sms)) return rc;
   const int ipu = items_per_unit(g);
   const long long total = 2ll * g.Ukv * ipu;  // one item per 128-row tile of a key/value unit
   if (total > 0x7fffff00ll) return MOSAIC_E_UNSUPPORTED;
@@ -571,10 +573,16 @@ int launch_dkdv_tc(const HostCtx& c, const void* q, const void* k, const void* v
   dkdv_order_kernel<<<(unsigned)((total + win_items - 1) / win_items), 1024, 0, c.stream>>>(
       g, csr_off, ipu, (int)total, (int)win_items, order, order + total);
   if (cudaGetLastError() != cudaSuccess) return MOSAIC_E_CUDA;
-  dkdv_tc_kernel<<<(unsigned)grid, kThreads, smem, c.stream>>>(g, mq, mdo, mk, mv, mnl, mnd, csr_off, csr_q, order,
+  dkdv_tc_kernel<F16><<<(unsigned)grid, kThreads, smem, c.stream>>>(g, mq, mdo, mk, mv, mnl, mnd, csr_off, csr_q, order,
                                                                (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, c.status,
                                                                work_counter, ipu, (int)total);
   return cudaGetLastError() == cudaSuccess ? MOSAIC_OK : MOSAIC_E_CUDA;
+}
+
+int launch_dkdv_tc(const HostCtx& c, const void* q, const void* k, const void* v, const void* d_o,
+                   const float* neg_lse2, const float* neg_d, const int32_t* csr_off, const int32_t* csr_q, void* dk,
+                   void* dv, int* work_counter, int32_t* order) {
+  return c.g.f16 ? launch_dkdv_tc_t<true>(c, q, k, v, d_o, neg_lse2, neg_d, csr_off, csr_q, dk, dv, work_counter, order) : launch_dkdv_tc_t<false>(c, q, k, v, d_o, neg_lse2, neg_d, csr_off, csr_q, dk, dv, work_counter, order);
 }
 
 }  // namespace mosaic

@@ -46,6 +46,7 @@ struct Smem {
 
 }  // namespace
 
+template <bool F16>
 __global__ void __launch_bounds__(kThreads, 1)
     dq_tc_kernel(const Geo g, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_do,
                  const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
@@ -134,7 +135,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     // ------------------------------------------------------------- MMA issuer of tile t
     // The whole warp walks the loop; one elected lane issues the tensor-core instructions.
     const int t = warp - 9;
-    constexpr uint32_t idesc_nt = make_idesc(false), idesc_nn = make_idesc(true);
+    constexpr uint32_t idesc_nt = make_idesc(false, 64u, F16), idesc_nn = make_idesc(true, 64u, F16);
     const uint64_t qdesc = smem_desc(s32(sm.q[t])), dodesc = smem_desc(s32(sm.d_o[t]));
     const uint32_t tcol_dq = tmem + kColDQ + 64 * t, tcol_s = tmem + kColS + 128 * t, tcol_dp = tcol_s + 64;
     const uint32_t tcol_ds = tmem + kColDS + 32 * t;
@@ -267,7 +268,7 @@ __global__ void __launch_bounds__(kThreads, 1)
               unpack2(fma2(pack2(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])), scale2, neg_lse2), x0, x1);
               const uint64_t dmd = add2(pack2(__uint_as_float(dp[i]), __uint_as_float(dp[i + 1])), neg_d2);
               unpack2(mul2(pack2(ex2(x0), ex2(x1)), dmd), d0, d1);
-              pk[i >> 1] = bf16x2(d0, d1);
+              pk[i >> 1] = pack2<F16>(d0, d1);
             }
           } else {
             tc_fence_before();
@@ -306,7 +307,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             uint32_t w[16];
 #pragma unroll
             for (int i = 0; i < 16; ++i)
-              w[i] = bf16x2(__uint_as_float(ov[2 * i]) * g.scale, __uint_as_float(ov[2 * i + 1]) * g.scale);
+              w[i] = pack2<F16>(__uint_as_float(ov[2 * i]) * g.scale, __uint_as_float(ov[2 * i + 1]) * g.scale);
 #pragma unroll
             for (int i = 0; i < 4; ++i)
               dst[part * 4 + i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
@@ -327,7 +328,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 }
 
 // `work_counter` must be zero when the kernel starts (a word of the workspace status block).
-int launch_dq_tc(const HostCtx& c, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
+template <bool F16>
+static int launch_dq_tc_t(const HostCtx& c, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
                  const float* D, const int32_t* block_idx, void* dq, int* work_counter) {
   const Geo& g = c.g;
   CUtensorMap mq, mdo, mk, mv;
@@ -336,15 +338,20 @@ int launch_dq_tc(const HostCtx& c, const void* q, const void* k, const void* v, 
   const size_t smem = sizeof(Smem) + 1024;
   static unsigned long long configured = 0;  // devices on which the kernel's shared-memory opt-in is set
   int sms = 0;
-  if (const int rc = launch_setup(reinterpret_cast<const void*>(dq_tc_kernel), smem, &configured, &sms)) return rc;
+  if (const int rc = launch_setup(reinterpret_cast<const void*>(dq_tc_kernel<F16>), smem, &configured, &sms)) return rc;
   const int ipu = items_per_unit(g);
   const long long total = (long long)g.U * ipu;
   if (total > 0x7fffff00ll) return MOSAIC_E_UNSUPPORTED;
   const long long grid = total < (long long)sms ? total : (long long)sms;
-  dq_tc_kernel<<<(unsigned)grid, kThreads, smem, c.stream>>>(g, mq, mdo, mk, mv, block_idx, lse, D,
+  dq_tc_kernel<F16><<<(unsigned)grid, kThreads, smem, c.stream>>>(g, mq, mdo, mk, mv, block_idx, lse, D,
                                                              (__nv_bfloat16*)dq, c.status, work_counter, ipu,
                                                              (int)total);
   return cudaGetLastError() == cudaSuccess ? MOSAIC_OK : MOSAIC_E_CUDA;
+}
+
+int launch_dq_tc(const HostCtx& c, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
+                 const float* D, const int32_t* block_idx, void* dq, int* work_counter) {
+  return c.g.f16 ? launch_dq_tc_t<true>(c, q, k, v, d_o, lse, D, block_idx, dq, work_counter) : launch_dq_tc_t<false>(c, q, k, v, d_o, lse, D, block_idx, dq, work_counter);
 }
 
 }  // namespace mosaic

@@ -1,5 +1,7 @@
 // Shared device/host definitions of the MOSAIC block-sparse attention kernels (sm_100a).
 #pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -27,6 +29,7 @@ struct Geo {
   int rlat, rlon, topk;
   int local_off;    // 1: the local neighbourhood is not attended (selection branch of the three-branch form)
   int local_groups; // 1: the local set is the aligned group of rlat x rlon blocks that holds the block
+  int f16;          // 1: the 16-bit tensors are IEEE binary16, 0: bf16
   float scale;      // softmax scale
   float scale_log2; // scale * log2(e)
   long long N;      // tokens per unit
@@ -36,6 +39,26 @@ struct Geo {
 __host__ __device__ __forceinline__ int kv_unit(const Geo& g, int u) {
   const int b = u / g.H;
   return b * g.Hkv + (u - b * g.H) / (g.H / g.Hkv);
+}
+
+// Two 16-bit elements of the problem's storage type (bf16 or binary16) packed in a word <-> two floats.
+__device__ __forceinline__ void unpack16x2(uint32_t x, bool f16, float& lo, float& hi) {
+  if (f16) {
+    const float2 v = __half22float2(*reinterpret_cast<const __half2*>(&x));
+    lo = v.x;
+    hi = v.y;
+  } else {
+    lo = __uint_as_float(x << 16);
+    hi = __uint_as_float(x & 0xffff0000u);
+  }
+}
+__device__ __forceinline__ uint32_t pack16x2(float lo, float hi, bool f16) {
+  if (f16) {
+    const __half2 v = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&v);
+  }
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
 }
 
 // Record the first device-side fault in the workspace status word (never traps).

@@ -70,6 +70,7 @@ struct Smem {
 
 }  // namespace
 
+template <bool F16>
 __global__ void __launch_bounds__(kThreads, 1)
     fwd_tc_kernel(const Geo g, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_v, const int32_t* __restrict__ block_idx,
@@ -169,7 +170,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     // S is double-buffered: QK^T of product n+1 is issued before P V of product n, so the tensor core
     // fills the next S while the softmax warps work on the current one.
     const int t = warp - 9;
-    constexpr uint32_t idesc_qk = make_idesc(false), idesc_pv = make_idesc(true);
+    constexpr uint32_t idesc_qk = make_idesc(false, 64u, F16), idesc_pv = make_idesc(true, 64u, F16);
     const uint32_t tcol_o = tmem + kColO + 64 * t, tcol_s = tmem + kColS + 128 * t, tcol_q = tmem + kColQ + 32 * t;
     const uint32_t tbits = 3u << (2 * t);
     long long step = 0;   // ring position (all chunks, attended by this tile or not)
@@ -332,8 +333,8 @@ __global__ void __launch_bounds__(kThreads, 1)
               if ((i >> 2) % kPolyEvery == kPolyEvery - 1) { ex2_poly2(y23, p2, p3); } else { p2 = ex2(x2); p3 = ex2(x3); }
               sum_a = add2(sum_a, pack2(p0, p1));
               sum_b = add2(sum_b, pack2(p2, p3));
-              pk[i >> 1] = bf16x2(p0, p1);
-              pk[(i >> 1) + 1] = bf16x2(p2, p3);
+              pk[i >> 1] = pack2<F16>(p0, p1);
+              pk[(i >> 1) + 1] = pack2<F16>(p2, p3);
             }
 #pragma unroll
             for (int i = 0; i < 32; i += 4) {
@@ -346,8 +347,8 @@ __global__ void __launch_bounds__(kThreads, 1)
               if ((i >> 2) % kPolyEvery == kPolyEvery - 1) { ex2_poly2(y23, p2, p3); } else { p2 = ex2(x2); p3 = ex2(x3); }
               sum_a = add2(sum_a, pack2(p0, p1));
               sum_b = add2(sum_b, pack2(p2, p3));
-              pk[16 + (i >> 1)] = bf16x2(p0, p1);
-              pk[16 + (i >> 1) + 1] = bf16x2(p2, p3);
+              pk[16 + (i >> 1)] = pack2<F16>(p0, p1);
+              pk[16 + (i >> 1) + 1] = pack2<F16>(p2, p3);
             }
             tmem_st32(tsb, pk);  // P (bf16 pairs) over the first 32 columns of this S buffer
             float s0, s1;
@@ -414,7 +415,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             uint32_t w[16];
 #pragma unroll
             for (int i = 0; i < 16; ++i)
-              w[i] = bf16x2(__uint_as_float(ov[2 * i]) * inv, __uint_as_float(ov[2 * i + 1]) * inv);
+              w[i] = pack2<F16>(__uint_as_float(ov[2 * i]) * inv, __uint_as_float(ov[2 * i + 1]) * inv);
 #pragma unroll
             for (int i = 0; i < 4; ++i)
               dst[part * 4 + i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
@@ -440,23 +441,33 @@ __global__ void __launch_bounds__(kThreads, 1)
 }
 
 // ---------------------------------------------------------------------------------------------
+namespace {
+template <bool F16>
+int launch_fwd_tc_t(const HostCtx& c, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+                    const int32_t* block_idx, void* o, float* lse, int* work_counter) {
+  const Geo& g = c.g;
+  const size_t smem = sizeof(Smem) + 1024;
+  static unsigned long long configured = 0;  // devices on which the kernel's shared-memory opt-in is set
+  int sms = 0;
+  if (const int rc = launch_setup(reinterpret_cast<const void*>(fwd_tc_kernel<F16>), smem, &configured, &sms)) return rc;
+  const int ipu = items_per_unit(g);
+  const long long total = (long long)g.U * ipu;
+  if (total > 0x7fffff00ll) return MOSAIC_E_UNSUPPORTED;
+  const long long grid = total < (long long)sms ? total : (long long)sms;
+  fwd_tc_kernel<F16><<<(unsigned)grid, kThreads, smem, c.stream>>>(g, mq, mk, mv, block_idx, (__nv_bfloat16*)o, lse,
+                                                                  c.status, work_counter, ipu, (int)total);
+  return cudaGetLastError() == cudaSuccess ? MOSAIC_OK : MOSAIC_E_CUDA;
+}
+}  // namespace
+
 // `work_counter` must be zero when the kernel starts (a word of the workspace status block).
 int launch_fwd_tc(const HostCtx& c, const void* q, const void* k, const void* v, const int32_t* block_idx, void* o,
                   float* lse, int* work_counter) {
   const Geo& g = c.g;
   CUtensorMap mq, mk, mv;
   if (!make_map(&mq, q, g, g.U) || !make_map(&mk, k, g, g.Ukv) || !make_map(&mv, v, g, g.Ukv)) return MOSAIC_E_CUDA;
-  const size_t smem = sizeof(Smem) + 1024;
-  static unsigned long long configured = 0;  // devices on which the kernel's shared-memory opt-in is set
-  int sms = 0;
-  if (const int rc = launch_setup(reinterpret_cast<const void*>(fwd_tc_kernel), smem, &configured, &sms)) return rc;
-  const int ipu = items_per_unit(g);
-  const long long total = (long long)g.U * ipu;
-  if (total > 0x7fffff00ll) return MOSAIC_E_UNSUPPORTED;
-  const long long grid = total < (long long)sms ? total : (long long)sms;
-  fwd_tc_kernel<<<(unsigned)grid, kThreads, smem, c.stream>>>(g, mq, mk, mv, block_idx, (__nv_bfloat16*)o, lse,
-                                                             c.status, work_counter, ipu, (int)total);
-  return cudaGetLastError() == cudaSuccess ? MOSAIC_OK : MOSAIC_E_CUDA;
+  return g.f16 ? launch_fwd_tc_t<true>(c, mq, mk, mv, block_idx, o, lse, work_counter)
+               : launch_fwd_tc_t<false>(c, mq, mk, mv, block_idx, o, lse, work_counter);
 }
 
 }  // namespace mosaic

@@ -7,7 +7,7 @@
 //
 // HBM-bound: every element of Q and K is read and written once.  Eight lanes per token, a lane owns eight channels
 // (four pairs, 16 bytes) and walks all units of both tensors with the same four (cos, sin), which it computes once
-// in fp64; the rotation is fp64 too (a few fp64 FMAs per 16 bytes moved), rounded to fp32 and then to bf16.
+// in fp64; the rotation is fp64 too (a few fp64 FMAs per 16 bytes moved), rounded to fp32 and then to the storage type.
 #include <cuda_bf16.h>
 
 #include "common.cuh"
@@ -16,15 +16,16 @@ namespace mosaic {
 
 namespace {
 
-__device__ __forceinline__ uint4 rotate8(const uint4& v, const double (&c)[4], const double (&s)[4]) {
+__device__ __forceinline__ uint4 rotate8(const uint4& v, const double (&c)[4], const double (&s)[4], bool f16) {
   const uint32_t x[4] = {v.x, v.y, v.z, v.w};
   uint32_t r[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    const double x0 = (double)__uint_as_float(x[i] << 16), x1 = (double)__uint_as_float(x[i] & 0xffff0000u);
+    float lo, hi;
+    unpack16x2(x[i], f16, lo, hi);
+    const double x0 = (double)lo, x1 = (double)hi;
     const float y0 = __double2float_rn(x0 * c[i] - x1 * s[i]), y1 = __double2float_rn(x0 * s[i] + x1 * c[i]);
-    const __nv_bfloat162 p = __floats2bfloat162_rn(y0, y1);
-    r[i] = *reinterpret_cast<const uint32_t*>(&p);
+    r[i] = pack16x2(y0, y1, f16);
   }
   return make_uint4(r[0], r[1], r[2], r[3]);
 }
@@ -44,11 +45,11 @@ __global__ void __launch_bounds__(256) rope_kernel(Geo g, const uint4* __restric
   }
   for (int u = 0; u < g.U; ++u) {
     const long long at = ((long long)u * g.N + x) * 8 + part;
-    q_out[at] = rotate8(__ldg(q + at), c, s);
+    q_out[at] = rotate8(__ldg(q + at), c, s, g.f16 != 0);
   }
   for (int u = 0; u < g.Ukv; ++u) {
     const long long at = ((long long)u * g.N + x) * 8 + part;
-    k_out[at] = rotate8(__ldg(k + at), c, s);
+    k_out[at] = rotate8(__ldg(k + at), c, s, g.f16 != 0);
   }
 }
 

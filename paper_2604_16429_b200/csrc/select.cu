@@ -46,8 +46,10 @@ __global__ void __launch_bounds__(256) pool_kernel(Geo g, const uint4* __restric
       const uint32_t x[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        acc[2 * e] += (double)__uint_as_float(x[e] << 16);
-        acc[2 * e + 1] += (double)__uint_as_float(x[e] & 0xffff0000u);
+        float lo, hi;
+        unpack16x2(x[e], g.f16 != 0, lo, hi);
+        acc[2 * e] += (double)lo;
+        acc[2 * e + 1] += (double)hi;
       }
     }
   }

@@ -263,9 +263,12 @@ __device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
   asm("mul.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
 }
-__device__ __forceinline__ uint32_t bf16x2(float lo, float hi) {
+// two floats -> two 16-bit operands in one word (bf16, or binary16 when F16)
+template <bool F16>
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   uint32_t r;
-  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  if (F16) asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  else asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
   return r;
 }
 
@@ -299,10 +302,11 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
   d |= (uint64_t)2 << 61;               // SWIZZLE_128B
   return d;
 }
-// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 64 unless given.
-__host__ __device__ constexpr uint32_t make_idesc(bool b_mn_major, uint32_t n = 64u) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((n >> 3) << 17) |
-         ((128u >> 4) << 24);
+// Instruction descriptor: 16-bit x 16-bit -> fp32 (both operands bf16, or both binary16 when f16), M = 128,
+// N = 64 unless given.
+__host__ __device__ constexpr uint32_t make_idesc(bool b_mn_major, uint32_t n = 64u, bool f16 = false) {
+  return (1u << 4) | ((f16 ? 0u : 1u) << 7) | ((f16 ? 0u : 1u) << 10) | ((b_mn_major ? 1u : 0u) << 16) |
+         ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
 
 // The four halves of work item `it` (index inside the unit).  Missing halves repeat half 0 (their rows

@@ -44,11 +44,11 @@ class Guarded:
 
 def geom_of(w, scale=0.0) -> Geom:
     return Geom(w.nlat, w.nlon, d=w.d, bh=w.bh, bw=w.bw, rlat=w.rlat, rlon=w.rlon, topk=w.topk, scale=scale,
-                local_groups=getattr(w, "local_groups", False))
+                local_groups=getattr(w, "local_groups", False), f16=getattr(w, "f16", False))
 
 
-def device_inputs(x: dict) -> dict:
-    return {k: mb.from_bits(v) for k, v in x.items()}
+def device_inputs(x: dict, f16=False) -> dict:
+    return {k: mb.from_bits(v, f16=f16) for k, v in x.items()}
 
 
 def oracle_select_all(w, x) -> np.ndarray:
@@ -73,7 +73,7 @@ def gpu_select(w, dx, scale=0.0):
 def gpu_fwd(w, dx, idx, scale=0.0):
     p = mb.Params.from_workload(w, scale=scale)
     ws = Guarded((mb.workspace_bytes(p, mb.OP_FWD),), torch.uint8)
-    o = Guarded(tuple(dx["q"].shape), torch.bfloat16, fill=float("nan"))
+    o = Guarded(tuple(dx["q"].shape), dx["q"].dtype, fill=float("nan"))
     lse = Guarded((w.B, w.H, w.N), torch.float32, fill=float("nan"))
     mb.mosaic_bsa_fwd(p, dx["q"], dx["k"], dx["v"], idx, o=o.t, lse=lse.t, ws=ws.t)
     mb.check_status(ws.t, "fwd")
@@ -84,7 +84,7 @@ def gpu_fwd(w, dx, idx, scale=0.0):
 def gpu_bwd(w, dx, o, lse, idx, scale=0.0):
     p = mb.Params.from_workload(w, scale=scale)
     ws = Guarded((mb.workspace_bytes(p, mb.OP_BWD),), torch.uint8)
-    outs = [Guarded(tuple(dx["q"].shape), torch.bfloat16, fill=float("nan")) for _ in range(3)]
+    outs = [Guarded(tuple(dx[n].shape), dx["q"].dtype, fill=float("nan")) for n in ("q", "k", "k")]
     mb.mosaic_bsa_bwd(p, dx["q"], dx["k"], dx["v"], o, lse, dx["do"], idx, dq=outs[0].t, dk=outs[1].t,
                       dv=outs[2].t, ws=ws.t)
     mb.check_status(ws.t, "bwd")

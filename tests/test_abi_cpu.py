@@ -41,7 +41,7 @@ def test_workspace_sizes():
     (dict(nlat=121), -1),            # grid not divisible by the block
     (dict(topk=-1), -1),
     (dict(B=0), -1),
-    (dict(flags=2), -1),             # unknown flag bit
+    (dict(flags=4), -1),             # unknown flag bit
     (dict(flags=1, rlat=0), -1),     # group mode needs a group of at least one block
     (dict(flags=1, rlat=8, rlon=8), -2),
     (dict(d=32), -2),                # unsupported head dimension

@@ -43,10 +43,12 @@ __global__ void __launch_bounds__(256) rope_kernel(Geo g, const uint4* __restric
     const int i = 4 * (part & 3) + j;                         // pair inside the half, D = kD / 2
     sincos(p * pow(theta, -2.0 * i / (kD / 2)), &s[j], &c[j]);
   }
+#pragma unroll 4
   for (int u = 0; u < g.U; ++u) {
     const long long at = ((long long)u * g.N + x) * 8 + part;
     q_out[at] = rotate8(__ldg(q + at), c, s, g.f16 != 0);
   }
+#pragma unroll 4
   for (int u = 0; u < g.Ukv; ++u) {
     const long long at = ((long long)u * g.N + x) * 8 + part;
     k_out[at] = rotate8(__ldg(k + at), c, s, g.f16 != 0);

@@ -187,3 +187,40 @@ def test_three_branch_backward_one_branch_at_a_time_and_empty_rows():
             assert np.all(got[0][0, 0][tok5] == 0)
             tu = oracle.block_tokens(G.geom_of(w), j0)
             assert np.all(got[1][0, 0][tu] == 0) and np.all(got[2][0, 0][tu] == 0)
+
+
+def test_three_branch_backward_at_the_papers_stage_three_shape_in_binary16():
+    """The whole stage-3 problem (nside 16: N = 3072, 20 heads, 128-token blocks in 1024-token local groups, 4 selected
+    blocks) with the paper's GQA ratio 4 and binary16 storage, as one launch sequence; two heads of two different
+    key/value heads against the oracle."""
+    base = synth.WORKLOADS["hp_nside16"]
+    w = synth.Workload(**{**base.__dict__, "name": "hp_nside16_gqa_f16", "Hkv": 5, "f16": True, "backward": True})
+    x = synth.make_inputs(w)
+    dx = G.device_inputs(x, f16=True)
+    p = mb.Params.from_workload(w)
+    idx = G.gpu_select(w, dx)
+    idx_h = idx.cpu().numpy()
+    gates = np.random.default_rng(96).standard_normal((w.B, w.H, w.N, 3))
+    gt = torch.from_numpy(gates.astype(np.float32)).cuda()
+    ws = G.Guarded((mb.workspace_bytes(p, mb.OP_BWD_BRANCHES),), torch.uint8)
+    dq, dk, dv, dg = mb.mosaic_bsa_bwd_branches(p, dx["q"], dx["k"], dx["v"], idx, gt, dx["do"], ws=ws.t)
+    mb.check_status(ws.t, "bwd_branches")
+    ws.check("workspace")
+    assert all(torch.isfinite(t.float()).all() for t in (dq, dk, dv, dg))
+    g = G.geom_of(w)
+    r = w.H // w.kv_heads
+    for hk in (0, 4):
+        dK_sum, dV_sum = np.zeros((w.N, w.d)), np.zeros((w.N, w.d))
+        for h in range(hk * r, (hk + 1) * r):
+            assert np.array_equal(idx_h[0, h], oracle.select(g, x["q"][0, h], x["k"][0, hk]))
+            gq = gates[0, h].astype(np.float32).astype(np.float64)
+            dQ, dK, dV, dG = oracle.bwd3(g, x["q"][0, h], x["k"][0, hk], x["v"][0, hk], x["do"][0, h], idx_h[0, h], gq)
+            tol = G.BWD_MAX_ABS + 2.0 ** -8 * np.abs(dQ).max()
+            assert np.abs(dq[0, h].float().cpu().numpy() - dQ).max() <= tol
+            do_abs = np.abs(oracle.widen16(g, x["do"][0, h])).sum(axis=-1)
+            assert (np.abs(dg[0, h].cpu().numpy() - dG) <= 4 * G.FWD_MEAN_ABS * do_abs[:, None] + 1e-3).all()
+            dK_sum += dK
+            dV_sum += dV
+        for name, a, ref in (("dK", dk, dK_sum), ("dV", dv, dV_sum)):
+            tol = G.BWD_MAX_ABS + 2.0 ** -8 * np.abs(ref).max()
+            assert np.abs(a[0, hk].float().cpu().numpy() - ref).max() <= tol, name

@@ -117,7 +117,6 @@ __device__ __forceinline__ float from_ordered_bits(unsigned o) {
 }
 
 constexpr int kKStr = kD + 4;   // padded row of the staged vectors (floats): 16-byte reads of one row per lane hit every bank once
-constexpr int kExact = 64;      // most survivors of a row that the counting rank handles (more: insertion path)
 
 template <int NW, int RI, int CAP, int JT>
 struct TopkSmem {
@@ -126,7 +125,7 @@ struct TopkSmem {
       float ks[2][JT][kKStr];  // pooled keys of two chunks (one being read, one in flight)
       float nk[2][JT];         // their norm bounds
     } scr;
-    unsigned long long ekey[NW * RI][kExact];  // exact phase: score keys of the rows' survivors
+    unsigned long long ekey[NW * RI][CAP];  // exact phase: score keys of the rows' survivors (every row that did not overflow)
   };
   float qs[NW * RI][kKStr];     // pooled queries of this CTA
   int surv[NW * RI][CAP];       // surviving key ids per row ...
@@ -423,11 +422,11 @@ __global__ void __launch_bounds__(NW * 32, MB) topk_kernel(Geo g, const float* _
   // rows whose survivors fit the counting rank: flatten (row, entry) pairs over the lanes, two chains in flight
   int base_of[RI + 1];
   base_of[0] = 0;
-  unsigned slow = 0;  // rows that take the insertion path (more than kExact survivors, or overflowed)
+  unsigned slow = 0;  // rows that take the insertion path (their survivors overflowed)
 #pragma unroll
   for (int a = 0; a < RI; ++a) {
     const bool row_ok = i0 + warp * RI + a < g.m;
-    const bool fast = row_ok && cnt[a] <= kExact;
+    const bool fast = row_ok && cnt[a] <= CAP;
     if (row_ok && !fast) slow |= 1u << a;
     base_of[a + 1] = base_of[a] + (fast ? cnt[a] : 0);
   }
@@ -472,25 +471,18 @@ __global__ void __launch_bounds__(NW * 32, MB) topk_kernel(Geo g, const float* _
     } else {
       unsigned long long lkey = 0ull;
       int lid = -1;
-      if (cnt[a] <= CAP) {
-        for (int e0 = 0; e0 < cnt[a]; e0 += 32) {
-          const int e = e0 + lane;
-          const int j = e < cnt[a] ? sm.surv[row][e] : -1;
-          insert_batch(j >= 0 ? exact_key(sm.qs[row], pk_u, j) : 0ull, j, lkey, lid, g.topk, lane);
+      // too many survivors to hold: score every key of the unit
+      for (int jb = 0; jb < g.m; jb += 32) {
+        const int j = jb + lane;
+        bool cand = j < g.m;
+        if (cand) {
+          const int jy = j / g.nbw, jx = j - jy * g.nbw;
+          int dx = jx - ix[a];
+          dx += dx < 0 ? g.nbw : 0;
+          cand = g.local_groups ? !(jy / g.rlat == iy[a] / g.rlat && jx / g.rlon == ix[a] / g.rlon)
+                                : !(abs(jy - iy[a]) <= g.rlat && (dx <= g.rlon || g.nbw - dx <= g.rlon));
         }
-      } else {  // too many survivors to hold: score every key of the unit
-        for (int jb = 0; jb < g.m; jb += 32) {
-          const int j = jb + lane;
-          bool cand = j < g.m;
-          if (cand) {
-            const int jy = j / g.nbw, jx = j - jy * g.nbw;
-            int dx = jx - ix[a];
-            dx += dx < 0 ? g.nbw : 0;
-            cand = g.local_groups ? !(jy / g.rlat == iy[a] / g.rlat && jx / g.rlon == ix[a] / g.rlon)
-                                  : !(abs(jy - iy[a]) <= g.rlat && (dx <= g.rlon || g.nbw - dx <= g.rlon));
-          }
-          insert_batch(cand ? exact_key(sm.qs[row], pk_u, j) : 0ull, j, lkey, lid, g.topk, lane);
-        }
+        insert_batch(cand ? exact_key(sm.qs[row], pk_u, j) : 0ull, j, lkey, lid, g.topk, lane);
       }
       if (lane < g.topk) out[lane] = lkey != 0ull ? lid : -1;
     }
@@ -550,12 +542,19 @@ int launch_select(const HostCtx& c, const void* q, const void* k, int32_t* block
   }
   if (g.topk > 0) {
     // the most query blocks per CTA (64, 32, 16) that still gives every SM about two CTAs; small problems are
-    // latency-bound and take 8 rows per CTA and 64-key chunks, so that more warps are resident
+    // latency-bound and take 8 rows per CTA and 64-key chunks, so that more warps are resident.  The survivors of a
+    // row grow with top-k (the threshold is the k-th best of 64 tracked bounds), and a row whose survivors overflow
+    // scores every key exactly: beyond top-k 16 only the configurations with room for 192 survivors are used.
     auto ctas = [&](int ti) { return (long long)g.U * ((g.m + ti - 1) / ti); };
-    const int rc = ctas(64) >= 296   ? launch_topk<8, 4, 96, 64, 3>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx)
-                   : ctas(32) >= 296 ? launch_topk<4, 8, 128, 128, 1>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx)
-                   : ctas(16) >= 296 ? launch_topk<4, 4, 192, 128, 2>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx)
-                                     : launch_topk<4, 2, 96, 64, 4>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx);
+    int rc;
+    if (g.topk > 16)
+      rc = ctas(16) >= 296 ? launch_topk<4, 4, 192, 128, 2>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx)
+                           : launch_topk<4, 2, 192, 64, 4>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx);
+    else
+      rc = ctas(64) >= 296   ? launch_topk<8, 4, 96, 64, 3>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx)
+           : ctas(32) >= 296 ? launch_topk<4, 8, 128, 128, 1>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx)
+           : ctas(16) >= 296 ? launch_topk<4, 4, 192, 128, 2>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx)
+                             : launch_topk<4, 2, 192, 64, 4>(c, pooled_q, pooled_k, norm_q, norm_k, block_idx);
     if (rc) return rc;
   }
   return MOSAIC_OK;

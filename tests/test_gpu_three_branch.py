@@ -224,3 +224,36 @@ def test_three_branch_backward_at_the_papers_stage_three_shape_in_binary16():
         for name, a, ref in (("dK", dk, dK_sum), ("dV", dv, dV_sum)):
             tol = G.BWD_MAX_ABS + 2.0 ** -8 * np.abs(ref).max()
             assert np.abs(a[0, hk].float().cpu().numpy() - ref).max() <= tol, name
+
+
+def test_three_branch_backward_without_selection_and_at_the_1p5_degree_size():
+    """Top-k 0: the selection branch is absent, its gate gradient is zero and the other two branches carry the whole
+    gradient.  Then the whole 1.5-degree problem as one launch sequence, two units against the oracle."""
+    w0 = synth.small_case(48, 64, 8, 8, 0, B=1, H=2, seed=97, backward=True)
+    x0 = synth.make_inputs(w0)
+    idx0 = torch.zeros((w0.B, w0.H, w0.m, 0), dtype=torch.int32, device="cuda")
+    gates0 = np.random.default_rng(97).standard_normal((w0.B, w0.H, w0.N, 3))
+    got0 = _run_bwd3(w0, x0, idx0, gates0)
+    _compare_bwd3(w0, x0, idx0.cpu().numpy(), gates0, got0)
+    assert np.all(got0[3][..., 1] == 0)
+
+    base = synth.WORKLOADS["c2_1p5deg"]
+    w = synth.Workload(**{**base.__dict__, "backward": True})
+    x = synth.make_inputs(w)
+    dx = G.device_inputs(x)
+    p = mb.Params.from_workload(w)
+    idx = G.gpu_select(w, dx)
+    idx_h = idx.cpu().numpy()
+    gates = np.random.default_rng(98).standard_normal((w.B, w.H, w.N, 3))
+    gt = torch.from_numpy(gates.astype(np.float32)).cuda()
+    dq, dk, dv, dg = mb.mosaic_bsa_bwd_branches(p, dx["q"], dx["k"], dx["v"], idx, gt, dx["do"])
+    assert all(torch.isfinite(t.float()).all() for t in (dq, dk, dv, dg))
+    g = G.geom_of(w)
+    for h in (1, 6):
+        gq = gates[0, h].astype(np.float32).astype(np.float64)
+        dQ, dK, dV, dG = oracle.bwd3(g, x["q"][0, h], x["k"][0, h], x["v"][0, h], x["do"][0, h], idx_h[0, h], gq)
+        for name, a, ref in (("dQ", dq, dQ), ("dK", dk, dK), ("dV", dv, dV)):
+            tol = G.BWD_MAX_ABS + 2.0 ** -8 * np.abs(ref).max()
+            assert np.abs(a[0, h].float().cpu().numpy() - ref).max() <= tol, (name, h)
+        do_abs = np.abs(synth.bf16_bits_to_f32(x["do"][0, h]).astype(np.float64)).sum(axis=-1)
+        assert (np.abs(dg[0, h].cpu().numpy() - dG) <= 4 * G.FWD_MEAN_ABS * do_abs[:, None] + 1e-3).all()
